@@ -1,0 +1,174 @@
+/*
+ * okq — 2-bit KV-cache quantisation and fused decode attention (OmniKVQuant hot path)
+ * for NVIDIA B200 (sm_100a).  Plain C ABI: device pointers, sizes, a CUDA stream passed
+ * as void*.  The library allocates no device memory, keeps no global state (other than
+ * the per-thread record of the last CUDA error), launches asynchronously on the given
+ * stream and never aborts the process.
+ *
+ * Conventions
+ *   - Every pointer inside okq_cache and every tensor argument is a DEVICE pointer owned
+ *     by the caller, aligned to 16 bytes.  `const okq_cache*` itself and `strides` are
+ *     HOST pointers, read before the call returns.
+ *   - head_dim is 128, the key window is 32 tokens, codes are 2 bits; anything else is
+ *     OKQ_ERR_UNSUPPORTED.  The GQA group n_q_heads / n_kv_heads must be an integer <= 8.
+ *   - Modality ids: 0 text, 1 audio, 2 video (the paper's set {V, A, L}).
+ *   - Errors that the host can see (null or misaligned pointers, bad shapes, workspace
+ *     too small) are returned before anything is launched.  Errors only the device can
+ *     see (a sequence would grow past `capacity`) set the cache's device status word to a
+ *     non-zero okq_status and skip the write; the caller reads the word when it next
+ *     synchronises.
+ *
+ * Storage format (fp16 metadata; 84 bytes per token per KV head = 2.625 bits/element,
+ * the figure the paper's error-comparison table gives for FP16 (m, s) metadata):
+ * the cache is an array of "window records", one per 32 consecutive tokens of one
+ * (layer, sequence, KV head), OKQ_RECORD_BYTES each:
+ *     [   0,  256)  key minimum m_gc, fp16 x 128 (channel order permuted, see below)
+ *     [ 256,  512)  key step s_gc,    fp16 x 128 (same order)
+ *     [ 512,  576)  key norms,   fp16 x 32 tokens
+ *     [ 576,  640)  value norms, fp16 x 32 tokens
+ *     [ 640, 1664)  key codes,   2 bits x 32 tokens x 128 channels
+ *     [1664, 2688)  value codes, 2 bits x 32 tokens x 128 channels
+ * Inside a record the channel / token order is the one the decode kernel's tensor-core
+ * fragments want; okq_cache_export / okq_cache_import convert to and from the canonical
+ * arrays (token-major codes with channel c of a token in byte c/4 at bits 2*(c%4);
+ * metadata as [window][channel][m, s]).
+ */
+#ifndef OKQ_H
+#define OKQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define OKQ_HEAD_DIM 128
+#define OKQ_WINDOW 32
+#define OKQ_RECORD_BYTES 2688
+#define OKQ_MAX_GROUP 8
+
+typedef enum {
+  OKQ_OK = 0,
+  OKQ_ERR_INVALID_ARG = 1, /* null pointer, negative size, layer range out of bounds, ... */
+  OKQ_ERR_UNSUPPORTED = 2, /* head_dim != 128, window != 32, GQA group > 8 or not integral */
+  OKQ_ERR_ALIGNMENT = 3,   /* a device pointer is not 16-byte aligned */
+  OKQ_ERR_CAPACITY = 4,    /* a sequence would exceed `capacity` (also the device status value) */
+  OKQ_ERR_WORKSPACE = 5,   /* decode workspace smaller than okq_decode_workspace_bytes() */
+  OKQ_ERR_CUDA = 6,        /* a CUDA runtime call failed; see okq_last_cuda_error() */
+  OKQ_ERR_TIMEOUT = 7      /* reserved: a bounded device-side wait gave up */
+} okq_status;
+
+/* Static, NUL-terminated description of a status value. */
+const char* okq_status_string(okq_status s);
+/* cudaError_t value behind the calling thread's most recent OKQ_ERR_CUDA (0 if none). */
+int okq_last_cuda_error(void);
+
+/* A 2-bit KV cache.  Plain data filled in by the caller. */
+typedef struct okq_cache {
+  int32_t n_layers, batch, n_kv_heads, n_q_heads;
+  int32_t head_dim;  /* 128 */
+  int32_t window;    /* 32 */
+  int32_t capacity;  /* max tokens per sequence, multiple of 32 */
+  int32_t reserved;  /* 0 */
+  void* records;     /* [n_layers][batch][n_kv_heads][capacity/32][OKQ_RECORD_BYTES] */
+  uint8_t* modality; /* [batch][capacity], shared by all layers and heads */
+  void* k_tail;      /* [n_layers][batch][n_kv_heads][32][128] fp16: raw keys not yet in a full window */
+  void* v_tail;      /* same for values */
+  int32_t* seq_len;  /* [n_layers][batch] tokens held; the first (seq_len & ~31) are packed */
+  int32_t* status;   /* [1] sticky first device-side error, 0 = none */
+} okq_cache;
+
+/* Byte sizes of the six device buffers of a cache with the given shape fields (pointers
+ * are ignored), in the order records, modality, k_tail, v_tail, seq_len, status.
+ * Returns OKQ_OK or the shape error. */
+okq_status okq_cache_sizes(const okq_cache* shape, size_t out_bytes[6]);
+
+/* Bytes of scratch okq_decode_attention needs for `layer_count` layers with `num_splits`
+ * (0 = let the library choose, the same choice the call makes).  0 on a shape error. */
+size_t okq_decode_workspace_bytes(const okq_cache* cache, int32_t layer_count, int32_t num_splits);
+
+/*
+ * Key quantiser (paper Eq. 2 followed by Eq. 4): for every (sequence, KV head) of `layer`
+ * quantise tokens [0, n_tokens) of k_fp16.  Per token: fp16 norm, z = H k/norm with
+ * H = Had_128 diag(signs)/sqrt(128); per 32-token window and channel: m = min z,
+ * s = (max - m)/3 as fp16, code = clamp(rint((z - m)/s), 0, 3).  The trailing
+ * n_tokens % 32 tokens are copied raw to k_tail.  Sets seq_len[layer][*] = n_tokens.
+ *   k_fp16   device, fp16, element (b, h, i, c) at k_fp16[b*strides[0] + h*strides[1] + i*strides[2] + c]
+ *   strides  host, in elements; each a multiple of 8 so rows stay 16-byte aligned
+ *   signs    device, float[128], each +1 or -1
+ * Errors: OKQ_ERR_INVALID_ARG (n_tokens < 0, layer out of range, null), OKQ_ERR_CAPACITY
+ * (n_tokens > capacity), OKQ_ERR_ALIGNMENT, OKQ_ERR_CUDA.
+ */
+okq_status okq_quantize_keys(const okq_cache* cache, int32_t layer, const void* k_fp16,
+                             const int64_t strides[3], int32_t n_tokens, const float* signs,
+                             void* stream);
+
+/*
+ * Value quantiser (paper Eq. 6 then Eq. 3): per token fp16 norm, z = R_m v/norm with the
+ * matrix of the token's modality m, code = index of the nearest of the four fixed
+ * Gaussian codebook levels.  Also stores `modality` into the cache and copies the
+ * trailing n_tokens % 32 tokens raw to v_tail.  Sets seq_len[layer][*] = n_tokens.
+ *   modality device, uint8 [batch][n_tokens]
+ *   R        device, float [n_R][3][128][128] row-major, z = R[.][m] u; n_R is 1 (shared
+ *            by the KV heads) or n_kv_heads
+ * The rotation is evaluated as one fused-multiply-add chain per output coordinate over
+ * the input index in ascending order, which makes the codes reproducible bit for bit.
+ */
+okq_status okq_quantize_values(const okq_cache* cache, int32_t layer, const void* v_fp16,
+                               const int64_t strides[3], int32_t n_tokens, const uint8_t* modality,
+                               const float* R, int32_t n_R, void* stream);
+
+/*
+ * Streaming append (the paper's protocol keeps recent tokens in fp16 before they are
+ * quantised): add one token per sequence to layers [layer, layer+layer_count).  The token
+ * goes raw into the tail; when the tail reaches 32 tokens they are quantised as one window
+ * exactly as the bulk calls would and the tail empties.  seq_len advances by one.
+ *   k_new, v_new   device fp16 [layer_count][batch][n_kv_heads][128]
+ *   modality_new   device uint8 [batch]
+ *   signs          device float [layer_count][128]
+ *   R              device float [layer_count][n_R][3][128][128]
+ * A sequence already at `capacity` is left unchanged and the device status word becomes
+ * OKQ_ERR_CAPACITY.
+ */
+okq_status okq_append(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* k_new,
+                      const void* v_new, const uint8_t* modality_new, const float* signs,
+                      const float* R, int32_t n_R, void* stream);
+
+/*
+ * Fused decode attention over the packed cache (paper Eq. 1 evaluated in the order the
+ * paper describes for its kernel: the query is rotated once per head, scores are taken
+ * against the codes in the rotated space, the softmax-weighted codebook levels are summed
+ * per modality and R_m^T is applied once per head after aggregation).  One query token per
+ * sequence, all cached tokens visible (packed windows and the raw tail), no mask.
+ *   q          device fp16 [layer_count][batch][n_q_heads][128]
+ *   sm_scale   softmax scale, normally 1/sqrt(128)
+ *   signs, R   as for okq_append
+ *   workspace  device scratch of at least okq_decode_workspace_bytes(cache, layer_count, num_splits)
+ *   num_splits split-K factor over the sequence (0 = automatic)
+ *   out        device float [layer_count][batch][n_q_heads][128]
+ * A sequence with seq_len 0 yields zeros.
+ */
+okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t layer_count,
+                                const void* q, float sm_scale, const float* signs, const float* R,
+                                int32_t n_R, void* workspace, size_t workspace_bytes,
+                                int32_t num_splits, float* out, void* stream);
+
+/*
+ * Canonical view of one layer (checkpointing and parity checks; the paper has no
+ * counterpart, the arrays are simply Eq. 2-4 and Eq. 6 outputs in natural order).
+ * All windows up to capacity are converted, whatever seq_len says.
+ *   k_codes, v_codes  device uint8 [batch][n_kv_heads][capacity][32]
+ *   k_norm, v_norm    device fp16  [batch][n_kv_heads][capacity]
+ *   k_meta            device fp16  [batch][n_kv_heads][capacity/32][128][2]  (m, s)
+ */
+okq_status okq_cache_export(const okq_cache* cache, int32_t layer, uint8_t* k_codes, void* k_norm,
+                            void* k_meta, uint8_t* v_codes, void* v_norm, void* stream);
+okq_status okq_cache_import(const okq_cache* cache, int32_t layer, const uint8_t* k_codes,
+                            const void* k_norm, const void* k_meta, const uint8_t* v_codes,
+                            const void* v_norm, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OKQ_H */

@@ -1,0 +1,189 @@
+"""Thin ctypes binding of the okq C ABI (argument marshalling only).
+
+PyTorch is used for device memory and streams; every step of the path runs in the CUDA
+library.  If the library is missing this module raises: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libokq.so")
+
+HEAD_DIM, WINDOW, RECORD_BYTES, MAX_GROUP = 128, 32, 2688, 8
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(8)
+
+
+class okq_cache(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("batch", C.c_int32), ("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("window", C.c_int32), ("capacity", C.c_int32), ("reserved", C.c_int32),
+                ("records", C.c_void_p), ("modality", C.c_void_p), ("k_tail", C.c_void_p), ("v_tail", C.c_void_p),
+                ("seq_len", C.c_void_p), ("status", C.c_void_p)]
+
+
+class OkqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().okq_status_string(status).decode()
+        if status == ERR_CUDA:
+            msg += f" (cudaError {lib().okq_last_cuda_error()})"
+        super().__init__(f"{where}: {msg}")
+
+
+_lib = None
+
+
+def lib():
+    """Load libokq.so (built in-tree by `python -m paper_2609_11582_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_11582_b200.build` "
+                               "(the okq path has no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.okq_status_string.restype = C.c_char_p
+        L.okq_status_string.argtypes = [C.c_int]
+        L.okq_last_cuda_error.restype = C.c_int
+        L.okq_cache_sizes.restype = C.c_int
+        L.okq_cache_sizes.argtypes = [C.POINTER(okq_cache), C.POINTER(C.c_size_t)]
+        L.okq_decode_workspace_bytes.restype = C.c_size_t
+        L.okq_decode_workspace_bytes.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32]
+        L.okq_quantize_keys.restype = C.c_int
+        L.okq_quantize_keys.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_void_p, C.POINTER(C.c_int64), C.c_int32,
+                                        C.c_void_p, C.c_void_p]
+        L.okq_quantize_values.restype = C.c_int
+        L.okq_quantize_values.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_void_p, C.POINTER(C.c_int64), C.c_int32,
+                                          C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.okq_append.restype = C.c_int
+        L.okq_append.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                 C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.okq_decode_attention.restype = C.c_int
+        L.okq_decode_attention.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32, C.c_void_p, C.c_float,
+                                           C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_int32,
+                                           C.c_void_p, C.c_void_p]
+        L.okq_cache_export.restype = C.c_int
+        L.okq_cache_export.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 6
+        L.okq_cache_import.restype = C.c_int
+        L.okq_cache_import.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 6
+        _lib = L
+    return _lib
+
+
+def exported_symbols():
+    return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
+            "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
+            "okq_cache_import"]
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _check(st: int, where: str):
+    if st != OK:
+        raise OkqError(st, where)
+
+
+def cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, head_dim=HEAD_DIM, window=WINDOW):
+    shape = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, head_dim, window, capacity, 0)
+    out = (C.c_size_t * 6)()
+    _check(lib().okq_cache_sizes(C.byref(shape), out), "okq_cache_sizes")
+    return list(out)
+
+
+class Cache:
+    """Device buffers of a 2-bit KV cache plus the C struct that describes them."""
+
+    def __init__(self, n_layers, batch, n_kv_heads, n_q_heads, capacity, device="cuda"):
+        sizes = cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity)
+        self.n_layers, self.batch, self.n_kv_heads, self.n_q_heads, self.capacity = (
+            n_layers, batch, n_kv_heads, n_q_heads, capacity)
+        self.device = torch.device(device)
+        self.records = torch.zeros(sizes[0], dtype=torch.uint8, device=device)
+        self.modality = torch.zeros(sizes[1], dtype=torch.uint8, device=device)
+        self.k_tail = torch.zeros(sizes[2] // 2, dtype=torch.float16, device=device)
+        self.v_tail = torch.zeros(sizes[3] // 2, dtype=torch.float16, device=device)
+        self.seq_len = torch.zeros(n_layers * batch, dtype=torch.int32, device=device)
+        self.status = torch.zeros(4, dtype=torch.int32, device=device)
+        self.c = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, HEAD_DIM, WINDOW, capacity, 0,
+                           self.records.data_ptr(), self.modality.data_ptr(), self.k_tail.data_ptr(),
+                           self.v_tail.data_ptr(), self.seq_len.data_ptr(), self.status.data_ptr())
+
+    @property
+    def group(self):
+        return self.n_q_heads // self.n_kv_heads
+
+    def packed_bytes(self, n_tokens):
+        """Bytes of packed records a decode step over n_tokens per sequence must read."""
+        return self.n_layers * self.batch * self.n_kv_heads * (n_tokens // WINDOW) * RECORD_BYTES
+
+    def device_status(self) -> int:
+        return int(self.status[0].item())
+
+
+def quantize_keys(cache: Cache, layer: int, k: torch.Tensor, signs: torch.Tensor, n_tokens=None, stream=None):
+    """k: fp16 [batch, n_kv_heads, n, 128] (last dim contiguous); signs: float32 [128]."""
+    assert k.dtype == torch.float16 and k.stride(3) == 1
+    n = k.shape[2] if n_tokens is None else n_tokens
+    strides = (C.c_int64 * 3)(k.stride(0), k.stride(1), k.stride(2))
+    _check(lib().okq_quantize_keys(C.byref(cache.c), layer, _ptr(k), strides, n, _ptr(signs), _stream(stream)),
+           "okq_quantize_keys")
+
+
+def quantize_values(cache: Cache, layer: int, v: torch.Tensor, modality: torch.Tensor, R: torch.Tensor,
+                    n_tokens=None, stream=None):
+    """v: fp16 [batch, n_kv_heads, n, 128]; modality: uint8 [batch, n]; R: float32 [n_R, 3, 128, 128]."""
+    assert v.dtype == torch.float16 and v.stride(3) == 1 and modality.dtype == torch.uint8 and modality.is_contiguous()
+    n = v.shape[2] if n_tokens is None else n_tokens
+    assert modality.shape[-1] == n
+    strides = (C.c_int64 * 3)(v.stride(0), v.stride(1), v.stride(2))
+    n_R = R.shape[0] if R.dim() == 4 else 1
+    _check(lib().okq_quantize_values(C.byref(cache.c), layer, _ptr(v), strides, n, _ptr(modality), _ptr(R), n_R,
+                                     _stream(stream)), "okq_quantize_values")
+
+
+def append(cache: Cache, layer: int, layer_count: int, k_new, v_new, modality_new, signs, R, n_R=1, stream=None):
+    _check(lib().okq_append(C.byref(cache.c), layer, layer_count, _ptr(k_new), _ptr(v_new), _ptr(modality_new),
+                            _ptr(signs), _ptr(R), n_R, _stream(stream)), "okq_append")
+
+
+def decode_workspace_bytes(cache: Cache, layer_count: int, num_splits: int = 0) -> int:
+    return lib().okq_decode_workspace_bytes(C.byref(cache.c), layer_count, num_splits)
+
+
+def decode_attention(cache: Cache, layer: int, layer_count: int, q, signs, R, workspace, out, n_R=1,
+                     sm_scale=None, num_splits=0, stream=None):
+    """q: fp16 [layer_count, batch, n_q_heads, 128]; out: float32 same shape; workspace: uint8 device tensor."""
+    scale = HEAD_DIM ** -0.5 if sm_scale is None else sm_scale
+    _check(lib().okq_decode_attention(C.byref(cache.c), layer, layer_count, _ptr(q), scale, _ptr(signs), _ptr(R), n_R,
+                                      _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                      num_splits, _ptr(out), _stream(stream)), "okq_decode_attention")
+
+
+def cache_export(cache: Cache, layer: int, stream=None):
+    """Canonical arrays of one layer as a dict of device tensors."""
+    B, H, cap, dev = cache.batch, cache.n_kv_heads, cache.capacity, cache.device
+    out = {"k_codes": torch.empty(B, H, cap, 32, dtype=torch.uint8, device=dev),
+           "k_norm": torch.empty(B, H, cap, dtype=torch.float16, device=dev),
+           "k_meta": torch.empty(B, H, cap // WINDOW, HEAD_DIM, 2, dtype=torch.float16, device=dev),
+           "v_codes": torch.empty(B, H, cap, 32, dtype=torch.uint8, device=dev),
+           "v_norm": torch.empty(B, H, cap, dtype=torch.float16, device=dev)}
+    _check(lib().okq_cache_export(C.byref(cache.c), layer, _ptr(out["k_codes"]), _ptr(out["k_norm"]),
+                                  _ptr(out["k_meta"]), _ptr(out["v_codes"]), _ptr(out["v_norm"]), _stream(stream)),
+           "okq_cache_export")
+    return out
+
+
+def cache_import(cache: Cache, layer: int, arrays: dict, stream=None):
+    a = {k: v.contiguous() for k, v in arrays.items()}
+    _check(lib().okq_cache_import(C.byref(cache.c), layer, _ptr(a["k_codes"]), _ptr(a["k_norm"]), _ptr(a["k_meta"]),
+                                  _ptr(a["v_codes"]), _ptr(a["v_norm"]), _stream(stream)), "okq_cache_import")

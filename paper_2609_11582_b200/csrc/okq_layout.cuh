@@ -1,0 +1,86 @@
+// Physical layout of a window record and small helpers shared by the CUDA kernels.
+//
+// A record holds the 32 tokens of one window of one (layer, sequence, KV head).  The
+// order of codes inside it follows the register fragments of mma.sync.m16n8k16, so that
+// the decode kernel feeds the tensor cores with 16-byte shared-memory reads and a few
+// mask/shift operations per 16 codes:
+//
+//  * Key codes are the B operand of  S^T[head][token] = W[head][channel] * C[channel][token].
+//    Lane l = 4*g + t of a warp owns, for the tokens g, g+8, g+16, g+24 of the window, the
+//    32 channels {16*kappa + 8*pair + 2*t + e}.  Those are two 32-bit words per token; in
+//    a word, register r = 2*kappa + pair (r & 7 inside the word) sits at bit offset
+//    8*((r>>2)&1) + 2*(r&3), its two channels e = 0/1 in the low/high 16 bits.
+//  * Value codes are the A operand of  O^T[channel][head] = C[channel][token] * P[token][head].
+//    Lane l = 4*g + t owns the channels {16*mu + 8*sh + g} (mu = 0..7, sh = 0/1) and the
+//    tokens {16*kv + 8*pv + 2*t + e}: one word per mu, field index j = 2*kv + pv at bit
+//    offset 8*sh + 2*j, token parity e in the low/high half.
+//  * (m, s) are stored as two planes of 128 fp16 in the order pi(c) that makes each
+//    lane's 32 channels contiguous.
+#pragma once
+#include <cstdint>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+namespace okq {
+
+constexpr int D = 128;
+constexpr int W = 32;
+constexpr int RECORD_BYTES = 2688;
+constexpr int OFF_KM = 0;
+constexpr int OFF_KS = 256;
+constexpr int OFF_KNORM = 512;
+constexpr int OFF_VNORM = 576;
+constexpr int OFF_KCODE = 640;
+constexpr int OFF_VCODE = 1664;
+
+// position of channel c inside the m / s planes
+__host__ __device__ inline int meta_pos(int c) {
+  int kappa = c >> 4, slot = c & 15;
+  int pair = slot >> 3, t = (slot & 7) >> 1, e = slot & 1;
+  return t * 32 + kappa * 4 + pair * 2 + e;
+}
+
+// key code of (token i in window, channel c): 32-bit word index in the key-code block and bit offset
+__host__ __device__ inline void kcode_pos(int i, int c, int& word, int& bit) {
+  int nu = i >> 3, g = i & 7;
+  int kappa = c >> 4, slot = c & 15;
+  int pair = slot >> 3, t = (slot & 7) >> 1, e = slot & 1;
+  int r = 2 * kappa + pair;
+  int ww = r >> 3, sh = (r >> 2) & 1, j = r & 3;
+  word = (nu >> 1) * 128 + (4 * g + t) * 4 + (nu & 1) * 2 + ww;
+  bit = 16 * e + 8 * sh + 2 * j;
+}
+
+// value code of (token i in window, channel c)
+__host__ __device__ inline void vcode_pos(int i, int c, int& word, int& bit) {
+  int mu = c >> 4, sh = (c >> 3) & 1, g = c & 7;
+  int kv = i >> 4, pv = (i >> 3) & 1, t = (i & 7) >> 1, e = i & 1;
+  int j = 2 * kv + pv;
+  word = (mu >> 2) * 128 + (4 * g + t) * 4 + (mu & 3);
+  bit = 16 * e + 8 * sh + 2 * j;
+}
+
+struct CacheView {
+  int n_layers, batch, n_kv_heads, n_q_heads, capacity;
+  unsigned char* records;
+  unsigned char* modality;
+  __half* k_tail;
+  __half* v_tail;
+  int* seq_len;
+  int* status;
+  __host__ __device__ inline size_t n_windows() const { return (size_t)capacity / W; }
+  __host__ __device__ inline unsigned char* record(int layer, int b, int h, size_t win) const {
+    return records + ((((size_t)layer * batch + b) * n_kv_heads + h) * n_windows() + win) * RECORD_BYTES;
+  }
+  __host__ __device__ inline size_t tail_off(int layer, int b, int h) const {
+    return (((size_t)layer * batch + b) * n_kv_heads + h) * (size_t)(W * D);
+  }
+};
+
+// value codebook: Lloyd-Max levels of N(0, 1/128) and the decision threshold, fp32
+constexpr float CB_INNER = 0x1.47d908p-5f;
+constexpr float CB_OUTER = 0x1.116a3p-3f;
+constexpr float CB_THRESH = 0x1.636072p-4f;
+constexpr float RSQRT_D = 0x1.6a09e6p-4f;  // float(1/sqrt(128))
+
+}  // namespace okq

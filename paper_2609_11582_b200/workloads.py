@@ -151,7 +151,7 @@ def gen_kv(w: Workload, layer: int, device="cpu", n_tokens: int | None = None,
         H = w.n_kv_heads
         mu0 = torch.randn(H, 1, HEAD_DIM, generator=g, device=device)
         steps = torch.randn(H, n, HEAD_DIM, generator=g, device=device) * 0.05
-        steps[:, 0, :] = 0
+        steps[:, :1, :] = 0
         mu = mu0 + torch.cumsum(steps, dim=1)
         del steps
         k = mu + torch.randn(H, n, HEAD_DIM, generator=g, device=device)

@@ -1,0 +1,80 @@
+"""CPU-only checks of the C ABI: the library loads, exports every declared symbol, and the
+host-side validation returns the documented status codes without touching a device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2609_11582_b200 import binding as B
+from paper_2609_11582_b200 import build as build_mod
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    build_mod.build()
+    return B.lib()
+
+
+def test_every_declared_symbol_is_exported(L):
+    hdr = open(os.path.join(ROOT, "include", "okq.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(okq_[a-z_]+)\s*\(", hdr))
+    assert declared == set(B.exported_symbols())
+    for s in declared:
+        assert hasattr(L, s), s
+
+
+def test_status_strings(L):
+    assert L.okq_status_string(0) == b"ok"
+    seen = {L.okq_status_string(i) for i in range(8)}
+    assert len(seen) == 8
+    assert L.okq_last_cuda_error() == 0
+
+
+def test_cache_sizes_and_record_format(L):
+    s = B.cache_sizes(28, 8, 4, 28, 16384)
+    units = 28 * 8 * 4
+    assert s[0] == units * (16384 // 32) * 2688
+    # 2688 B per 32-token window = 84 B per token per KV head = 2.625 bits per element
+    assert B.RECORD_BYTES / 32 == 84 and B.RECORD_BYTES * 8 / (32 * 2 * 128) == 2.625
+    assert s[1] == 8 * 16384 and s[2] == s[3] == units * 32 * 128 * 2 and s[4] == 28 * 8 * 4
+
+
+def test_shape_validation(L):
+    def sizes(**kw):
+        d = dict(n_layers=1, batch=1, n_kv_heads=1, n_q_heads=7, head_dim=128, window=32, capacity=64)
+        d.update(kw)
+        c = B.okq_cache(d["n_layers"], d["batch"], d["n_kv_heads"], d["n_q_heads"], d["head_dim"], d["window"],
+                        d["capacity"], 0)
+        out = (C.c_size_t * 6)()
+        return L.okq_cache_sizes(C.byref(c), out)
+    assert sizes() == B.OK
+    assert sizes(head_dim=64) == B.ERR_UNSUPPORTED
+    assert sizes(window=16) == B.ERR_UNSUPPORTED
+    assert sizes(n_q_heads=9) == B.ERR_UNSUPPORTED          # group 9 > 8
+    assert sizes(n_kv_heads=2, n_q_heads=7) == B.ERR_UNSUPPORTED
+    assert sizes(capacity=70) == B.ERR_INVALID_ARG
+    assert sizes(batch=0) == B.ERR_INVALID_ARG
+
+
+def test_pointer_validation_before_any_launch(L):
+    c = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, 0, 0, 0, 0, 0, 0)
+    strides = (C.c_int64 * 3)(64 * 128, 64 * 128, 128)
+    assert L.okq_quantize_keys(C.byref(c), 0, 4096, strides, 64, 4096, None) == B.ERR_INVALID_ARG   # null buffers
+    fake = 1 << 20
+    c = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, fake, fake, fake, fake, fake, fake)
+    assert L.okq_quantize_keys(C.byref(c), 1, fake, strides, 64, fake, None) == B.ERR_INVALID_ARG   # layer out of range
+    assert L.okq_quantize_keys(C.byref(c), 0, fake, strides, 96, fake, None) == B.ERR_CAPACITY
+    assert L.okq_quantize_keys(C.byref(c), 0, fake + 2, strides, 64, fake, None) == B.ERR_ALIGNMENT
+    bad = (C.c_int64 * 3)(64 * 128, 64 * 128, 100)
+    assert L.okq_quantize_keys(C.byref(c), 0, fake, bad, 64, fake, None) == B.ERR_ALIGNMENT
+    assert L.okq_quantize_values(C.byref(c), 0, fake, strides, 64, fake, fake, 2, None) == B.ERR_INVALID_ARG  # n_R
+    assert L.okq_append(C.byref(c), 0, 2, fake, fake, fake, fake, fake, 1, None) == B.ERR_INVALID_ARG
+    assert L.okq_decode_attention(C.byref(c), 0, 1, fake, 0.1, fake, fake, 1, fake, 16, 0, fake, None) == B.ERR_WORKSPACE
+    assert L.okq_decode_workspace_bytes(C.byref(c), 1, 3) > 0
+    assert L.okq_decode_workspace_bytes(C.byref(c), 0, 3) == 0
+    c8 = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, fake + 8, fake, fake, fake, fake, fake)
+    assert L.okq_append(C.byref(c8), 0, 1, fake, fake, fake, fake, fake, 1, None) == B.ERR_ALIGNMENT
