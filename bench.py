@@ -1,0 +1,302 @@
+#!/usr/bin/env python
+"""Benchmark of the okq hot path: one decode step = okq_append of one new text token per
+sequence to every layer + okq_decode_attention over every layer's packed cache.
+
+Default workload: the 7B-shaped full decode step (28 layers, 28/4 heads, batch 8, 16384
+tokens of context per sequence), synthetic seeded inputs.  Prints ONE JSON line.
+
+  value        packed-KV bytes of the step / device time of the step (GB/s), whole job
+  e2e          the same with this step's queries / new tokens copied from pinned host memory
+               and the attention output copied back, inside the timed region
+  roofline     the split-K decode kernel alone (CUDA events recorded around it on its stream)
+  cpu_baseline the CPU oracle timed on a bounded sample of the same workload
+
+`--impl reference` times the CPU oracle (the only reference this method has) instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_11582_b200 import workloads as WL  # noqa: E402
+
+METRIC = "2-bit KV decode-attention effective HBM GB/s (packed-KV bytes per decode step / step time)"
+BYTES_PER_TOKEN_HEAD = 84          # 32 B key codes + 2 B key norm + 16 B (m, s) + 32 B value codes + 2 B value norm
+# dram__bytes_read.sum + dram__bytes_write.sum of one split-K decode launch, measured with ncu
+# on a smaller case and scaled per token-head (see profiles/); None until measured.
+NCU_DRAM_BYTES_PER_TOKEN_HEAD = None
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Reads SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def oracle_prepare(w, n_layers_s, n_seq_s):
+    """Inputs of the CPU oracle for n_layers_s x n_seq_s sequences of the workload (the oracle
+    quantises the sampled fp16 inputs itself).  Returns (attention args, unit_rot, token-heads)."""
+    from oracle import okq_oracle as O
+    mod = WL.modality_layout(w).numpy()
+    kqs, vqs, qs, signs, Rs, kt, vt = [], [], [], [], [], [], []
+    U_per = n_seq_s * w.n_kv_heads
+    for l in range(n_layers_s):
+        k, v = WL.gen_kv(w, l, device="cpu", seqs=slice(0, n_seq_s))
+        kb = k.view(torch.int16).numpy().view(np.uint16).reshape(U_per, w.n_tokens, 128)
+        vb = v.view(torch.int16).numpy().view(np.uint16).reshape(U_per, w.n_tokens, 128)
+        sg = WL.gen_signs(w, l).numpy(); R = WL.gen_rotations(w, l).numpy()
+        kq, vq, _ = O.quantize_batch(kb, vb, mod, sg, R)
+        kqs.append(kq); vqs.append(vq); signs.append(sg); Rs.append(R)
+        q = WL.gen_queries(w, l)[:n_seq_s].view(torch.int16).numpy().view(np.uint16)
+        qs.append(q.reshape(n_seq_s, w.n_kv_heads, w.group, 128).reshape(U_per, w.group, 128))
+        npk = (w.n_tokens // 32) * 32
+        kt.append(kb[:, npk:]); vt.append(vb[:, npk:])
+    cat = lambda ds, key: np.concatenate([d[key] for d in ds])
+    kq = {k: cat(kqs, k) for k in ("codes", "norm", "meta")}
+    vq = {k: cat(vqs, k) for k in ("codes", "norm")}
+    unit_rot = np.repeat(np.arange(n_layers_s), U_per)
+    args = (np.concatenate(qs), kq, vq, mod, np.concatenate(kt), np.concatenate(vt), np.stack(signs), np.stack(Rs))
+    return args, unit_rot, n_layers_s * U_per * w.n_tokens
+
+
+def oracle_pass(args, unit_rot):
+    """One timed pass of the oracle's rotated-space attention; returns (seconds, threads)."""
+    from oracle import okq_oracle as O
+    t0 = time.perf_counter()
+    _, th = O.attention(1, *args, unit_rot=unit_rot)
+    return time.perf_counter() - t0, th
+
+
+def run_reference(args, w):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    # a bounded sample per "step": one oracle attention pass over 1 layer x 4 sequences
+    n_seq_s = min(4, w.batch)
+    oargs, unit_rot, th_units = oracle_prepare(w, 1, n_seq_s)
+    per_step, threads = [], 1
+    for _ in range(args.warmup + args.steps):
+        t, threads = oracle_pass(oargs, unit_rot)
+        per_step.append(t)
+    ts = per_step[args.warmup:]
+    t = sum(ts) / len(ts)
+    gbs = th_units * BYTES_PER_TOKEN_HEAD / t / 1e9
+    sample = (f"1 layer x {n_seq_s} sequences x {w.n_kv_heads} KV heads x {w.n_tokens} tokens per step "
+              "(oracle rotated-space attention; GB/s = packed bytes of the sample / time)")
+    line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "n_layers": w.n_layers, "batch": w.batch, "n_q_heads": w.n_q_heads,
+                       "n_kv_heads": w.n_kv_heads, "context": w.n_tokens, "sample": sample},
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=32)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="okq", choices=["okq", "reference"])
+    ap.add_argument("--workload", default="step7b", choices=sorted(WL.WORKLOADS))
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = WL.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    from paper_2609_11582_b200 import binding as B
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- build the packed cache on the device (setup, untimed)
+    L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
+    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev)
+    mod = WL.modality_layout(w).unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
+    signs = torch.stack([WL.gen_signs(w, l) for l in range(L)]).to(dev)
+    R = torch.stack([WL.gen_rotations(w, l) for l in range(L)]).unsqueeze(1).contiguous().to(dev)
+    for l in range(L):
+        k, v = WL.gen_kv(w, l, device=dev)
+        B.quantize_keys(cache, l, k, signs[l])
+        B.quantize_values(cache, l, v, mod, R[l])
+        del k, v
+    torch.cuda.synchronize()
+    seq0 = cache.seq_len.clone()
+
+    total = args.warmup + args.steps
+    q_host = torch.stack([WL.gen_queries(w, l) for l in range(L)]).pin_memory()          # [L,B,Hq,128] fp16
+    newtok = [WL.gen_new_token(w, 0, s) for s in range(total)]
+    kn_host = torch.stack([t[0].unsqueeze(0).expand(L, -1, -1, -1) for t in newtok]).contiguous().pin_memory()
+    vn_host = torch.stack([t[1].unsqueeze(0).expand(L, -1, -1, -1) for t in newtok]).contiguous().pin_memory()
+    mn_host = torch.zeros(Bn, dtype=torch.uint8).pin_memory()
+    out_host = torch.empty(L, Bn, Hq, 128, dtype=torch.float32).pin_memory()
+
+    q_dev = q_host.to(dev); kn_dev = kn_host.to(dev); vn_dev = vn_host.to(dev); mn_dev = mn_host.to(dev)
+    out = torch.empty(L, Bn, Hq, 128, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(16, B.decode_workspace_bytes(cache, L, args.splits)), dtype=torch.uint8, device=dev)
+    packed_bytes = L * Bn * H * N * BYTES_PER_TOKEN_HEAD
+
+    def step_resident(s):
+        B.append(cache, 0, L, kn_dev[s], vn_dev[s], mn_dev, signs, R)
+        B.decode_attention(cache, 0, L, q_dev, signs, R, ws, out, num_splits=args.splits)
+
+    def step_e2e(s):
+        qd = q_host.to(dev, non_blocking=True)
+        kd = kn_host[s].to(dev, non_blocking=True)
+        vd = vn_host[s].to(dev, non_blocking=True)
+        md = mn_host.to(dev, non_blocking=True)
+        B.append(cache, 0, L, kd, vd, md, signs, R)
+        B.decode_attention(cache, 0, L, qd, signs, R, ws, out, num_splits=args.splits)
+        out_host.copy_(out, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(step_fn, with_kernel_events):
+        cache.seq_len.copy_(seq0)
+        for s in range(args.warmup):
+            step_fn(s)
+        cache.seq_len.copy_(seq0)       # the timed steps start from the same context length
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in kev:      # torch creates the CUDA event on first record; the library re-records it later
+            a.record(); b.record()
+        barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        for i in range(args.steps):
+            if with_kernel_events:
+                B.profile_events(*kev[i])
+            ev[i][0].record()
+            step_fn(args.warmup + i)
+            ev[i][1].record()
+        barrier()
+        B.profile_events(None, None)
+        clocks = sampler.stop()
+        ms = sum(a.elapsed_time(b) for a, b in ev)
+        kms = sum(a.elapsed_time(b) for a, b in kev) / args.steps if with_kernel_events else None
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, kms, clocks
+
+    ms_total, kernel_ms, clocks = timed(step_resident, True)
+    if cache.device_status() != 0:
+        raise RuntimeError("device status word set during the benchmark")
+    ms_e2e, _, _ = timed(step_e2e, False)
+    ms_step = ms_total / args.steps
+    value = world * packed_bytes / (ms_step * 1e-3) / 1e9
+    e2e_value = world * packed_bytes / (ms_e2e / args.steps * 1e-3) / 1e9
+    peak, peak_kind = measured_peaks()
+    achieved = packed_bytes / (kernel_ms * 1e-3) / 1e9
+    traffic = None if NCU_DRAM_BYTES_PER_TOKEN_HEAD is None else NCU_DRAM_BYTES_PER_TOKEN_HEAD * L * Bn * H * N
+
+    if rank != 0:
+        return
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_l, n_s = min(2, L), min(8, Bn)
+        oargs, unit_rot, th_units = oracle_prepare(w, n_l, n_s)
+        passes = [oracle_pass(oargs, unit_rot) for _ in range(3)]
+        t, threads = min(p[0] for p in passes), passes[0][1]
+        cpu = {"value": th_units * BYTES_PER_TOKEN_HEAD / t / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+               "sample": f"{n_l} layers x {n_s} sequences x {H} KV heads x {N} tokens (oracle rotated-space attention, "
+                         f"best of 3 passes, {t:.2f} s per pass); GB/s = packed bytes of the sample / time",
+               "seconds_per_sample_pass": t}
+    line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "n_layers": L, "batch": Bn, "n_q_heads": Hq, "n_kv_heads": H, "context": N,
+                       "step": "okq_append(1 text token/seq, all layers) + okq_decode_attention(all layers), one call each",
+                       "packed_kv_bytes_per_step": packed_bytes, "l2": "inputs (1.2 GB of records per step) exceed L2",
+                       "parallelism": "replicas only" if world > 1 else "1 gpu"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": "GB/s", "ms_per_step": ms_e2e / args.steps,
+                    "h2d_bytes_per_step": q_host.numel() * 2 + kn_host[0].numel() * 2 + vn_host[0].numel() * 2 + Bn,
+                    "d2h_bytes_per_step": out_host.numel() * 4},
+            "gpu_launches": 4 * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "okq split-K decode kernel (one launch per step)",
+                         "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                         "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0,
+                         "kernel_ms": kernel_ms, "traffic": traffic},
+            "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

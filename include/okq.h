@@ -155,6 +155,15 @@ okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t l
                                 int32_t num_splits, float* out, void* stream);
 
 /*
+ * Profiling aid (the paper has no counterpart): until cleared with two nulls, every
+ * okq_decode_attention call made by the calling thread records `before` on its stream
+ * just ahead of the split-K kernel and `after` just behind it (ahead of the combine
+ * kernel), so a benchmark can time the dominant kernel alone.  Both are cudaEvent_t
+ * handles passed as void*, owned by the caller.
+ */
+void okq_profile_events(void* before, void* after);
+
+/*
  * Canonical view of one layer (checkpointing and parity checks; the paper has no
  * counterpart, the arrays are simply Eq. 2-4 and Eq. 6 outputs in natural order).
  * All windows up to capacity are converted, whatever seq_len says.

@@ -65,6 +65,8 @@ def lib():
         L.okq_decode_attention.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32, C.c_void_p, C.c_float,
                                            C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_int32,
                                            C.c_void_p, C.c_void_p]
+        L.okq_profile_events.restype = None
+        L.okq_profile_events.argtypes = [C.c_void_p, C.c_void_p]
         L.okq_cache_export.restype = C.c_int
         L.okq_cache_export.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 6
         L.okq_cache_import.restype = C.c_int
@@ -76,7 +78,7 @@ def lib():
 def exported_symbols():
     return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
-            "okq_cache_import"]
+            "okq_cache_import", "okq_profile_events"]
 
 
 def _ptr(t) -> int:
@@ -167,6 +169,11 @@ def decode_attention(cache: Cache, layer: int, layer_count: int, q, signs, R, wo
     _check(lib().okq_decode_attention(C.byref(cache.c), layer, layer_count, _ptr(q), scale, _ptr(signs), _ptr(R), n_R,
                                       _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
                                       num_splits, _ptr(out), _stream(stream)), "okq_decode_attention")
+
+
+def profile_events(before=None, after=None):
+    """Record two torch.cuda.Event objects around the split-K kernel of later decode calls (None clears)."""
+    lib().okq_profile_events(None if before is None else before.cuda_event, None if after is None else after.cuda_event)
 
 
 def cache_export(cache: Cache, layer: int, stream=None):

@@ -368,6 +368,8 @@ __global__ void __launch_bounds__(128) k_combine(DecodeParams P) {
   }
 }
 
+static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+
 static int auto_splits(const okq_cache* c, int layer_count) {
   long long units = (long long)layer_count * c->batch * c->n_kv_heads;
   long long want = (2 * 148 + units - 1) / units;
@@ -383,6 +385,11 @@ static int auto_splits(const okq_cache* c, int layer_count) {
 using namespace okq;
 
 extern "C" {
+
+void okq_profile_events(void* before, void* after) {
+  g_ev_before = static_cast<cudaEvent_t>(before);
+  g_ev_after = static_cast<cudaEvent_t>(after);
+}
 
 size_t okq_decode_workspace_bytes(const okq_cache* cache, int32_t layer_count, int32_t num_splits) {
   if (check_cache(cache, false) != OKQ_OK || layer_count <= 0 || num_splits < 0) return 0;
@@ -416,7 +423,9 @@ okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t l
     attr_set = true;
   }
   dim3 grid(P.n_splits, cache->n_kv_heads, cache->batch * layer_count);
+  if (g_ev_before) cudaEventRecord(g_ev_before, s);
   k_decode_simt<<<grid, 128, sizeof(DecodeSmem), s>>>(P);
+  if (g_ev_after) cudaEventRecord(g_ev_after, s);
   k_combine<<<dim3(cache->n_kv_heads, cache->batch * layer_count), 128, 0, s>>>(P);
   return launch_status();
 }
