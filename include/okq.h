@@ -145,7 +145,9 @@ okq_status okq_append(const okq_cache* cache, int32_t layer, int32_t layer_count
  *   sm_scale   softmax scale, normally 1/sqrt(128)
  *   signs, R   as for okq_append
  *   workspace  device scratch of at least okq_decode_workspace_bytes(cache, layer_count, num_splits)
- *   num_splits split-K factor over the sequence (0 = automatic)
+ *   num_splits 0 = one persistent CTA per SM, each owning an equal slice of the flattened
+ *              (layer, sequence, head, window) axis; n > 0 = n CTAs per (sequence, KV head)
+ *              on average (at most 1024 in total)
  *   out        device float [layer_count][batch][n_q_heads][128]
  * A sequence with seq_len 0 yields zeros.
  */
@@ -153,6 +155,19 @@ okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t l
                                 const void* q, float sm_scale, const float* signs, const float* R,
                                 int32_t n_R, void* workspace, size_t workspace_bytes,
                                 int32_t num_splits, float* out, void* stream);
+
+/*
+ * The same computation on CUDA cores only (fp32 multiply-adds, dot products reduced with
+ * warp shuffles): the straightforward form of the paper's kernel, kept as an independent
+ * cross-check of the tensor-core path and as the measured arithmetic-bound baseline.
+ * Arguments, workspace size and errors as for okq_decode_attention; num_splits is the
+ * number of CTAs per (sequence, KV head).
+ */
+okq_status okq_decode_attention_simt(const okq_cache* cache, int32_t layer, int32_t layer_count,
+                                     const void* q, float sm_scale, const float* signs,
+                                     const float* R, int32_t n_R, void* workspace,
+                                     size_t workspace_bytes, int32_t num_splits, float* out,
+                                     void* stream);
 
 /*
  * Profiling aid (the paper has no counterpart): until cleared with two nulls, every

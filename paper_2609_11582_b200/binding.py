@@ -65,6 +65,8 @@ def lib():
         L.okq_decode_attention.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32, C.c_void_p, C.c_float,
                                            C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_int32,
                                            C.c_void_p, C.c_void_p]
+        L.okq_decode_attention_simt.restype = C.c_int
+        L.okq_decode_attention_simt.argtypes = L.okq_decode_attention.argtypes
         L.okq_profile_events.restype = None
         L.okq_profile_events.argtypes = [C.c_void_p, C.c_void_p]
         L.okq_cache_export.restype = C.c_int
@@ -78,7 +80,7 @@ def lib():
 def exported_symbols():
     return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
-            "okq_cache_import", "okq_profile_events"]
+            "okq_cache_import", "okq_profile_events", "okq_decode_attention_simt"]
 
 
 def _ptr(t) -> int:
@@ -163,10 +165,12 @@ def decode_workspace_bytes(cache: Cache, layer_count: int, num_splits: int = 0) 
 
 
 def decode_attention(cache: Cache, layer: int, layer_count: int, q, signs, R, workspace, out, n_R=1,
-                     sm_scale=None, num_splits=0, stream=None):
-    """q: fp16 [layer_count, batch, n_q_heads, 128]; out: float32 same shape; workspace: uint8 device tensor."""
+                     sm_scale=None, num_splits=0, stream=None, simt=False):
+    """q: fp16 [layer_count, batch, n_q_heads, 128]; out: float32 same shape; workspace: uint8 device tensor.
+    simt=True calls okq_decode_attention_simt (CUDA-core cross-check) instead."""
     scale = HEAD_DIM ** -0.5 if sm_scale is None else sm_scale
-    _check(lib().okq_decode_attention(C.byref(cache.c), layer, layer_count, _ptr(q), scale, _ptr(signs), _ptr(R), n_R,
+    fn = lib().okq_decode_attention_simt if simt else lib().okq_decode_attention
+    _check(fn(C.byref(cache.c), layer, layer_count, _ptr(q), scale, _ptr(signs), _ptr(R), n_R,
                                       _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
                                       num_splits, _ptr(out), _stream(stream)), "okq_decode_attention")
 

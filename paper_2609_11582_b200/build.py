@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libokq.so")
-SOURCES = ["okq_host.cu", "okq_quant.cu", "okq_decode.cu"]
+SOURCES = ["okq_host.cu", "okq_quant.cu", "okq_decode.cu", "okq_decode_mma.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]
 
@@ -28,7 +28,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     flags = list(FLAGS)
     if verbose:
         flags += ["-Xptxas", "-v"]
-    cmd = [nvcc, *flags, "-shared", "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lcudart"]
+    cmd = [nvcc, *flags, "-rdc=false", "-shared", "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lcudart"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or r.returncode != 0:
         sys.stderr.write(r.stdout + r.stderr)

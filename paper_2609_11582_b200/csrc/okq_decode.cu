@@ -7,29 +7,9 @@
 // head.  No fp16 K or V is ever rebuilt.
 #include "okq_common.cuh"
 #include "okq_device.cuh"
+#include "okq_decode_shared.cuh"
 
 namespace okq {
-
-constexpr int GP = OKQ_MAX_GROUP;  // padded GQA group
-constexpr int NACC = 4;            // 3 modality accumulators + 1 raw (tail) accumulator
-
-struct Partial {
-  float m[GP];
-  float l[GP];
-  float acc[NACC][GP][D];
-};
-
-struct DecodeParams {
-  CacheView cv;
-  int layer0, layer_count, n_splits, group;
-  const __half* q;     // [layer_count][batch][n_q_heads][128]
-  const float* signs;  // [layer_count][128]
-  const float* R;      // [layer_count][n_R][3][128][128]
-  int n_R;
-  float sm_scale;
-  Partial* partials;   // [layer_count*batch*n_kv_heads][n_splits]
-  float* out;          // [layer_count][batch][n_q_heads][128]
-};
 
 struct WarpSmem {
   __align__(16) unsigned char rec[RECORD_BYTES];
@@ -380,6 +360,60 @@ static int auto_splits(const okq_cache* c, int layer_count) {
   return (int)want;
 }
 
+static int sm_count() {
+  static thread_local int cached_dev = -1, cached = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev != cached_dev) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached = n;
+    cached_dev = dev;
+  }
+  return cached;
+}
+
+// persistent grid of the tensor-core kernel
+static int mma_ctas(const okq_cache* c, int layer_count, int num_splits) {
+  if (num_splits <= 0) return sm_count();
+  long long n = (long long)num_splits * layer_count * c->batch * c->n_kv_heads;
+  return (int)(n > 1024 ? 1024 : n);
+}
+
+static size_t simt_workspace(const okq_cache* c, int layer_count, int num_splits) {
+  int S = num_splits > 0 ? num_splits : auto_splits(c, layer_count);
+  return (size_t)layer_count * c->batch * c->n_kv_heads * S * sizeof(Partial);
+}
+
+static size_t mma_workspace(const okq_cache* c, int layer_count, int num_splits) {
+  return ((size_t)layer_count * c->batch * c->n_kv_heads + mma_ctas(c, layer_count, num_splits)) * sizeof(PartialF);
+}
+
+static okq_status check_decode(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* q,
+                               const float* signs, const float* R, int32_t n_R, void* workspace,
+                               size_t workspace_bytes, int32_t num_splits, float* out) {
+  okq_status st = check_cache(cache, true);
+  if (st != OKQ_OK) return st;
+  if (!q || !signs || !R || !workspace || !out || num_splits < 0) return OKQ_ERR_INVALID_ARG;
+  if (layer < 0 || layer_count <= 0 || layer + layer_count > cache->n_layers) return OKQ_ERR_INVALID_ARG;
+  if (n_R != 1 && n_R != cache->n_kv_heads) return OKQ_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(signs) || !aligned16(R) || !aligned16(workspace) || !aligned16(out))
+    return OKQ_ERR_ALIGNMENT;
+  if (workspace_bytes < okq_decode_workspace_bytes(cache, layer_count, num_splits)) return OKQ_ERR_WORKSPACE;
+  return OKQ_OK;
+}
+
+static DecodeParams make_params(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* q,
+                                float sm_scale, const float* signs, const float* R, int32_t n_R, float* out) {
+  DecodeParams P;
+  P.cv = make_view(cache);
+  P.layer0 = layer; P.layer_count = layer_count; P.n_splits = 1;
+  P.group = cache->n_q_heads / cache->n_kv_heads;
+  P.q = static_cast<const __half*>(q); P.signs = signs; P.R = R; P.n_R = n_R; P.sm_scale = sm_scale;
+  P.partials = nullptr; P.partials_f = nullptr; P.out = out;
+  return P;
+}
+
 }  // namespace okq
 
 using namespace okq;
@@ -393,28 +427,41 @@ void okq_profile_events(void* before, void* after) {
 
 size_t okq_decode_workspace_bytes(const okq_cache* cache, int32_t layer_count, int32_t num_splits) {
   if (check_cache(cache, false) != OKQ_OK || layer_count <= 0 || num_splits < 0) return 0;
-  int S = num_splits > 0 ? num_splits : auto_splits(cache, layer_count);
-  return (size_t)layer_count * cache->batch * cache->n_kv_heads * S * sizeof(Partial);
+  size_t a = simt_workspace(cache, layer_count, num_splits), b = mma_workspace(cache, layer_count, num_splits);
+  return a > b ? a : b;
 }
 
 okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* q,
                                 float sm_scale, const float* signs, const float* R, int32_t n_R, void* workspace,
                                 size_t workspace_bytes, int32_t num_splits, float* out, void* stream) {
-  okq_status st = check_cache(cache, true);
+  okq_status st = check_decode(cache, layer, layer_count, q, signs, R, n_R, workspace, workspace_bytes, num_splits, out);
   if (st != OKQ_OK) return st;
-  if (!q || !signs || !R || !workspace || !out || num_splits < 0) return OKQ_ERR_INVALID_ARG;
-  if (layer < 0 || layer_count <= 0 || layer + layer_count > cache->n_layers) return OKQ_ERR_INVALID_ARG;
-  if (n_R != 1 && n_R != cache->n_kv_heads) return OKQ_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(signs) || !aligned16(R) || !aligned16(workspace) || !aligned16(out))
-    return OKQ_ERR_ALIGNMENT;
-  if (workspace_bytes < okq_decode_workspace_bytes(cache, layer_count, num_splits)) return OKQ_ERR_WORKSPACE;
-  DecodeParams P;
-  P.cv = make_view(cache);
-  P.layer0 = layer; P.layer_count = layer_count;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // one launch covers at most MAX_ENTRIES (layer, sequence) pairs
+  const int layers_per_launch = cache->batch >= MAX_ENTRIES ? 1 : MAX_ENTRIES / cache->batch;
+  if (cache->batch > MAX_ENTRIES) return OKQ_ERR_UNSUPPORTED;
+  const size_t q_stride = (size_t)cache->batch * cache->n_q_heads * D;
+  for (int l0 = 0; l0 < layer_count; l0 += layers_per_launch) {
+    const int lc = layer_count - l0 < layers_per_launch ? layer_count - l0 : layers_per_launch;
+    DecodeParams P = make_params(cache, layer + l0, lc, static_cast<const __half*>(q) + l0 * q_stride, sm_scale,
+                                 signs + (size_t)l0 * D, R + (size_t)l0 * n_R * 3 * D * D, n_R, out + l0 * q_stride);
+    P.partials_f = static_cast<PartialF*>(workspace);
+    const int n_cta = mma_ctas(cache, lc, num_splits);
+    st = launch_decode_mma(P, n_cta, s, g_ev_before, g_ev_after);
+    if (st != OKQ_OK) return st;
+  }
+  return launch_status();
+}
+
+okq_status okq_decode_attention_simt(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* q,
+                                     float sm_scale, const float* signs, const float* R, int32_t n_R,
+                                     void* workspace, size_t workspace_bytes, int32_t num_splits, float* out,
+                                     void* stream) {
+  okq_status st = check_decode(cache, layer, layer_count, q, signs, R, n_R, workspace, workspace_bytes, num_splits, out);
+  if (st != OKQ_OK) return st;
+  DecodeParams P = make_params(cache, layer, layer_count, q, sm_scale, signs, R, n_R, out);
   P.n_splits = num_splits > 0 ? num_splits : auto_splits(cache, layer_count);
-  P.group = cache->n_q_heads / cache->n_kv_heads;
-  P.q = static_cast<const __half*>(q); P.signs = signs; P.R = R; P.n_R = n_R; P.sm_scale = sm_scale;
-  P.partials = static_cast<Partial*>(workspace); P.out = out;
+  P.partials = static_cast<Partial*>(workspace);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   static thread_local bool attr_set = false;
   if (!attr_set) {

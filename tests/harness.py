@@ -73,13 +73,13 @@ class Case:
         torch.cuda.synchronize()
         return e
 
-    def gpu_decode(self, layer, layer_count=1, num_splits=0):
+    def gpu_decode(self, layer, layer_count=1, num_splits=0, simt=False):
         c = self.cache
         ws = torch.empty(max(16, B.decode_workspace_bytes(c, layer_count, num_splits)), dtype=torch.uint8, device=c.device)
         out = torch.full((layer_count, c.batch, c.n_q_heads, D), float("nan"), dtype=torch.float32, device=c.device)
         B.decode_attention(c, layer, layer_count, self.d_q[layer:layer + layer_count].contiguous(),
                            self.d_signs[layer:layer + layer_count].contiguous(),
-                           self.d_R[layer:layer + layer_count].contiguous(), ws, out, num_splits=num_splits)
+                           self.d_R[layer:layer + layer_count].contiguous(), ws, out, num_splits=num_splits, simt=simt)
         torch.cuda.synchronize()
         return out.cpu().numpy().astype(np.float64)
 
