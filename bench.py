@@ -166,8 +166,11 @@ def main():
     ap.add_argument("--workload", default="step7b", choices=sorted(WL.WORKLOADS))
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling on a small case)")
     args = ap.parse_args()
     w = WL.WORKLOADS[args.workload]
+    if args.layers > 0:
+        w = WL.scaled(w, n_layers=args.layers, name=f"{w.name}[layers={args.layers}]")
     if args.impl == "reference":
         return run_reference(args, w)
 

@@ -147,8 +147,8 @@ __global__ void __launch_bounds__(128) k_decode_simt(DecodeParams P) {
         }
       }
     }
-    const float kn = __half2float(reinterpret_cast<const __half*>(ws.rec + OFF_KNORM)[lane]) * P.sm_scale;
-    const float vn = __half2float(reinterpret_cast<const __half*>(ws.rec + OFF_VNORM)[lane]);
+    const float kn = __half2float(reinterpret_cast<const __half*>(ws.rec + OFF_KNORM)[norm_pos(lane)]) * P.sm_scale;
+    const float vn = __half2float(reinterpret_cast<const __half*>(ws.rec + OFF_VNORM)[norm_pos(lane)]);
     float pw[GP];
 #pragma unroll
     for (int j = 0; j < GP; j++) {

@@ -13,12 +13,15 @@
 //   * the value codebook {-b,-a,a,b} is affine in the two code bits:
 //     cb[c] = (b-a)*c + (3a-b)*bit1(c) - b, so two bit-plane products plus the running sum
 //     of the weights reproduce it exactly.
-// Online softmax runs per warp in FlashAttention order; each warp streams its own windows
-// through a cp.async ring in shared memory.  Values accumulate in the rotated basis of the
-// current modality; the other modalities' accumulators wait in shared memory.  The grid is
-// persistent: CTA i owns an equal slice of the flattened (layer, sequence, head, window)
-// axis and writes one partial per (sequence, head) it touches; the combine kernel merges
-// them, adds the raw fp16 tail tokens, applies R_m^T once per head and normalises.
+// A CTA runs 8 warp pairs.  The "score" warp of a pair streams window records through a
+// cp.async ring, computes the scores and the online softmax (FlashAttention order) and hands
+// the fp16 numerators to its "value" warp through shared memory; the value warp accumulates
+// the codebook sums of the previous window meanwhile.  One named barrier per pair and
+// iteration keeps the two in step (no spin-waits anywhere).  Values accumulate in the rotated
+// basis of the current modality; the other modalities' accumulators wait in shared memory.
+// The grid is persistent: CTA i owns an equal slice of the flattened (layer, sequence, head,
+// window) axis and writes one partial per (sequence, head) it touches; the combine kernel
+// merges them, adds the raw fp16 tail tokens, applies R_m^T once per head and normalises.
 #include "okq_common.cuh"
 #include "okq_device.cuh"
 #include "okq_decode_shared.cuh"
@@ -27,18 +30,30 @@ namespace okq {
 
 namespace {
 
-constexpr int NWARP = 8;
-constexpr int NSTAGE = 3;
+constexpr int NPAIR = 8;                        // warp pairs per CTA
+constexpr int NTHREADS = NPAIR * 64;
+constexpr int NSTAGE = 4;                       // record ring per pair
+constexpr int PREFETCH = 2;                     // windows in flight ahead of the score warp
 constexpr int STAGE_BYTES = RECORD_BYTES + 32;  // record + the window's 32 modality bytes
 constexpr int SPILL_REGS = 33;                  // 32 accumulator registers + the running weight sum
 
+struct Handoff {
+  uint32_t pb[4][32];   // per lane: numerators p * vnorm * 2^6 / 4^nu of its 8 tokens, fp16 pairs
+  float m[GP];          // running maximum per head after this window (log2 domain)
+  float alpha[GP];      // factor the value accumulators must be multiplied by before this window
+  int rescale;          // non-zero if any alpha != 1
+  int pad[15];
+};
+
 struct MmaSmem {
-  __align__(16) unsigned char stage[NWARP][NSTAGE][STAGE_BYTES];
-  float spill[NWARP][3][SPILL_REGS][32];
-  float spill_m[NWARP][3][GP];
+  __align__(16) unsigned char stage[NPAIR][NSTAGE][STAGE_BYTES];
+  __align__(16) Handoff hand[NPAIR][2];
+  float spill[NPAIR][3][SPILL_REGS][32];
+  float spill_m[NPAIR][3][GP];
   float qs[GP][D];       // q' * 2^kh, natural channel order
+  uint2 qf[16][32];      // per lane and fragment register r: (hi, lo) fp16 pairs of q' / 4^(r&3)
   float fscale[GP];      // 2^(24-kh) * sm_scale * log2(e)
-  float wm[NWARP][GP], wl[NWARP][GP];
+  float wm[NPAIR][GP], wl[NPAIR][GP];
   int prefix[MAX_ENTRIES + 1];
 };
 
@@ -57,8 +72,19 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
 
+// hardware barrier shared by the two warps of a pair (ids 1..8; id 0 is __syncthreads)
+__device__ __forceinline__ void pair_barrier(int pair) {
+  asm volatile("bar.sync %0, 64;\n" ::"r"(pair + 1) : "memory");
+}
+
 __device__ __forceinline__ uint32_t h2u(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ __half2 u2h(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
 
 // fp16 pair (lo half = a, hi half = b), saturating instead of overflowing to infinity
 __device__ __forceinline__ uint32_t pack_sat(float a, float b) {
@@ -76,15 +102,248 @@ __device__ __forceinline__ void split_product(__half2 qh, __half2 ql, __half2 x,
   lo = h2u(__hfma2(ql, x, e));
 }
 
+struct Segment {
+  const unsigned char* rec0;   // first record of the (layer, sequence, head)
+  const unsigned char* mod0;   // modality row of the sequence
+  int w0, n_my;                // first window of this pair's list, number of windows (stride NPAIR)
+};
+
+// ---------------------------------------------------------------- score warp
+__device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int pair, int lane, float& run_m_out,
+                                           float& run_l_out) {
+  const int g = lane >> 2, t = lane & 3;
+  const float fsc = sm.fscale[g];
+  float run_m = -INFINITY, run_l = 0.f;
+
+  auto issue = [&](int k) {
+    if (k < sg.n_my) {
+      const int win = sg.w0 + k * NPAIR;
+      unsigned char* dst = sm.stage[pair][k % NSTAGE];
+      const unsigned char* src = sg.rec0 + (size_t)win * RECORD_BYTES;
+#pragma unroll
+      for (int i = 0; i < 6; i++) {
+        int c16 = lane + 32 * i;
+        if (c16 < RECORD_BYTES / 16) cp_async16(dst + 16 * c16, src + 16 * c16);
+      }
+      if (lane < 2) cp_async16(dst + RECORD_BYTES + 16 * lane, sg.mod0 + (size_t)win * W + 16 * lane);
+    }
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int k = 0; k < PREFETCH; k++) issue(k);
+
+  for (int k = 0; k <= sg.n_my; k++) {
+    if (k < sg.n_my) {
+      issue(k + PREFETCH);
+      cp_async_wait<PREFETCH>();
+      __syncwarp();
+      const unsigned char* st = sm.stage[pair][k % NSTAGE];
+      const uint4* mp = reinterpret_cast<const uint4*>(st + OFF_KM + 64 * t);
+      const uint4* sp = reinterpret_cast<const uint4*>(st + OFF_KS + 64 * t);
+      // bias sum_c q'_c m_c (against the constant operand 4^j 2^-24, two independent chains)
+      // and scores sum_c q'_c s_c code_c, one k-step (16 channels) at a time
+      float dbA[4] = {0.f, 0.f, 0.f, 0.f}, dbB[4] = {0.f, 0.f, 0.f, 0.f};
+      float d[4][4];
+#pragma unroll
+      for (int nu = 0; nu < 4; nu++)
+#pragma unroll
+        for (int i = 0; i < 4; i++) d[nu][i] = 0.f;
+      const uint4 kc0 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * lane);
+      const uint4 kc1 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 512 + 16 * lane);
+      const uint32_t kw[4][2] = {{kc0.x, kc0.y}, {kc0.z, kc0.w}, {kc1.x, kc1.y}, {kc1.z, kc1.w}};
+#pragma unroll
+      for (int kq = 0; kq < 4; kq++) {
+        const uint4 m4 = mp[kq], s4 = sp[kq];
+#pragma unroll
+        for (int half = 0; half < 2; half++) {
+          const int kappa = 2 * kq + half;
+          const uint2 q0 = sm.qf[2 * kappa][lane], q1 = sm.qf[2 * kappa + 1][lane];
+          uint32_t a0, a1, a2, a3;
+          split_product(u2h(q0.x), u2h(q0.y), u2h(half ? m4.z : m4.x), a0, a1);
+          split_product(u2h(q1.x), u2h(q1.y), u2h(half ? m4.w : m4.y), a2, a3);
+          if (half) mma16816(dbB, a0, a1, a2, a3, 0x00100010u, 0x00400040u);
+          else mma16816(dbA, a0, a1, a2, a3, 0x00010001u, 0x00040004u);
+          split_product(u2h(q0.x), u2h(q0.y), u2h(half ? s4.z : s4.x), a0, a1);
+          split_product(u2h(q1.x), u2h(q1.y), u2h(half ? s4.w : s4.y), a2, a3);
+          const int ww = kappa >> 2, sh = (kappa >> 1) & 1;
+          const uint32_t mk0 = half ? 0x00300030u : 0x00030003u;
+          const uint32_t mk1 = half ? 0x00c000c0u : 0x000c000cu;
+#pragma unroll
+          for (int nu = 0; nu < 4; nu++) {
+            uint32_t src = sh ? (kw[nu][ww] >> 8) : kw[nu][ww];
+            mma16816(d[nu], a0, a1, a2, a3, src & mk0, src & mk1);
+          }
+        }
+      }
+      // online softmax (log2 domain); this lane: head g, tokens 8*nu + 2*t + e
+      const uint4 kn4 = *reinterpret_cast<const uint4*>(st + OFF_KNORM + 16 * t);
+      const uint4 vn4 = *reinterpret_cast<const uint4*>(st + OFF_VNORM + 16 * t);
+      const uint32_t knu[4] = {kn4.x, kn4.y, kn4.z, kn4.w}, vnu[4] = {vn4.x, vn4.y, vn4.z, vn4.w};
+      const float bias0 = (dbA[0] + dbB[0]) + (dbA[2] + dbB[2]), bias1 = (dbA[1] + dbB[1]) + (dbA[3] + dbB[3]);
+      float sc[4][2];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int nu = 0; nu < 4; nu++) {
+        float2 kn = __half22float2(u2h(knu[nu]));
+        sc[nu][0] = ((d[nu][0] + d[nu][2]) + bias0) * (kn.x * fsc);
+        sc[nu][1] = ((d[nu][1] + d[nu][3]) + bias1) * (kn.y * fsc);
+        mx = fmaxf(mx, fmaxf(sc[nu][0], sc[nu][1]));
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(run_m, mx);
+      const float alpha = ex2(run_m - m_new);  // 0 on the first window
+      const int changed = __any_sync(0xffffffffu, m_new > run_m);
+      run_l *= alpha;
+      run_m = m_new;
+      Handoff& ho = sm.hand[pair][k & 1];
+      uint32_t pb[4];
+#pragma unroll
+      for (int nu = 0; nu < 4; nu++) {
+        float2 vn = __half22float2(u2h(vnu[nu]));
+        const float off = (float)(6 - 2 * nu) - run_m;
+        const float cinv = (float)(1 << (2 * nu)) * (1.0f / 64.0f);
+        float p0 = ex2(sc[nu][0] + off), p1 = ex2(sc[nu][1] + off);
+        run_l = fmaf(p0 + p1, cinv, run_l);
+        pb[nu] = pack_sat(p0 * vn.x, p1 * vn.y);
+      }
+#pragma unroll
+      for (int nu = 0; nu < 4; nu++) ho.pb[nu][lane] = pb[nu];
+      if (t == 0) { ho.m[g] = run_m; ho.alpha[g] = alpha; }
+      if (lane == 0) ho.rescale = changed;
+    }
+    pair_barrier(pair);
+  }
+  cp_async_wait<0>();
+  run_m_out = run_m;
+  run_l_out = run_l;
+}
+
+// ---------------------------------------------------------------- value warp
+__device__ __forceinline__ void value_warp(MmaSmem& sm, const Segment& sg, int pair, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  float acc[8][4];
+#pragma unroll
+  for (int mu = 0; mu < 8; mu++)
+#pragma unroll
+    for (int i = 0; i < 4; i++) acc[mu][i] = 0.f;
+  float run_S = 0.f;
+  int cur_mod = -1;
+  float cur_m = -INFINITY;   // running maximum of head g the live accumulators refer to
+
+  auto park = [&]() {
+    float* dst = &sm.spill[pair][cur_mod][0][lane];
+#pragma unroll
+    for (int mu = 0; mu < 8; mu++)
+#pragma unroll
+      for (int i = 0; i < 4; i++) dst[(4 * mu + i) * 32] = acc[mu][i];
+    dst[32 * 32] = run_S;
+    if (t == 0) sm.spill_m[pair][cur_mod][g] = cur_m;
+  };
+
+  for (int k = 0; k <= sg.n_my; k++) {
+    if (k >= 1) {
+      const unsigned char* st = sm.stage[pair][(k - 1) % NSTAGE];
+      const Handoff& ho = sm.hand[pair][(k - 1) & 1];
+      if (ho.rescale) {
+        const float a_lo = ho.alpha[2 * t], a_hi = ho.alpha[2 * t + 1];
+#pragma unroll
+        for (int mu = 0; mu < 8; mu++) {
+          acc[mu][0] *= a_lo; acc[mu][1] *= a_hi; acc[mu][2] *= a_lo; acc[mu][3] *= a_hi;
+        }
+        run_S *= ho.alpha[g];
+      }
+      cur_m = ho.m[g];
+      const unsigned char* wmod = st + RECORD_BYTES;
+      const int mymod = wmod[lane];
+      const int first = __shfl_sync(0xffffffffu, mymod, 0);
+      const bool uniform = __all_sync(0xffffffffu, mymod == first);
+      unsigned present = uniform ? (1u << first)
+                                 : ((__any_sync(0xffffffffu, mymod == 0) ? 1u : 0u) |
+                                    (__any_sync(0xffffffffu, mymod == 1) ? 2u : 0u) |
+                                    (__any_sync(0xffffffffu, mymod == 2) ? 4u : 0u));
+      const uint4 vc0 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 16 * lane);
+      const uint4 vc1 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 512 + 16 * lane);
+      const uint32_t vw[8] = {vc0.x, vc0.y, vc0.z, vc0.w, vc1.x, vc1.y, vc1.z, vc1.w};
+      uint32_t pb[4];
+#pragma unroll
+      for (int nu = 0; nu < 4; nu++) pb[nu] = ho.pb[nu][lane];
+      // (3a - b) / (2 (b - a)): weight of the bit-1 plane relative to the code plane
+      constexpr float DELTA_REL = (3.0f * CB_INNER - CB_OUTER) / (2.0f * (CB_OUTER - CB_INNER));
+      const __half2 drel = __float2half2_rn(DELTA_REL);
+      for (int pass = 0; pass < 3 && present; pass++) {
+        int m = (cur_mod >= 0 && (present >> cur_mod) & 1) ? cur_mod : (__ffs(present) - 1);
+        present &= ~(1u << m);
+        if (m != cur_mod) {
+          if (cur_mod >= 0) park();
+          __syncwarp();
+          const float* src = &sm.spill[pair][m][0][lane];
+          const float sm_lo = sm.spill_m[pair][m][2 * t], sm_hi = sm.spill_m[pair][m][2 * t + 1];
+          const float sm_g = sm.spill_m[pair][m][g];
+          const float f_lo = sm_lo == -INFINITY ? 0.f : ex2(sm_lo - ho.m[2 * t]);
+          const float f_hi = sm_hi == -INFINITY ? 0.f : ex2(sm_hi - ho.m[2 * t + 1]);
+          const float f_g = sm_g == -INFINITY ? 0.f : ex2(sm_g - cur_m);
+#pragma unroll
+          for (int mu = 0; mu < 8; mu++) {
+            acc[mu][0] = src[(4 * mu + 0) * 32] * f_lo; acc[mu][1] = src[(4 * mu + 1) * 32] * f_hi;
+            acc[mu][2] = src[(4 * mu + 2) * 32] * f_lo; acc[mu][3] = src[(4 * mu + 3) * 32] * f_hi;
+          }
+          run_S = src[32 * 32] * f_g;
+          cur_mod = m;
+          __syncwarp();
+        }
+        uint32_t b0[4], b1[4];
+        unsigned halfmask = 3u;  // which 16-token halves hold a token of modality m
+        if (uniform) {
+#pragma unroll
+          for (int nu = 0; nu < 4; nu++) b0[nu] = pb[nu];
+        } else {
+          bool any_lo = false, any_hi = false;
+#pragma unroll
+          for (int nu = 0; nu < 4; nu++) {
+            const bool k0 = wmod[8 * nu + 2 * t] == m, k1 = wmod[8 * nu + 2 * t + 1] == m;
+            b0[nu] = pb[nu] & ((k0 ? 0x0000ffffu : 0u) | (k1 ? 0xffff0000u : 0u));
+            if (nu < 2) any_lo |= (k0 | k1); else any_hi |= (k0 | k1);
+          }
+          halfmask = (__any_sync(0xffffffffu, any_lo) ? 1u : 0u) | (__any_sync(0xffffffffu, any_hi) ? 2u : 0u);
+        }
+#pragma unroll
+        for (int nu = 0; nu < 4; nu++) {
+          b1[nu] = h2u(__hmul2(u2h(b0[nu]), drel));
+          float2 pf = __half22float2(u2h(b0[nu]));   // weight sum from the rounded numerators
+          run_S = fmaf(pf.x + pf.y, (float)(1 << (2 * nu)) * (1.0f / 64.0f), run_S);
+        }
+#pragma unroll 1   // rolled on purpose: unrolling both halves makes ptxas spill the accumulators
+        for (int kv = 0; kv < 2; kv++) {
+          if (!((halfmask >> kv) & 1)) continue;
+          const uint32_t mA = 0x00030003u << (4 * kv), mB = 0x000c000cu << (4 * kv);
+          const uint32_t nA = 0x00020002u << (4 * kv), nB = 0x00080008u << (4 * kv);
+          const uint32_t p0 = kv ? b0[2] : b0[0], p1 = kv ? b0[3] : b0[1];
+          const uint32_t q0 = kv ? b1[2] : b1[0], q1 = kv ? b1[3] : b1[1];
+#pragma unroll
+          for (int mu = 0; mu < 8; mu++) {
+            const uint32_t w = vw[mu], w8 = w >> 8;
+            mma16816(acc[mu], w & mA, w8 & mA, w & mB, w8 & mB, p0, p1);
+            mma16816(acc[mu], w & nA, w8 & nA, w & nB, w8 & nB, q0, q1);
+          }
+        }
+      }
+    }
+    pair_barrier(pair);
+  }
+  if (cur_mod >= 0) park();
+}
+
 }  // namespace
 
-// grid = n_cta (persistent), 256 threads
-__global__ void __launch_bounds__(NWARP * 32, 1) k_decode_mma(DecodeParams P) {
+// grid = n_cta (persistent), 512 threads
+__global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   MmaSmem& sm = *reinterpret_cast<MmaSmem*>(smem_raw);
   const CacheView& cv = P.cv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t = lane & 3;
+  const int pair = warp & (NPAIR - 1);
+  const bool is_score = warp < NPAIR;
   const int G = P.group, Hkv = cv.n_kv_heads;
   const int n_entries = P.layer_count * cv.batch;
 
@@ -108,9 +367,10 @@ __global__ void __launch_bounds__(NWARP * 32, 1) k_decode_mma(DecodeParams P) {
     const int seg = min(pos_end - pos, nwin - w0);
     const int unit = e * Hkv + h;
 
-    // ---- per-segment setup: q' for the group's heads, scaled to the fp16 range
-    {
-      const int hh = warp;  // one head per warp (GP == NWARP)
+    // ---- per-segment setup
+    if (is_score) {
+      // q' for head `pair` of the group, scaled into the fp16 range
+      const int hh = pair;
       float4 qr = make_float4(0, 0, 0, 0);
       if (hh < G) {
         const __half* qrow = P.q + (((size_t)li * cv.batch + b) * cv.n_q_heads + h * G + hh) * D;
@@ -128,275 +388,65 @@ __global__ void __launch_bounds__(NWARP * 32, 1) k_decode_mma(DecodeParams P) {
       const float up = exp2f((float)kh);
       *reinterpret_cast<float4*>(&sm.qs[hh][4 * lane]) = make_float4(v[0] * up, v[1] * up, v[2] * up, v[3] * up);
       if (lane == 0) sm.fscale[hh] = exp2f((float)(24 - kh)) * P.sm_scale * 1.4426950408889634f;
-      // clear this warp's spilled accumulators
-      float* sp = &sm.spill[warp][0][0][0];
+    } else {
+      // clear this pair's parked accumulators
+      float* sp = &sm.spill[pair][0][0][0];
       for (int i = lane; i < 3 * SPILL_REGS * 32; i += 32) sp[i] = 0.f;
-      if (lane < 3 * GP) (&sm.spill_m[warp][0][0])[lane] = -INFINITY;
+      if (lane < 3 * GP) (&sm.spill_m[pair][0][0])[lane] = -INFINITY;
     }
     __syncthreads();
-
-    // query fragments: head g, channels {16k + 8p + 2t + e}, pre-divided by 4^j, j = (2k + p) & 3
-    __half2 qh[16], ql[16];
-#pragma unroll
-    for (int r = 0; r < 16; r++) {
-      const int c0 = 16 * (r >> 1) + 8 * (r & 1) + 2 * t;
+    {  // fragment registers of the queries: lane (g, t) holds head g, channels {16k + 8p + 2t + e} for
+       // r = 2k + p, pre-divided by 4^(r&3) (the position scale of the matching code field)
+      const int r = tid >> 5, gg = lane >> 2, tt = lane & 3;
+      const int c0 = 16 * (r >> 1) + 8 * (r & 1) + 2 * tt;
       const float sc = 1.0f / (float)(1 << (2 * (r & 3)));
-      float x0 = sm.qs[g][c0] * sc, x1 = sm.qs[g][c0 + 1] * sc;
-      __half2 hi2 = __floats2half2_rn(x0, x1);
-      float2 hf = __half22float2(hi2);
-      qh[r] = hi2;
-      ql[r] = __floats2half2_rn(x0 - hf.x, x1 - hf.y);
-    }
-    const float fsc = sm.fscale[g];
-
-    float acc[8][4];
-#pragma unroll
-    for (int mu = 0; mu < 8; mu++)
-#pragma unroll
-      for (int k = 0; k < 4; k++) acc[mu][k] = 0.f;
-    float run_m = -INFINITY, run_l = 0.f, run_S = 0.f;
-    int cur_mod = -1;
-
-    // ---- this warp's windows: w0 + warp, w0 + warp + NWARP, ...
-    const int n_my = seg > warp ? (seg - warp + NWARP - 1) / NWARP : 0;
-    const unsigned char* rec0 = cv.record(layer, b, h, 0);
-    const unsigned char* mod0 = cv.modality + (size_t)b * cv.capacity;
-    auto issue = [&](int k) {
-      if (k < n_my) {
-        const int win = w0 + warp + k * NWARP;
-        unsigned char* dst = sm.stage[warp][k % NSTAGE];
-        const unsigned char* src = rec0 + (size_t)win * RECORD_BYTES;
-#pragma unroll
-        for (int i = 0; i < 6; i++) {
-          int c16 = lane + 32 * i;
-          if (c16 < RECORD_BYTES / 16) cp_async16(dst + 16 * c16, src + 16 * c16);
-        }
-        if (lane < 2) cp_async16(dst + RECORD_BYTES + 16 * lane, mod0 + (size_t)win * W + 16 * lane);
-      }
-      cp_async_commit();
-    };
-#pragma unroll
-    for (int k = 0; k < NSTAGE - 1; k++) issue(k);
-
-    for (int k = 0; k < n_my; k++) {
-      issue(k + NSTAGE - 1);
-      cp_async_wait<NSTAGE - 1>();
-      __syncwarp();
-      const unsigned char* st = sm.stage[warp][k % NSTAGE];
-
-      // ================= scores =================
-      const uint4* mp = reinterpret_cast<const uint4*>(st + OFF_KM + 64 * t);
-      const uint4* sp = reinterpret_cast<const uint4*>(st + OFF_KS + 64 * t);
-      float db[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int kq = 0; kq < 4; kq++) {  // bias: sum_c q'_c m_c against the constant operand 4^j 2^-24
-        uint4 m4 = mp[kq];
-        uint32_t a0, a1, a2, a3;
-        split_product(qh[4 * kq + 0], ql[4 * kq + 0], u2h(m4.x), a0, a1);
-        split_product(qh[4 * kq + 1], ql[4 * kq + 1], u2h(m4.y), a2, a3);
-        mma16816(db, a0, a1, a2, a3, 0x00010001u, 0x00040004u);
-        split_product(qh[4 * kq + 2], ql[4 * kq + 2], u2h(m4.z), a0, a1);
-        split_product(qh[4 * kq + 3], ql[4 * kq + 3], u2h(m4.w), a2, a3);
-        mma16816(db, a0, a1, a2, a3, 0x00100010u, 0x00400040u);
-      }
-      float d[4][4];
-#pragma unroll
-      for (int nu = 0; nu < 4; nu++)
-#pragma unroll
-        for (int i = 0; i < 4; i++) d[nu][i] = db[i];
-      {
-        const uint4 kc0 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * lane);
-        const uint4 kc1 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 512 + 16 * lane);
-        // word[nu][ww]
-        const uint32_t kw[4][2] = {{kc0.x, kc0.y}, {kc0.z, kc0.w}, {kc1.x, kc1.y}, {kc1.z, kc1.w}};
-#pragma unroll
-        for (int kq = 0; kq < 4; kq++) {
-          uint4 s4 = sp[kq];
-#pragma unroll
-          for (int half = 0; half < 2; half++) {
-            const int kappa = 2 * kq + half;
-            uint32_t a0, a1, a2, a3;
-            split_product(qh[2 * kappa], ql[2 * kappa], u2h(half ? s4.z : s4.x), a0, a1);
-            split_product(qh[2 * kappa + 1], ql[2 * kappa + 1], u2h(half ? s4.w : s4.y), a2, a3);
-            const int ww = kappa >> 2, sh = (kappa >> 1) & 1;
-            const uint32_t mk0 = half ? 0x00300030u : 0x00030003u;
-            const uint32_t mk1 = half ? 0x00c000c0u : 0x000c000cu;
-#pragma unroll
-            for (int nu = 0; nu < 4; nu++) {
-              uint32_t src = sh ? (kw[nu][ww] >> 8) : kw[nu][ww];
-              mma16816(d[nu], a0, a1, a2, a3, src & mk0, src & mk1);
-            }
-          }
-        }
-      }
-
-      // ================= online softmax (log2 domain) =================
-      float sc[4][2], pf[4][2];
-      {
-        const __half2* knp = reinterpret_cast<const __half2*>(st + OFF_KNORM);
-        float mx = -INFINITY;
-#pragma unroll
-        for (int nu = 0; nu < 4; nu++) {
-          float2 kn = __half22float2(knp[4 * nu + t]);
-          sc[nu][0] = (d[nu][0] + d[nu][2]) * (kn.x * fsc);
-          sc[nu][1] = (d[nu][1] + d[nu][3]) * (kn.y * fsc);
-          mx = fmaxf(mx, fmaxf(sc[nu][0], sc[nu][1]));
-        }
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float m_new = fmaxf(run_m, mx);
-        if (__any_sync(0xffffffffu, m_new > run_m)) {
-          const float alpha = exp2f(run_m - m_new);  // 0 on the first window
-          run_l *= alpha;
-          run_S *= alpha;
-          const float a_lo = __shfl_sync(0xffffffffu, alpha, 8 * t);       // head 2t
-          const float a_hi = __shfl_sync(0xffffffffu, alpha, 8 * t + 4);   // head 2t+1
-#pragma unroll
-          for (int mu = 0; mu < 8; mu++) {
-            acc[mu][0] *= a_lo; acc[mu][1] *= a_hi; acc[mu][2] *= a_lo; acc[mu][3] *= a_hi;
-          }
-          run_m = m_new;
-        }
-        const __half2* vnp = reinterpret_cast<const __half2*>(st + OFF_VNORM);
-#pragma unroll
-        for (int nu = 0; nu < 4; nu++) {
-          float2 vn = __half22float2(vnp[4 * nu + t]);
-          float p0 = exp2f(sc[nu][0] - run_m), p1 = exp2f(sc[nu][1] - run_m);
-          run_l += p0 + p1;
-          pf[nu][0] = p0 * vn.x;
-          pf[nu][1] = p1 * vn.y;
-        }
-      }
-
-      // ================= values =================
-      const unsigned char* wmod = st + RECORD_BYTES;
-      const int mymod = wmod[lane];
-      const int first = __shfl_sync(0xffffffffu, mymod, 0);
-      const bool uniform = __all_sync(0xffffffffu, mymod == first);
-      unsigned present = uniform ? (1u << first)
-                                 : ((__any_sync(0xffffffffu, mymod == 0) ? 1u : 0u) |
-                                    (__any_sync(0xffffffffu, mymod == 1) ? 2u : 0u) |
-                                    (__any_sync(0xffffffffu, mymod == 2) ? 4u : 0u));
-      const uint4 vc0 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 16 * lane);
-      const uint4 vc1 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 512 + 16 * lane);
-      const uint32_t vw[8] = {vc0.x, vc0.y, vc0.z, vc0.w, vc1.x, vc1.y, vc1.z, vc1.w};
-      // numerators as fp16 pairs: p * vnorm * 2^6 / 4^nu, and the same times (3a-b)/(2(b-a))
-      constexpr float DELTA_REL = (3.0f * CB_INNER - CB_OUTER) / (2.0f * (CB_OUTER - CB_INNER));
-      uint32_t pb[4], pd[4];
-#pragma unroll
-      for (int nu = 0; nu < 4; nu++) {
-        const float c = 64.0f / (float)(1 << (2 * nu));
-        pb[nu] = pack_sat(pf[nu][0] * c, pf[nu][1] * c);
-        pd[nu] = pack_sat(pf[nu][0] * (c * DELTA_REL), pf[nu][1] * (c * DELTA_REL));
-      }
-      // process the modalities present, starting with the one already in registers
-      for (int pass = 0; pass < 3 && present; pass++) {
-        int m = (cur_mod >= 0 && (present >> cur_mod) & 1) ? cur_mod : (__ffs(present) - 1);
-        present &= ~(1u << m);
-        if (m != cur_mod) {
-          // swap accumulators: park the current modality, fetch modality m rescaled to run_m
-          if (cur_mod >= 0) {
-            float* dst = &sm.spill[warp][cur_mod][0][lane];
-#pragma unroll
-            for (int mu = 0; mu < 8; mu++)
-#pragma unroll
-              for (int i = 0; i < 4; i++) dst[(4 * mu + i) * 32] = acc[mu][i];
-            dst[32 * 32] = run_S;
-            if (t == 0) sm.spill_m[warp][cur_mod][g] = run_m;
-          }
-          __syncwarp();
-          const float* src = &sm.spill[warp][m][0][lane];
-          const float sm_lo = sm.spill_m[warp][m][2 * t], sm_hi = sm.spill_m[warp][m][2 * t + 1];
-          const float sm_g = sm.spill_m[warp][m][g];
-          const float m_lo = __shfl_sync(0xffffffffu, run_m, 8 * t), m_hi = __shfl_sync(0xffffffffu, run_m, 8 * t + 4);
-          const float f_lo = sm_lo == -INFINITY ? 0.f : exp2f(sm_lo - m_lo);
-          const float f_hi = sm_hi == -INFINITY ? 0.f : exp2f(sm_hi - m_hi);
-          const float f_g = sm_g == -INFINITY ? 0.f : exp2f(sm_g - run_m);
-#pragma unroll
-          for (int mu = 0; mu < 8; mu++) {
-            acc[mu][0] = src[(4 * mu + 0) * 32] * f_lo; acc[mu][1] = src[(4 * mu + 1) * 32] * f_hi;
-            acc[mu][2] = src[(4 * mu + 2) * 32] * f_lo; acc[mu][3] = src[(4 * mu + 3) * 32] * f_hi;
-          }
-          run_S = src[32 * 32] * f_g;
-          cur_mod = m;
-          __syncwarp();
-        }
-        uint32_t b0[4], b1[4];
-        unsigned halfmask = 3u;  // which 16-token halves hold a token of modality m
-        if (uniform) {
-#pragma unroll
-          for (int nu = 0; nu < 4; nu++) { b0[nu] = pb[nu]; b1[nu] = pd[nu]; run_S += pf[nu][0] + pf[nu][1]; }
-        } else {
-          bool any_lo = false, any_hi = false;
-#pragma unroll
-          for (int nu = 0; nu < 4; nu++) {
-            const bool k0 = wmod[8 * nu + 2 * t] == m, k1 = wmod[8 * nu + 2 * t + 1] == m;
-            const uint32_t msk = (k0 ? 0x0000ffffu : 0u) | (k1 ? 0xffff0000u : 0u);
-            b0[nu] = pb[nu] & msk;
-            b1[nu] = pd[nu] & msk;
-            run_S += (k0 ? pf[nu][0] : 0.f) + (k1 ? pf[nu][1] : 0.f);
-            if (nu < 2) any_lo |= (k0 | k1); else any_hi |= (k0 | k1);
-          }
-          halfmask = (__any_sync(0xffffffffu, any_lo) ? 1u : 0u) | (__any_sync(0xffffffffu, any_hi) ? 2u : 0u);
-        }
-#pragma unroll
-        for (int kv = 0; kv < 2; kv++) {
-          if (!((halfmask >> kv) & 1)) continue;
-          const uint32_t mA = 0x00030003u << (4 * kv), mB = 0x000c000cu << (4 * kv);
-          const uint32_t nA = 0x00020002u << (4 * kv), nB = 0x00080008u << (4 * kv);
-#pragma unroll
-          for (int mu = 0; mu < 8; mu++) {
-            const uint32_t w = vw[mu], w8 = w >> 8;
-            mma16816(acc[mu], w & mA, w8 & mA, w & mB, w8 & mB, b0[2 * kv], b0[2 * kv + 1]);
-            mma16816(acc[mu], w & nA, w8 & nA, w & nB, w8 & nB, b1[2 * kv], b1[2 * kv + 1]);
-          }
-        }
-      }
-      __syncwarp();  // every lane is done with this stage before it is refilled
-    }
-    cp_async_wait<0>();
-
-    // ---- park the live accumulators and merge the warps
-    if (cur_mod >= 0) {
-      float* dst = &sm.spill[warp][cur_mod][0][lane];
-#pragma unroll
-      for (int mu = 0; mu < 8; mu++)
-#pragma unroll
-        for (int i = 0; i < 4; i++) dst[(4 * mu + i) * 32] = acc[mu][i];
-      dst[32 * 32] = run_S;
-      if (t == 0) sm.spill_m[warp][cur_mod][g] = run_m;
-    }
-    {
-      float lt = run_l;
-      lt += __shfl_xor_sync(0xffffffffu, lt, 1);
-      lt += __shfl_xor_sync(0xffffffffu, lt, 2);
-      if (t == 0) { sm.wm[warp][g] = run_m; sm.wl[warp][g] = lt; }
+      const float x0 = sm.qs[gg][c0] * sc, x1 = sm.qs[gg][c0 + 1] * sc;
+      const __half2 hi2 = __floats2half2_rn(x0, x1);
+      const float2 hf = __half22float2(hi2);
+      sm.qf[r][lane] = make_uint2(h2u(hi2), h2u(__floats2half2_rn(x0 - hf.x, x1 - hf.y)));
     }
     __syncthreads();
+
+    Segment sg;
+    sg.rec0 = cv.record(layer, b, h, 0);
+    sg.mod0 = cv.modality + (size_t)b * cv.capacity;
+    sg.w0 = w0 + pair;
+    sg.n_my = seg > pair ? (seg - pair + NPAIR - 1) / NPAIR : 0;
+    if (is_score) {
+      float run_m, run_l;
+      score_warp(sm, sg, pair, lane, run_m, run_l);
+      run_l += __shfl_xor_sync(0xffffffffu, run_l, 1);
+      run_l += __shfl_xor_sync(0xffffffffu, run_l, 2);
+      if ((lane & 3) == 0) { sm.wm[pair][lane >> 2] = run_m; sm.wl[pair][lane >> 2] = run_l; }
+    } else {
+      value_warp(sm, sg, pair, lane);
+    }
+    __syncthreads();
+
+    // ---- merge the eight pairs into one partial
     PartialF* out = P.partials_f + (size_t)unit + blockIdx.x;
     {
-      // every thread needs the merged maxima of the heads it touches
       float M[GP];
 #pragma unroll
       for (int j = 0; j < GP; j++) {
         float mj = -INFINITY;
 #pragma unroll
-        for (int w8 = 0; w8 < NWARP; w8++) mj = fmaxf(mj, sm.wm[w8][j]);
+        for (int w8 = 0; w8 < NPAIR; w8++) mj = fmaxf(mj, sm.wm[w8][j]);
         M[j] = mj;
       }
       if (tid < GP) {
         float L = 0.f;
-        for (int w8 = 0; w8 < NWARP; w8++)
+        for (int w8 = 0; w8 < NPAIR; w8++)
           L += sm.wm[w8][tid] == -INFINITY ? 0.f : sm.wl[w8][tid] * exp2f(sm.wm[w8][tid] - M[tid]);
         out->m[tid] = M[tid];
         out->l[tid] = L;
       }
-      for (int idx = tid; idx < 3 * SPILL_REGS * 32; idx += NWARP * 32) {
+      for (int idx = tid; idx < 3 * SPILL_REGS * 32; idx += NTHREADS) {
         const int l32 = idx & 31, r = (idx >> 5) % SPILL_REGS, m = idx / (SPILL_REGS * 32);
         const int head = r < 32 ? 2 * (l32 & 3) + (r & 1) : (l32 >> 2);
         float v = 0.f;
 #pragma unroll
-        for (int w8 = 0; w8 < NWARP; w8++) {
+        for (int w8 = 0; w8 < NPAIR; w8++) {
           const float smx = sm.spill_m[w8][m][head];
           if (smx != -INFINITY) v = fmaf(sm.spill[w8][m][r][l32], exp2f(smx - M[head]), v);
         }
@@ -518,7 +568,7 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
     attr_set = true;
   }
   if (before) cudaEventRecord(before, s);
-  k_decode_mma<<<n_cta, NWARP * 32, sizeof(MmaSmem), s>>>(P);
+  k_decode_mma<<<n_cta, NTHREADS, sizeof(MmaSmem), s>>>(P);
   if (after) cudaEventRecord(after, s);
   k_combine_mma<<<dim3(P.cv.n_kv_heads, P.cv.batch * P.layer_count), 128, 0, s>>>(P, n_cta);
   return OKQ_OK;

@@ -14,6 +14,8 @@
 //    Lane l = 4*g + t owns the channels {16*mu + 8*sh + g} (mu = 0..7, sh = 0/1) and the
 //    tokens {16*kv + 8*pv + 2*t + e}: one word per mu, field index j = 2*kv + pv at bit
 //    offset 8*sh + 2*j, token parity e in the low/high half.
+//  * The 32 key norms (and value norms) are stored in the order norm_pos(i), which puts the
+//    eight tokens whose scores a lane receives next to each other.
 //  * (m, s) are stored as two planes of 128 fp16 in the order pi(c) that makes each
 //    lane's 32 channels contiguous.
 #pragma once
@@ -38,6 +40,13 @@ __host__ __device__ inline int meta_pos(int c) {
   int kappa = c >> 4, slot = c & 15;
   int pair = slot >> 3, t = (slot & 7) >> 1, e = slot & 1;
   return t * 32 + kappa * 4 + pair * 2 + e;
+}
+
+// position of token i inside the key-norm / value-norm arrays: the four lanes of a quad each
+// find the norms of "their" tokens {8*nu + 2*t + e} in 16 contiguous bytes
+__host__ __device__ inline int norm_pos(int i) {
+  int nu = i >> 3, t = (i & 7) >> 1, e = i & 1;
+  return 8 * t + 2 * nu + e;
 }
 
 // key code of (token i in window, channel c): 32-bit word index in the key-code block and bit offset

@@ -43,7 +43,7 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
       z = make_float4(__fmul_rn(y.x, cinv), __fmul_rn(y.y, cinv), __fmul_rn(y.z, cinv), __fmul_rn(y.w, cinv));
     }
     *reinterpret_cast<float4*>(&sm.z[i * ZS + 4 * lane]) = z;
-    if (lane == 0) knorm[i] = nh;
+    if (lane == 0) knorm[norm_pos(i)] = nh;
   }
   __syncthreads();
   {  // per channel: window minimum and step (Eq. 4)
@@ -104,7 +104,7 @@ __device__ void quantize_value_window(const __half* rows, long long stride, cons
     float nf = __half2float(nh);
     *reinterpret_cast<float4*>(&sm.z[i * ZS + 4 * lane]) = x;
     if (lane == 0) {
-      vnorm[i] = nh;
+      vnorm[norm_pos(i)] = nh;
       sm.inv[i] = nf != 0.0f ? __fdiv_rn(1.0f, nf) : 0.0f;
     }
   }
@@ -302,8 +302,8 @@ __global__ void k_export(CacheView cv, int layer, unsigned char* k_codes, __half
     v_codes[(tok0 + i) * 32 + byte] = (unsigned char)vb;
   }
   if (threadIdx.x < W) {
-    k_norm[tok0 + threadIdx.x] = reinterpret_cast<const __half*>(rec + OFF_KNORM)[threadIdx.x];
-    v_norm[tok0 + threadIdx.x] = reinterpret_cast<const __half*>(rec + OFF_VNORM)[threadIdx.x];
+    k_norm[tok0 + threadIdx.x] = reinterpret_cast<const __half*>(rec + OFF_KNORM)[norm_pos(threadIdx.x)];
+    v_norm[tok0 + threadIdx.x] = reinterpret_cast<const __half*>(rec + OFF_VNORM)[norm_pos(threadIdx.x)];
   }
   {
     int c = threadIdx.x, p = meta_pos(c);
@@ -339,8 +339,8 @@ __global__ void k_import(CacheView cv, int layer, const unsigned char* k_codes, 
     reinterpret_cast<uint32_t*>(rec + OFF_VCODE)[i] = vw[i];
   }
   if (threadIdx.x < W) {
-    reinterpret_cast<__half*>(rec + OFF_KNORM)[threadIdx.x] = k_norm[tok0 + threadIdx.x];
-    reinterpret_cast<__half*>(rec + OFF_VNORM)[threadIdx.x] = v_norm[tok0 + threadIdx.x];
+    reinterpret_cast<__half*>(rec + OFF_KNORM)[norm_pos(threadIdx.x)] = k_norm[tok0 + threadIdx.x];
+    reinterpret_cast<__half*>(rec + OFF_VNORM)[norm_pos(threadIdx.x)] = v_norm[tok0 + threadIdx.x];
   }
   {
     int c = threadIdx.x, p = meta_pos(c);
