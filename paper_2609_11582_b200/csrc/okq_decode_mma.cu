@@ -35,10 +35,11 @@ constexpr int NTHREADS = NPAIR * 64;
 constexpr int NSTAGE = 4;                       // record ring per pair
 constexpr int PREFETCH = 2;                     // windows in flight ahead of the score warp
 constexpr int STAGE_BYTES = RECORD_BYTES + 32;  // record + the window's 32 modality bytes
+constexpr float RESCALE_LOG2 = 3.0f;            // numerators stay below 2^3 * 2^6 * vnorm in fp16
 constexpr int SPILL_REGS = 33;                  // 32 accumulator registers + the running weight sum
 
 struct Handoff {
-  uint32_t pb[4][32];   // per lane: numerators p * vnorm * 2^6 / 4^nu of its 8 tokens, fp16 pairs
+  uint4 pb[32];         // per lane: numerators p * vnorm * 2^6 / 4^nu of its 8 tokens, fp16 pairs (nu = x,y,z,w)
   float m[GP];          // running maximum per head after this window (log2 domain)
   float alpha[GP];      // factor the value accumulators must be multiplied by before this window
   int rescale;          // non-zero if any alpha != 1
@@ -105,7 +106,7 @@ __device__ __forceinline__ void split_product(__half2 qh, __half2 ql, __half2 x,
 struct Segment {
   const unsigned char* rec0;   // first record of the (layer, sequence, head)
   const unsigned char* mod0;   // modality row of the sequence
-  int w0, n_my;                // first window of this pair's list, number of windows (stride NPAIR)
+  int w0, n_my;                // this pair's contiguous window range: first window, count
 };
 
 // ---------------------------------------------------------------- score warp
@@ -117,7 +118,7 @@ __device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int p
 
   auto issue = [&](int k) {
     if (k < sg.n_my) {
-      const int win = sg.w0 + k * NPAIR;
+      const int win = sg.w0 + k;
       unsigned char* dst = sm.stage[pair][k % NSTAGE];
       const unsigned char* src = sg.rec0 + (size_t)win * RECORD_BYTES;
 #pragma unroll
@@ -191,7 +192,9 @@ __device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int p
       }
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      const float m_new = fmaxf(run_m, mx);
+      // the reference maximum only moves when it is exceeded by more than 2^RESCALE_LOG2, so the
+      // value accumulators are rescaled a few times per range instead of at every new maximum
+      const float m_new = mx > run_m + RESCALE_LOG2 ? mx : run_m;
       const float alpha = ex2(run_m - m_new);  // 0 on the first window
       const int changed = __any_sync(0xffffffffu, m_new > run_m);
       run_l *= alpha;
@@ -207,8 +210,7 @@ __device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int p
         run_l = fmaf(p0 + p1, cinv, run_l);
         pb[nu] = pack_sat(p0 * vn.x, p1 * vn.y);
       }
-#pragma unroll
-      for (int nu = 0; nu < 4; nu++) ho.pb[nu][lane] = pb[nu];
+      ho.pb[lane] = make_uint4(pb[0], pb[1], pb[2], pb[3]);
       if (t == 0) { ho.m[g] = run_m; ho.alpha[g] = alpha; }
       if (lane == 0) ho.rescale = changed;
     }
@@ -265,9 +267,8 @@ __device__ __forceinline__ void value_warp(MmaSmem& sm, const Segment& sg, int p
       const uint4 vc0 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 16 * lane);
       const uint4 vc1 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 512 + 16 * lane);
       const uint32_t vw[8] = {vc0.x, vc0.y, vc0.z, vc0.w, vc1.x, vc1.y, vc1.z, vc1.w};
-      uint32_t pb[4];
-#pragma unroll
-      for (int nu = 0; nu < 4; nu++) pb[nu] = ho.pb[nu][lane];
+      const uint4 pb4 = ho.pb[lane];
+      const uint32_t pb[4] = {pb4.x, pb4.y, pb4.z, pb4.w};
       // (3a - b) / (2 (b - a)): weight of the bit-1 plane relative to the code plane
       constexpr float DELTA_REL = (3.0f * CB_INNER - CB_OUTER) / (2.0f * (CB_OUTER - CB_INNER));
       const __half2 drel = __float2half2_rn(DELTA_REL);
@@ -410,8 +411,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
     Segment sg;
     sg.rec0 = cv.record(layer, b, h, 0);
     sg.mod0 = cv.modality + (size_t)b * cv.capacity;
-    sg.w0 = w0 + pair;
-    sg.n_my = seg > pair ? (seg - pair + NPAIR - 1) / NPAIR : 0;
+    const int cnt = (seg + NPAIR - 1) / NPAIR;   // contiguous ranges: few modality changes per pair
+    sg.w0 = w0 + pair * cnt;
+    sg.n_my = max(0, min(cnt, seg - pair * cnt));
     if (is_score) {
       float run_m, run_l;
       score_warp(sm, sg, pair, lane, run_m, run_l);
