@@ -47,6 +47,7 @@ extern "C" {
 #define OKQ_WINDOW 32
 #define OKQ_RECORD_BYTES 2688
 #define OKQ_MAX_GROUP 8
+#define OKQ_NOALLOC_SCRATCH_BYTES (32u << 20) /* fixed scratch of okq_decode_attention_noalloc */
 
 typedef enum {
   OKQ_OK = 0,
@@ -155,6 +156,33 @@ okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t l
                                 const void* q, float sm_scale, const float* signs, const float* R,
                                 int32_t n_R, void* workspace, size_t workspace_bytes,
                                 int32_t num_splits, float* out, void* stream);
+
+/*
+ * okq_decode_attention for callers that have no scratch buffer to give and no way to get
+ * one: code running where cudaMalloc is off limits (inside a serving loop whose memory was
+ * carved up at start-up, under a caching allocator that must not be bypassed, in a plugin
+ * that is only handed its inputs and outputs).  The paper has no counterpart; this is the
+ * same kernel pair with its split-K partials kept in a fixed OKQ_NOALLOC_SCRATCH_BYTES
+ * (32 MiB) array that is part of the library's device image, so every GPU that loads the
+ * library carries those 32 MiB until the process exits.  The call allocates nothing: no
+ * cudaMalloc, no cudaFree, no allocating library routine.
+ *
+ *   - Arguments are those of okq_decode_attention without workspace / workspace_bytes.
+ *   - Limit: (layer_count * batch * n_kv_heads + number of CTAs) * 12736 bytes must fit in the
+ *     scratch, i.e. about 2630 (sequence, KV head) pairs per launch with the automatic grid;
+ *     anything larger returns OKQ_ERR_WORKSPACE and launches nothing (use
+ *     okq_decode_attention with your own buffer).
+ *   - The first call on each device looks up the scratch's device address (with that device
+ *     current) and remembers it; make that first call outside any stream capture.
+ *   - Every call on a device shares the one array.  Nothing in it has to be cleared: each
+ *     launch overwrites the partials it later reads.  Two calls that overlap on the GPU
+ *     (different streams, or different host threads) race on it and give wrong results;
+ *     calls on one stream are ordered and safe.
+ */
+okq_status okq_decode_attention_noalloc(const okq_cache* cache, int32_t layer, int32_t layer_count,
+                                        const void* q, float sm_scale, const float* signs,
+                                        const float* R, int32_t n_R, int32_t num_splits, float* out,
+                                        void* stream);
 
 /*
  * The same computation on CUDA cores only (fp32 multiply-adds, dot products reduced with

@@ -67,6 +67,9 @@ def lib():
                                            C.c_void_p, C.c_void_p]
         L.okq_decode_attention_simt.restype = C.c_int
         L.okq_decode_attention_simt.argtypes = L.okq_decode_attention.argtypes
+        L.okq_decode_attention_noalloc.restype = C.c_int
+        L.okq_decode_attention_noalloc.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32, C.c_void_p, C.c_float,
+                                                   C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.okq_profile_events.restype = None
         L.okq_profile_events.argtypes = [C.c_void_p, C.c_void_p]
         L.okq_cache_export.restype = C.c_int
@@ -80,7 +83,8 @@ def lib():
 def exported_symbols():
     return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
-            "okq_cache_import", "okq_profile_events", "okq_decode_attention_simt"]
+            "okq_cache_import", "okq_profile_events", "okq_decode_attention_simt",
+            "okq_decode_attention_noalloc"]
 
 
 def _ptr(t) -> int:
@@ -173,6 +177,16 @@ def decode_attention(cache: Cache, layer: int, layer_count: int, q, signs, R, wo
     _check(fn(C.byref(cache.c), layer, layer_count, _ptr(q), scale, _ptr(signs), _ptr(R), n_R,
                                       _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
                                       num_splits, _ptr(out), _stream(stream)), "okq_decode_attention")
+
+
+def decode_attention_noalloc(cache: Cache, layer: int, layer_count: int, q, signs, R, out, n_R=1, sm_scale=None,
+                             num_splits=0, stream=None):
+    """okq_decode_attention_noalloc: same result as decode_attention, scratch held inside the library
+    (32 MiB per GPU, shared by all calls on that GPU; overlapping calls race).  Allocates nothing."""
+    scale = HEAD_DIM ** -0.5 if sm_scale is None else sm_scale
+    _check(lib().okq_decode_attention_noalloc(C.byref(cache.c), layer, layer_count, _ptr(q), scale, _ptr(signs),
+                                              _ptr(R), n_R, num_splits, _ptr(out), _stream(stream)),
+           "okq_decode_attention_noalloc")
 
 
 def profile_events(before=None, after=None):

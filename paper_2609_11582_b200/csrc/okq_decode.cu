@@ -350,6 +350,30 @@ __global__ void __launch_bounds__(128) k_combine(DecodeParams P) {
 
 static thread_local cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
+// Scratch of okq_decode_attention_noalloc: lives in the library's device image, so every GPU
+// that loads the library holds these bytes until the process exits.  In host code the name
+// below is only a handle; the device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[OKQ_NOALLOC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+static void* g_noalloc_ptr[MAX_DEVICES];   // device address of g_noalloc_scratch, per device (0 = not resolved yet)
+
+// Resolves the scratch address on the current device (first call per device only).
+static okq_status noalloc_scratch(void** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
+  if (dev < 0 || dev >= MAX_DEVICES) return OKQ_ERR_UNSUPPORTED;
+  void* p = __atomic_load_n(&g_noalloc_ptr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess || !p) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
+    __atomic_store_n(&g_noalloc_ptr[dev], p, __ATOMIC_RELEASE);   // every thread resolves the same address
+  }
+  *out = p;
+  return OKQ_OK;
+}
+
 static int auto_splits(const okq_cache* c, int layer_count) {
   long long units = (long long)layer_count * c->batch * c->n_kv_heads;
   long long want = (2 * 148 + units - 1) / units;
@@ -448,6 +472,35 @@ okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t l
     P.partials_f = static_cast<PartialF*>(workspace);
     const int n_cta = mma_ctas(cache, lc, num_splits);
     st = launch_decode_mma(P, n_cta, s, g_ev_before, g_ev_after);
+    if (st != OKQ_OK) return st;
+  }
+  return launch_status();
+}
+
+okq_status okq_decode_attention_noalloc(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* q,
+                                        float sm_scale, const float* signs, const float* R, int32_t n_R,
+                                        int32_t num_splits, float* out, void* stream) {
+  okq_status st = check_cache(cache, false);
+  if (st != OKQ_OK) return st;
+  if (layer_count <= 0 || num_splits < 0) return OKQ_ERR_INVALID_ARG;
+  // the largest launch of the call decides how much of the fixed scratch is needed
+  const int layers_per_launch = cache->batch >= MAX_ENTRIES ? 1 : MAX_ENTRIES / cache->batch;
+  const int lc_max = layer_count < layers_per_launch ? layer_count : layers_per_launch;
+  if (mma_workspace(cache, lc_max, num_splits) > (size_t)OKQ_NOALLOC_SCRATCH_BYTES) return OKQ_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  st = noalloc_scratch(&scratch);
+  if (st != OKQ_OK) return st;
+  st = check_decode(cache, layer, layer_count, q, signs, R, n_R, scratch, (size_t)-1, num_splits, out);
+  if (st != OKQ_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cache->batch > MAX_ENTRIES) return OKQ_ERR_UNSUPPORTED;
+  const size_t q_stride = (size_t)cache->batch * cache->n_q_heads * D;
+  for (int l0 = 0; l0 < layer_count; l0 += layers_per_launch) {
+    const int lc = layer_count - l0 < layers_per_launch ? layer_count - l0 : layers_per_launch;
+    DecodeParams P = make_params(cache, layer + l0, lc, static_cast<const __half*>(q) + l0 * q_stride, sm_scale,
+                                 signs + (size_t)l0 * D, R + (size_t)l0 * n_R * 3 * D * D, n_R, out + l0 * q_stride);
+    P.partials_f = static_cast<PartialF*>(scratch);
+    st = launch_decode_mma(P, mma_ctas(cache, lc, num_splits), s, nullptr, nullptr);
     if (st != OKQ_OK) return st;
   }
   return launch_status();
