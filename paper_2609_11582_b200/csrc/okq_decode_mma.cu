@@ -321,11 +321,22 @@ __device__ __forceinline__ void value_warp(MmaSmem& sm, const Segment& sg, int p
           const uint32_t nA = 0x00020002u << (4 * kv), nB = 0x00080008u << (4 * kv);
           const uint32_t p0 = kv ? b0[2] : b0[0], p1 = kv ? b0[3] : b0[1];
           const uint32_t q0 = kv ? b1[2] : b1[0], q1 = kv ? b1[3] : b1[1];
+          // the two bit-plane products of one m-tile hit the same accumulator: keep them four
+          // MMAs apart so the second never waits for the first
 #pragma unroll
-          for (int mu = 0; mu < 8; mu++) {
-            const uint32_t w = vw[mu], w8 = w >> 8;
-            mma16816(acc[mu], w & mA, w8 & mA, w & mB, w8 & mB, p0, p1);
-            mma16816(acc[mu], w & nA, w8 & nA, w & nB, w8 & nB, q0, q1);
+          for (int mq = 0; mq < 8; mq += 4) {
+            uint32_t w8[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+              const uint32_t w = vw[mq + i];
+              w8[i] = w >> 8;
+              mma16816(acc[mq + i], w & mA, w8[i] & mA, w & mB, w8[i] & mB, p0, p1);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+              const uint32_t w = vw[mq + i];
+              mma16816(acc[mq + i], w & nA, w8[i] & nA, w & nB, w8[i] & nB, q0, q1);
+            }
           }
         }
       }
@@ -461,28 +472,46 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
   }
 }
 
-// grid (n_kv_heads, batch*layer_count), 128 threads: merge partials, add the raw tail,
-// apply R_m^T, normalise
-__global__ void __launch_bounds__(128) k_combine_mma(DecodeParams P, int n_cta) {
-  __shared__ float vec[3][GP][D];
-  __shared__ float tsc[W][GP];       // tail scores (log2 domain)
-  __shared__ float Ms[GP], Ls[GP];
-  __shared__ int prefix[MAX_ENTRIES + 1];
+constexpr int CB_SEQ = 4;                 // sequences per combine CTA (one 128-thread group each)
+constexpr int CB_ROWS = CB_SEQ * GP;      // (sequence, head) rows per combine CTA
+
+struct CombineSmem {
+  __align__(16) float Rm[D][D];  // one modality's rotation matrix, staged with cp.async
+  float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
+  float tsc[CB_SEQ][W][GP];     // tail scores (log2 domain)
+  float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
+  int prefix[MAX_ENTRIES + 1];
+};
+
+// grid (n_kv_heads, ceil(batch / CB_SEQ), layer_count), 4 x 128 threads (group = sequence,
+// thread = channel): merge the partials of each (sequence, head), add the raw tail tokens, apply
+// R_m^T (the four groups read the same matrix elements, so they come from L1 after the first
+// touch) and normalise.
+__global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, int n_cta) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  CombineSmem& sm = *reinterpret_cast<CombineSmem*>(smem_raw);
   const CacheView& cv = P.cv;
-  const int h = blockIdx.x, e = blockIdx.y, b = e % cv.batch, li = e / cv.batch, layer = P.layer0 + li;
-  const int c = threadIdx.x, G = P.group, Hkv = cv.n_kv_heads;
+  const int h = blockIdx.x, li = blockIdx.z, layer = P.layer0 + li;
+  const int bs = threadIdx.x >> 7, c = threadIdx.x & 127;
+  const int b = blockIdx.y * CB_SEQ + bs;
+  const bool live = b < cv.batch;
+  const int bb = live ? b : 0;
+  const int G = P.group, Hkv = cv.n_kv_heads;
   const int n_entries = P.layer_count * cv.batch;
-  const int total = block_prefix(cv, P.layer0, n_entries, prefix);
+  const int total = block_prefix(cv, P.layer0, n_entries, sm.prefix);
   const int per = total > 0 ? (total + n_cta - 1) / n_cta : 1;
-  const int seq = cv.seq_len[layer * cv.batch + b];
+  constexpr float ACC_SCALE = (CB_OUTER - CB_INNER) * 262144.0f;  // (b - a) * 2^18
+  constexpr float LOG2E = 1.4426950408889634f;
+
+  const int e = li * cv.batch + bb;
+  const int seq = live ? cv.seq_len[layer * cv.batch + bb] : 0;
   const int nwin = seq / W, n_tail = seq - nwin * W;
   const int unit = e * Hkv + h;
-  const int start = prefix[e] + h * nwin, end = start + nwin;
+  const int start = sm.prefix[e] + h * nwin, end = start + nwin;
   const int cta_lo = nwin > 0 ? start / per : 0, cta_hi = nwin > 0 ? (end - 1) / per : -1;
-  const __half* qbase = P.q + (((size_t)li * cv.batch + b) * cv.n_q_heads + h * G) * D;
-  const __half* kt = cv.k_tail + cv.tail_off(layer, b, h);
-  const __half* vt = cv.v_tail + cv.tail_off(layer, b, h);
-
+  const __half* qbase = P.q + (((size_t)li * cv.batch + bb) * cv.n_q_heads + h * G) * D;
+  const __half* kt = cv.k_tail + cv.tail_off(layer, bb, h);
+  const __half* vt = cv.v_tail + cv.tail_off(layer, bb, h);
   // tail scores: thread -> (token = c & 31, heads (c >> 5) * 2 + {0, 1})
   {
     const int tok = c & 31;
@@ -492,73 +521,101 @@ __global__ void __launch_bounds__(128) k_combine_mma(DecodeParams P, int n_cta) 
       float s = -INFINITY;
       if (tok < n_tail && j < G) {
         float a = 0.f;
-        for (int k = 0; k < D; k += 2) {
-          float2 qv = __half22float2(*reinterpret_cast<const __half2*>(qbase + j * D + k));
-          float2 kv = __half22float2(*reinterpret_cast<const __half2*>(kt + tok * D + k));
-          a = fmaf(qv.x, kv.x, a);
-          a = fmaf(qv.y, kv.y, a);
+        for (int k = 0; k < D; k += 8) {
+          const uint4 qv = *reinterpret_cast<const uint4*>(qbase + j * D + k);
+          const uint4 kv = *reinterpret_cast<const uint4*>(kt + tok * D + k);
+          const __half2* q2 = reinterpret_cast<const __half2*>(&qv);
+          const __half2* k2 = reinterpret_cast<const __half2*>(&kv);
+#pragma unroll
+          for (int u = 0; u < 4; u++) {
+            const float2 qf = __half22float2(q2[u]), kf = __half22float2(k2[u]);
+            a = fmaf(qf.x, kf.x, a);
+            a = fmaf(qf.y, kf.y, a);
+          }
         }
-        s = a * P.sm_scale * 1.4426950408889634f;
+        s = a * P.sm_scale * LOG2E;
       }
-      tsc[tok][j] = s;
+      sm.tsc[bs][tok][j] = s;
     }
   }
   __syncthreads();
   if (c < GP) {
     float M = -INFINITY;
     for (int ct = cta_lo; ct <= cta_hi; ct++) M = fmaxf(M, P.partials_f[(size_t)unit + ct].m[c]);
-    for (int i = 0; i < n_tail; i++) M = fmaxf(M, tsc[i][c]);
+    for (int i = 0; i < n_tail; i++) M = fmaxf(M, sm.tsc[bs][i][c]);
     float L = 0.f;
     for (int ct = cta_lo; ct <= cta_hi; ct++) {
       const PartialF& pp = P.partials_f[(size_t)unit + ct];
       if (pp.m[c] != -INFINITY) L += pp.l[c] * exp2f(pp.m[c] - M);
     }
-    for (int i = 0; i < n_tail; i++) L += exp2f(tsc[i][c] - M);
-    Ms[c] = M;
-    Ls[c] = L;
+    for (int i = 0; i < n_tail; i++) L += exp2f(sm.tsc[bs][i][c] - M);
+    sm.Ms[bs][c] = M;
+    sm.Ls[bs][c] = L;
   }
   __syncthreads();
-  constexpr float ACC_SCALE = (CB_OUTER - CB_INNER) * 262144.0f;  // (b - a) * 2^18
   float raw[GP];
 #pragma unroll
   for (int j = 0; j < GP; j++) {
-    raw[j] = 0.f;
-    if (j >= G) continue;
-    const float M = Ms[j];
-    float v[3] = {0.f, 0.f, 0.f};
-    const int r = 4 * (c >> 4) + 2 * ((c >> 3) & 1) + (j & 1), l32 = 4 * (c & 7) + (j >> 1);
-    for (int ct = cta_lo; ct <= cta_hi; ct++) {
-      const PartialF& pp = P.partials_f[(size_t)unit + ct];
-      if (pp.m[j] == -INFINITY) continue;
-      const float ef = exp2f(pp.m[j] - M);
+    float v[3] = {0.f, 0.f, 0.f}, a = 0.f;
+    if (j < G) {
+      const float M = sm.Ms[bs][j];
+      const int r = 4 * (c >> 4) + 2 * ((c >> 3) & 1) + (j & 1), l32 = 4 * (c & 7) + (j >> 1);
+      for (int ct = cta_lo; ct <= cta_hi; ct++) {
+        const PartialF& pp = P.partials_f[(size_t)unit + ct];
+        if (pp.m[j] == -INFINITY) continue;
+        const float ef = exp2f(pp.m[j] - M);
 #pragma unroll
-      for (int m = 0; m < 3; m++) {
-        // weight sum of head j: the four lanes of quad j hold partial sums
-        const float S = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
-        v[m] = fmaf(fmaf(ACC_SCALE, pp.frag[m][r][l32], -CB_OUTER * S), ef, v[m]);
+        for (int m = 0; m < 3; m++) {
+          // weight sum of head j: the four lanes of quad j hold partial sums
+          const float S = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
+          v[m] = fmaf(fmaf(ACC_SCALE, pp.frag[m][r][l32], -CB_OUTER * S), ef, v[m]);
+        }
       }
+      for (int i = 0; i < n_tail; i++) a = fmaf(exp2f(sm.tsc[bs][i][j] - M), __half2float(vt[i * D + c]), a);
     }
-    vec[0][j][c] = v[0]; vec[1][j][c] = v[1]; vec[2][j][c] = v[2];
-    float a = 0.f;
-    for (int i = 0; i < n_tail; i++) a = fmaf(exp2f(tsc[i][j] - M), __half2float(vt[i * D + c]), a);
+    sm.vec[0][bs * GP + j][c] = v[0];
+    sm.vec[1][bs * GP + j][c] = v[1];
+    sm.vec[2][bs * GP + j][c] = v[2];
     raw[j] = a;
   }
   __syncthreads();
+
+  // out[row][c] = sum_m sum_r R_m[r][c] * vec[m][row][r] for this group's GP rows; each matrix
+  // is staged in shared memory once per CTA
   float o[GP];
 #pragma unroll
   for (int j = 0; j < GP; j++) o[j] = 0.f;
   const float* Rset = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D;
-  for (int m = 0; m < 3; m++)
-    for (int r = 0; r < D; r++) {
-      const float rv = __ldg(Rset + ((size_t)m * D + r) * D + c);
-#pragma unroll
-      for (int j = 0; j < GP; j++) o[j] = fmaf(rv, vec[m][j][r], o[j]);
+  for (int m = 0; m < 3; m++) {
+    __syncthreads();   // everyone is done with the previous matrix
+    {
+      const float* src = Rset + (size_t)m * D * D;
+      float* dst = &sm.Rm[0][0];
+      for (int i = threadIdx.x; i < D * D / 4; i += CB_SEQ * 128) cp_async16(dst + 4 * i, src + 4 * i);
+      cp_async_commit();
+      cp_async_wait<0>();
     }
+    __syncthreads();
+#pragma unroll 2
+    for (int r = 0; r < D; r += 4) {
+      const float r0 = sm.Rm[r][c], r1 = sm.Rm[r + 1][c], r2 = sm.Rm[r + 2][c], r3 = sm.Rm[r + 3][c];
 #pragma unroll
-  for (int j = 0; j < GP; j++) {
-    if (j >= G) continue;
-    const float L = Ls[j];
-    P.out[(((size_t)li * cv.batch + b) * cv.n_q_heads + h * G + j) * D + c] = L > 0.f ? (o[j] + raw[j]) / L : 0.f;
+      for (int j = 0; j < GP; j++) {
+        const float4 x = *reinterpret_cast<const float4*>(&sm.vec[m][bs * GP + j][r]);
+        o[j] = fmaf(r0, x.x, o[j]);
+        o[j] = fmaf(r1, x.y, o[j]);
+        o[j] = fmaf(r2, x.z, o[j]);
+        o[j] = fmaf(r3, x.w, o[j]);
+      }
+    }
+  }
+  if (live) {
+#pragma unroll
+    for (int j = 0; j < GP; j++) {
+      if (j >= G) continue;
+      const float L = sm.Ls[bs][j];
+      P.out[(((size_t)li * cv.batch + b) * cv.n_q_heads + h * G + j) * D + c] = L > 0.f ? (o[j] + raw[j]) / L : 0.f;
+    }
   }
 }
 
@@ -566,13 +623,16 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
   static thread_local bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(k_decode_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MmaSmem));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_combine_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem));
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
     attr_set = true;
   }
   if (before) cudaEventRecord(before, s);
   k_decode_mma<<<n_cta, NTHREADS, sizeof(MmaSmem), s>>>(P);
   if (after) cudaEventRecord(after, s);
-  k_combine_mma<<<dim3(P.cv.n_kv_heads, P.cv.batch * P.layer_count), 128, 0, s>>>(P, n_cta);
+  k_combine_mma<<<dim3(P.cv.n_kv_heads, (P.cv.batch + CB_SEQ - 1) / CB_SEQ, P.layer_count), CB_SEQ * 128,
+                  sizeof(CombineSmem), s>>>(P, n_cta);
   return OKQ_OK;
 }
 
