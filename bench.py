@@ -33,9 +33,10 @@ from paper_2609_11582_b200 import workloads as WL  # noqa: E402
 
 METRIC = "2-bit KV decode-attention effective HBM GB/s (packed-KV bytes per decode step / step time)"
 BYTES_PER_TOKEN_HEAD = 84          # 32 B key codes + 2 B key norm + 16 B (m, s) + 32 B value codes + 2 B value norm
-# dram__bytes_read.sum + dram__bytes_write.sum of one split-K decode launch, measured with ncu
-# on a smaller case and scaled per token-head (see profiles/); None until measured.
-NCU_DRAM_BYTES_PER_TOKEN_HEAD = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one split-K decode launch, measured with ncu on a
+# 4-layer slice of the workload (176 MB of records, larger than L2) and divided by its token-heads;
+# traffic grows in proportion to the token-heads (profiles/decode_mma_layers4_ncu_full.md).
+NCU_DRAM_BYTES_PER_TOKEN_HEAD = 86.99
 
 
 def measured_peaks():

@@ -1,0 +1,103 @@
+"""GPU parity on the benchmark's other shapes and at the full size the benchmark times.
+
+  * 30B-A3B shape (GQA group 8, video 400 / audio 100 chunks), reduced layers and context;
+  * long-context decode (batch 1, many CTAs per (sequence, head));
+  * the full 7B decode step (28 layers x batch 8 x 16384 tokens, one append + one decode call
+    over all layers, inputs drawn on the GPU exactly as bench.py does), checked on sampled
+    (layer, sequence) pairs the oracle can afford, plus properties that hold at any size.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import okq_oracle as O
+from paper_2609_11582_b200 import binding as B
+from paper_2609_11582_b200 import workloads as WL
+from tests import harness as Hn
+
+pytestmark = pytest.mark.gpu
+D, W = 128, 32
+
+
+def test_group8_30b_shape():
+    w = WL.scaled(WL.WORKLOADS["step30b"], n_layers=2, batch=2, n_tokens=4096 + 7)
+    c = Hn.Case(w)
+    for l in range(2):
+        kq, vq, _, _ = c.oracle_quantize(l)
+        Hn.compare_cache(c, l, c.gpu_export(l), kq, vq)
+    got = c.gpu_decode(0, layer_count=2)
+    for l in range(2):
+        ref, _ = c.oracle_attention(l)
+        print("30B shape layer", l, Hn.assert_attention_close(got[l], ref))
+    simt = c.gpu_decode(0, layer_count=2, simt=True)
+    assert np.abs(simt - got).max() < 1e-3
+
+
+def test_long_context_batch1():
+    w = WL.scaled(WL.WORKLOADS["long7b"], n_layers=1, n_tokens=32768 + 31)
+    c = Hn.Case(w)
+    ref, _ = c.oracle_attention(0)
+    got = c.gpu_decode(0)[0]                 # 148 CTAs over 4 (sequence, head) units: 37 partials each
+    print("long context", Hn.assert_attention_close(got, ref))
+    got4 = c.gpu_decode(0, num_splits=3)[0]
+    Hn.assert_attention_close(got4, ref)
+
+
+def test_full_7b_step_sampled():
+    w = WL.WORKLOADS["step7b"]
+    dev = torch.device("cuda")
+    L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
+    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev)
+    mod_cpu = WL.modality_layout(w)
+    mod = mod_cpu.unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
+    signs = torch.stack([WL.gen_signs(w, l) for l in range(L)])
+    R = torch.stack([WL.gen_rotations(w, l) for l in range(L)])
+    d_signs, d_R = signs.to(dev), R.unsqueeze(1).contiguous().to(dev)
+    samples = [(0, 0), (13, 5), (27, 7)]
+    kept = {}
+    for l in range(L):
+        k, v = WL.gen_kv(w, l, device=dev)
+        B.quantize_keys(cache, l, k, d_signs[l])
+        B.quantize_values(cache, l, v, mod, d_R[l])
+        for (sl, sb) in samples:
+            if sl == l:
+                kept[(sl, sb)] = (k[sb].cpu(), v[sb].cpu())
+        del k, v
+    q = torch.stack([WL.gen_queries(w, l) for l in range(L)])
+    d_q = q.to(dev)
+    k_new, v_new, m_new = WL.gen_new_token(w, 0, 0, device=dev)
+    kn = k_new.unsqueeze(0).expand(L, -1, -1, -1).contiguous()
+    vn = v_new.unsqueeze(0).expand(L, -1, -1, -1).contiguous()
+    B.append(cache, 0, L, kn, vn, m_new, d_signs, d_R)
+    ws = torch.empty(B.decode_workspace_bytes(cache, L, 0), dtype=torch.uint8, device=dev)
+    out = torch.full((L, Bn, Hq, D), float("nan"), dtype=torch.float32, device=dev)
+    B.decode_attention(cache, 0, L, d_q, d_signs, d_R, ws, out)
+    torch.cuda.synchronize()
+    assert cache.device_status() == 0
+    assert (cache.seq_len == N + 1).all()
+    o = out.cpu().numpy().astype(np.float64)
+    # properties at any size: finite, and an attention output is a convex combination of value
+    # vectors, so its norm cannot exceed the largest value norm (reconstruction adds at most ~35 %)
+    assert np.isfinite(o).all()
+    assert np.linalg.norm(o, axis=-1).max() < 6.0
+    # sampled (layer, sequence) pairs against the oracle: packed cache bit for bit, attention within tolerance
+    for (sl, sb) in samples:
+        kc, vc = kept[(sl, sb)]
+        kb = Hn.u16(kc).reshape(H, N, D); vb = Hn.u16(vc).reshape(H, N, D)
+        kq, vq, _ = O.quantize_batch(kb, vb, mod_cpu.numpy(), signs[sl].numpy(), R[sl].numpy())
+        e = B.cache_export(cache, sl)
+        torch.cuda.synchronize()
+        cap = cache.capacity
+        assert (e["k_codes"][sb].cpu().numpy()[:, :N] == kq["codes"]).all()
+        assert (Hn.u16(e["k_norm"][sb])[:, :N] == kq["norm"]).all()
+        assert (Hn.u16(e["k_meta"][sb])[:, :N // W] == kq["meta"]).all()
+        assert (e["v_codes"][sb].cpu().numpy()[:, :N] == vq["codes"]).all()
+        assert (Hn.u16(e["v_norm"][sb])[:, :N] == vq["norm"]).all()
+        del e
+        qs = Hn.u16(q[sl, sb]).reshape(H, w.group, D)
+        kt = np.broadcast_to(Hn.u16(k_new[sb].cpu())[:, None, :], (H, 1, D))
+        vt = np.broadcast_to(Hn.u16(v_new[sb].cpu())[:, None, :], (H, 1, D))
+        modrow = np.concatenate([mod_cpu.numpy(), np.zeros(1, np.uint8)])
+        ref, _ = O.attention(1, qs, kq, vq, modrow, kt, vt, signs[sl].numpy(), R[sl].numpy())
+        errs = Hn.assert_attention_close(o[sl, sb], ref.reshape(Hq, D))
+        print(f"full step7b layer {sl} seq {sb}: rel-L2 {errs[0]:.2e} worst head {errs[1]:.2e} max-abs {errs[2]:.2e}")
