@@ -192,7 +192,7 @@ def main():
     for l in range(L):
         k, v = WL.gen_kv(w, l, device=dev)
         B.quantize_keys(cache, l, k, signs[l])
-        B.quantize_values(cache, l, v, mod, R[l])
+        B.quantize_values(cache, l, v, mod, R[l], bulk=True)   # prefill path: rotation on the tensor cores
         del k, v
     torch.cuda.synchronize()
     seq0 = cache.seq_len.clone()

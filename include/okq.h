@@ -121,6 +121,21 @@ okq_status okq_quantize_values(const okq_cache* cache, int32_t layer, const void
                                const float* R, int32_t n_R, void* stream);
 
 /*
+ * Bulk (prefill) form of okq_quantize_values with the rotation z = R_m v on the tensor cores
+ * (Eq. 6 as a dense [tokens x 128] x [128 x 128] product per modality; tcgen05.mma with R split
+ * into two fp16 matrices and fp32 accumulation in tensor memory).  Same arguments, same stored
+ * norms (bit-identical).  A code can differ from okq_quantize_values, by one level, only where
+ * the rotated coordinate lies within about 1e-7 of a codebook threshold: both results are valid
+ * nearest-level choices at fp32 accuracy.  If the tensor-core pipeline does not answer within a
+ * bounded wait the device status word becomes OKQ_ERR_TIMEOUT and the remaining tiles are
+ * skipped.
+ */
+okq_status okq_quantize_values_bulk(const okq_cache* cache, int32_t layer, const void* v_fp16,
+                                    const int64_t strides[3], int32_t n_tokens,
+                                    const uint8_t* modality, const float* R, int32_t n_R,
+                                    void* stream);
+
+/*
  * Streaming append (the paper's protocol keeps recent tokens in fp16 before they are
  * quantised): add one token per sequence to layers [layer, layer+layer_count).  The token
  * goes raw into the tail; when the tail reaches 32 tokens they are quantised as one window

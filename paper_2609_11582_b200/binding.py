@@ -58,6 +58,8 @@ def lib():
         L.okq_quantize_values.restype = C.c_int
         L.okq_quantize_values.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_void_p, C.POINTER(C.c_int64), C.c_int32,
                                           C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.okq_quantize_values_bulk.restype = C.c_int
+        L.okq_quantize_values_bulk.argtypes = L.okq_quantize_values.argtypes
         L.okq_append.restype = C.c_int
         L.okq_append.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
@@ -84,7 +86,7 @@ def exported_symbols():
     return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
             "okq_cache_import", "okq_profile_events", "okq_decode_attention_simt",
-            "okq_decode_attention_noalloc"]
+            "okq_decode_attention_noalloc", "okq_quantize_values_bulk"]
 
 
 def _ptr(t) -> int:
@@ -148,15 +150,17 @@ def quantize_keys(cache: Cache, layer: int, k: torch.Tensor, signs: torch.Tensor
 
 
 def quantize_values(cache: Cache, layer: int, v: torch.Tensor, modality: torch.Tensor, R: torch.Tensor,
-                    n_tokens=None, stream=None):
-    """v: fp16 [batch, n_kv_heads, n, 128]; modality: uint8 [batch, n]; R: float32 [n_R, 3, 128, 128]."""
+                    n_tokens=None, stream=None, bulk=False):
+    """v: fp16 [batch, n_kv_heads, n, 128]; modality: uint8 [batch, n]; R: float32 [n_R, 3, 128, 128].
+    bulk=True calls okq_quantize_values_bulk (tensor-core rotation)."""
     assert v.dtype == torch.float16 and v.stride(3) == 1 and modality.dtype == torch.uint8 and modality.is_contiguous()
     n = v.shape[2] if n_tokens is None else n_tokens
     assert modality.shape[-1] == n
     strides = (C.c_int64 * 3)(v.stride(0), v.stride(1), v.stride(2))
     n_R = R.shape[0] if R.dim() == 4 else 1
-    _check(lib().okq_quantize_values(C.byref(cache.c), layer, _ptr(v), strides, n, _ptr(modality), _ptr(R), n_R,
-                                     _stream(stream)), "okq_quantize_values")
+    fn = lib().okq_quantize_values_bulk if bulk else lib().okq_quantize_values
+    _check(fn(C.byref(cache.c), layer, _ptr(v), strides, n, _ptr(modality), _ptr(R), n_R, _stream(stream)),
+           "okq_quantize_values_bulk" if bulk else "okq_quantize_values")
 
 
 def append(cache: Cache, layer: int, layer_count: int, k_new, v_new, modality_new, signs, R, n_R=1, stream=None):

@@ -9,6 +9,7 @@
 namespace okq {
 
 void set_last_cuda_error(int e);
+int sm_count();   // SMs of the current device (cached per thread)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -384,19 +384,6 @@ static int auto_splits(const okq_cache* c, int layer_count) {
   return (int)want;
 }
 
-static int sm_count() {
-  static thread_local int cached_dev = -1, cached = 0;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-  if (dev != cached_dev) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    cached = n;
-    cached_dev = dev;
-  }
-  return cached;
-}
-
 // persistent grid of the tensor-core kernel
 static int mma_ctas(const okq_cache* c, int layer_count, int num_splits) {
   if (num_splits <= 0) return sm_count();

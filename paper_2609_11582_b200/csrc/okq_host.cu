@@ -6,6 +6,19 @@ namespace okq {
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 
+int sm_count() {
+  static thread_local int cached_dev = -1, cached = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev != cached_dev) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached = n;
+    cached_dev = dev;
+  }
+  return cached;
+}
+
 okq_status check_cache(const okq_cache* c, bool need_ptrs) {
   if (!c) return OKQ_ERR_INVALID_ARG;
   if (c->head_dim != OKQ_HEAD_DIM || c->window != OKQ_WINDOW) return OKQ_ERR_UNSUPPORTED;

@@ -350,6 +350,10 @@ __global__ void k_import(CacheView cv, int layer, const unsigned char* k_codes, 
   }
 }
 
+okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __half* v, const int64_t strides[3],
+                                     const unsigned char* modality, int n_tokens, const float* R, int n_R,
+                                     int n_sm, cudaStream_t s);
+
 static okq_status check_bulk(const okq_cache* c, int32_t layer, const void* x, const int64_t strides[3],
                              int32_t n_tokens) {
   okq_status st = check_cache(c, true);
@@ -403,6 +407,24 @@ okq_status okq_quantize_values(const okq_cache* cache, int32_t layer, const void
     k_quantize_values<<<grid, 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2], modality, n_tokens, R,
                                            n_R);
   }
+  k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
+                                                           n_tokens, cv.v_tail, n_tokens > 0 ? modality : nullptr);
+  return launch_status();
+}
+
+okq_status okq_quantize_values_bulk(const okq_cache* cache, int32_t layer, const void* v_fp16,
+                                    const int64_t strides[3], int32_t n_tokens, const uint8_t* modality,
+                                    const float* R, int32_t n_R, void* stream) {
+  okq_status st = check_bulk(cache, layer, v_fp16, strides, n_tokens);
+  if (st != OKQ_OK) return st;
+  if ((!modality && n_tokens > 0) || !R) return OKQ_ERR_INVALID_ARG;
+  if (n_R != 1 && n_R != cache->n_kv_heads) return OKQ_ERR_INVALID_ARG;
+  if (!aligned16(R)) return OKQ_ERR_ALIGNMENT;
+  CacheView cv = make_view(cache);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const __half* v = static_cast<const __half*>(v_fp16);
+  st = launch_quantize_values_tc(cv, layer, v, strides, modality, n_tokens, R, n_R, sm_count(), s);
+  if (st != OKQ_OK) return st;
   k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
                                                            n_tokens, cv.v_tail, n_tokens > 0 ? modality : nullptr);
   return launch_status();

@@ -176,3 +176,55 @@ def test_per_head_rotations():
     q = Hn.u16(c.q[0]).reshape(U, w.group, D)
     ref, _ = O.attention(1, q, kq, vq, c.mod_b.numpy(), kb[:, 256:], vb[:, 256:], signs, Rh.numpy(), unit_rot=np.arange(U))
     Hn.assert_attention_close(got, ref.reshape(1, w.n_q_heads, D))
+
+
+def _check_bulk_codes(c, layer, R_host):
+    """Codes of the tensor-core value quantiser against the oracle: identical except, at most, where the
+    oracle's rotated coordinate lies within 2^-20 of a codebook threshold (then they differ by one level)."""
+    kq, vq, _, vb = c.oracle_quantize(layer)
+    e = {k: v.cpu() for k, v in c.gpu_export(layer).items()}
+    U = c.w.batch * c.w.n_kv_heads
+    cap, npk = c.cache.capacity, (c.n // W) * W
+    assert (Hn.u16(e["v_norm"]).reshape(U, cap)[:, :npk] == vq["norm"]).all(), "value norms must be bit-identical"
+    got = O.unpack_codes(e["v_codes"].numpy().reshape(U, cap, 32)[:, :npk])
+    ref = O.unpack_codes(vq["codes"])
+    bad = np.argwhere(got != ref)
+    _, T = O.codebook()
+    thr = np.array([-T, 0.0, T], dtype=np.float64)
+    unit_seq = np.repeat(np.arange(c.w.batch), c.w.n_kv_heads)
+    for (u, i, ch) in bad:
+        m = c.mod_b.numpy()[unit_seq[u], i]
+        _, z = O.value_rotate(vb[u, i], R_host[m])
+        assert abs(int(got[u, i, ch]) - int(ref[u, i, ch])) == 1
+        assert np.abs(float(z[ch]) - thr).min() <= 2.0 ** -20, (u, i, ch, z[ch])
+    return len(bad), ref.size
+
+
+def test_bulk_value_quantiser_on_tensor_cores():
+    # several 128-token tiles, mixed-modality tiles, a partial last tile (2048 + 64 + 19 tokens)
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=2)
+    c = Hn.Case(w, n_tokens=2048 + 64 + 19)
+    dev = c.cache.device
+    B.quantize_values(c.cache, 0, c.v[0].to(dev), c.d_mod, c.d_R[0], bulk=True)
+    torch.cuda.synchronize()
+    assert c.cache.device_status() == 0
+    n_bad, n_all = _check_bulk_codes(c, 0, c.R[0].numpy())
+    print(f"tensor-core value codes: {n_bad} of {n_all} differ from the exact chain (all within 2^-20 of a threshold)")
+    assert n_bad <= n_all * 2e-4
+    # decode over the bulk-built cache still matches the oracle within tolerance
+    ref, _ = c.oracle_attention(0)
+    Hn.assert_attention_close(c.gpu_decode(0)[0], ref)
+    # raw tail and modality as in the exact path
+    U = w.batch * w.n_kv_heads
+    assert (Hn.u16(c.cache.v_tail).reshape(U, W, D)[:, :19] == Hn.u16(c.v[0]).reshape(U, c.n, D)[:, 2048 + 64:]).all()
+    # a signed permutation is rotated exactly by any arithmetic: codes must then be identical
+    rng = np.random.default_rng(5)
+    P = np.zeros((3, D, D), np.float32)
+    for m in range(3):
+        P[m, np.arange(D), rng.permutation(D)] = np.where(rng.random(D) < 0.5, -1.0, 1.0)
+    c.R[0] = torch.from_numpy(P)
+    dP = torch.from_numpy(P)[None].contiguous().to(dev)
+    B.quantize_values(c.cache, 0, c.v[0].to(dev), c.d_mod, dP, bulk=True)
+    torch.cuda.synchronize()
+    n_bad, _ = _check_bulk_codes(c, 0, P)
+    assert n_bad == 0
