@@ -158,17 +158,65 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_prefill(args, w, B, dev, rank):
+    """Secondary measurement: bulk okq_quantize_keys + okq_quantize_values_bulk over a fresh fp16 K/V cache of
+    every layer (the prefill half of the long-context configuration).  One JSON line."""
+    L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
+    cache = B.Cache(L, Bn, H, Hq, N, device=dev)
+    mod = WL.modality_layout(w).unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
+    signs = torch.stack([WL.gen_signs(w, l) for l in range(L)]).to(dev)
+    R = torch.stack([WL.gen_rotations(w, l) for l in range(L)]).unsqueeze(1).contiguous().to(dev)
+    kv = [WL.gen_kv(w, l, device=dev) for l in range(L)]
+    th = L * Bn * H * N
+    in_bytes, out_bytes = th * 512, th * BYTES_PER_TOKEN_HEAD
+
+    def timed(fn):
+        for _ in range(args.warmup):
+            fn()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in ev:
+            a.record(); fn(); b.record()
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in ev) / args.steps
+
+    ms_k = timed(lambda: [B.quantize_keys(cache, l, kv[l][0], signs[l]) for l in range(L)])
+    ms_v = timed(lambda: [B.quantize_values(cache, l, kv[l][1], mod, R[l], bulk=True) for l in range(L)])
+    ms_vx = timed(lambda: [B.quantize_values(cache, l, kv[l][1], mod, R[l]) for l in range(min(L, 2))]) * L / min(L, 2)
+    if cache.device_status() != 0:
+        raise RuntimeError("device status word set during the benchmark")
+    peak, peak_kind = measured_peaks()
+    ms = ms_k + ms_v
+    line = {"metric": "prefill quantisation: fp16 K/V bytes in + packed bytes out per second", "phase": "prefill",
+            "value": (in_bytes + out_bytes) / (ms * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "dtype": "f32/f16-mma", "data": "synthetic",
+            "config": {"workload": w.name, "n_layers": L, "batch": Bn, "n_kv_heads": H, "context": N},
+            "keys_ms": ms_k, "values_bulk_ms": ms_v, "values_exact_ms_scaled": ms_vx,
+            "keys_gbs": th * 306 / (ms_k * 1e-3) / 1e9, "values_bulk_gbs": th * 290 / (ms_v * 1e-3) / 1e9,
+            "values_bulk_tflops": th * 2 * 2 * 128 * 128 / (ms_v * 1e-3) / 1e12,
+            "roofline": {"bound": "hbm", "kernel": "key + value quantisers", "achieved": (in_bytes + out_bytes) / (ms * 1e-3) / 1e9,
+                         "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                         "frac": (in_bytes + out_bytes) / (ms * 1e-3) / 1e9 / peak, "traffic": None}}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=32)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="okq", choices=["okq", "reference"])
-    ap.add_argument("--workload", default="step7b", choices=sorted(WL.WORKLOADS))
+    ap.add_argument("--workload", default=None, choices=sorted(WL.WORKLOADS))
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling on a small case)")
+    ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
+                    help="decode: the headline decode step; prefill: bulk quantisation of a fresh fp16 K/V cache "
+                         "(secondary measurement, default workload prefill7b)")
     args = ap.parse_args()
+    if args.workload is None:
+        args.workload = "prefill7b" if args.phase == "prefill" else "step7b"
     w = WL.WORKLOADS[args.workload]
     if args.layers > 0:
         w = WL.scaled(w, n_layers=args.layers, name=f"{w.name}[layers={args.layers}]")
@@ -182,6 +230,9 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+
+    if args.phase == "prefill":
+        return run_prefill(args, w, B, dev, rank)
 
     # ---- build the packed cache on the device (setup, untimed)
     L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
