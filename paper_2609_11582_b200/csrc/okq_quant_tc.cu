@@ -26,16 +26,16 @@ namespace okq {
 namespace {
 
 constexpr int TILE = 128;               // tokens per tile
-constexpr int NT = 512;                 // threads per CTA: 16 warps, four per tensor-memory lane quarter
-constexpr int CSTRIDE = 132;            // row stride of the code-byte buffer (bank-conflict padding)
+constexpr int NT = 512;                 // worker threads per CTA: 16 warps, four per tensor-memory lane quarter
+constexpr int NT_ALL = NT + 32;         // plus one warp that only issues the MMAs
 constexpr int TILE_BYTES = TILE * D * 2;  // 32 KB: one fp16 operand tile
 
 struct TcSmem {
-  __align__(1024) unsigned char a[2][TILE_BYTES];   // value tiles (double buffered)
+  __align__(1024) unsigned char a[2][TILE_BYTES];      // value tiles (double buffered)
   __align__(1024) unsigned char b[2][2][TILE_BYTES];   // two resident matrices, each as R_hi, R_lo
-  unsigned char code[TILE * CSTRIDE];
-  float inv[TILE];
-  unsigned char mod[TILE];
+  uint32_t cw[2][TILE][8];                             // codes of a tile: per token, 16 channels x 2 bits per word
+  float inv[2][TILE];
+  __align__(4) unsigned char mod[2][TILE];
   __align__(8) unsigned long long mbar;
   uint32_t tmem_slot;
 };
@@ -58,12 +58,13 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_u32(smem)), "l"(gmem));
 }
 
-// bounded wait for one phase of the MMA-completion barrier
+// bounded wait for one phase of the MMA-completion barrier; each try lets the hardware suspend the
+// thread for up to about a millisecond, so a completed MMA is normally seen by the first try
 __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity) {
-  for (int it = 0; it < 4000000; it++) {
+  for (int it = 0; it < 4000; it++) {
     uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-                 : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                 : "=r"(ok) : "r"(mbar), "r"(parity), "r"(1000000u) : "memory");
     if (ok) return true;
   }
   return false;
@@ -71,24 +72,32 @@ __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity) {
 
 }  // namespace
 
-// persistent grid, NT threads.  Tiles are numbered (b, h, tile-in-sequence), tile = 4 windows.
-__global__ void __launch_bounds__(NT, 1) k_quantize_values_tc(CacheView cv, int layer, const __half* __restrict__ v,
+// persistent grid, NT_ALL threads.  Tiles are numbered (b, h, tile-in-sequence), tile = 4 windows; a CTA
+// owns a contiguous range of them.  A "job" is
+// one (tile, modality present in the tile); the MMAs of job j run on the tensor cores while the
+// threads do the epilogue (and packing) of job j-1 out of the other half of tensor memory.
+__global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(CacheView cv, int layer, const __half* __restrict__ v,
                                                              long long sb, long long sh, long long st,
                                                              const unsigned char* __restrict__ modality, int n_tokens,
                                                              const float* __restrict__ R, int n_R) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   TcSmem& sm = *reinterpret_cast<TcSmem*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool worker = tid < NT;            // warp 16 only issues MMAs
   const int n_win = n_tokens / W;
   const int tiles_per_unit = (n_win + 3) / 4;
-  const int n_tiles = tiles_per_unit * cv.n_kv_heads * cv.batch;
+  const int n_tiles_all = tiles_per_unit * cv.n_kv_heads * cv.batch;
+  // contiguous tile range of this CTA
+  const int per_cta = (n_tiles_all + gridDim.x - 1) / gridDim.x;
+  const int tile_begin = min(n_tiles_all, (int)blockIdx.x * per_cta);
+  const int n_tiles = min(n_tiles_all, tile_begin + per_cta);   // end of the range
 
   if (tid == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(smem_u32(&sm.mbar)));
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 128;\n" ::"r"(smem_u32(&sm.tmem_slot)) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;\n" ::"r"(smem_u32(&sm.tmem_slot)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
@@ -100,7 +109,7 @@ __global__ void __launch_bounds__(NT, 1) k_quantize_values_tc(CacheView cv, int 
   uint32_t phase = 0;
   int slot_key[2] = {-1, -1};   // (rotation set * 3 + modality) held by each resident slot
   int last_slot = 0;
-  bool failed = false;   // uniform across the block
+  bool failed = false;          // uniform across the block
 
   auto tile_coords = [&](int tile, int& b, int& h, int& win0) {
     b = tile / (tiles_per_unit * cv.n_kv_heads);
@@ -108,89 +117,116 @@ __global__ void __launch_bounds__(NT, 1) k_quantize_values_tc(CacheView cv, int 
     h = rem / tiles_per_unit;
     win0 = (rem - h * tiles_per_unit) * 4;
   };
-  auto issue_tile = [&](int tile, int buf) {
-    if (tile < n_tiles) {
-      int b, h, win0;
-      tile_coords(tile, b, h, win0);
+  auto issue_tile = [&](int tile, int buf, int b, int h, int win0) {
+    if (tile < n_tiles && worker) {
       const int rows = min(TILE, (n_win - win0) * W);
       const __half* src = v + b * sb + h * sh + (long long)win0 * W * st;
+      // a warp copies 8 rows x 4 chunks: 64 contiguous bytes per row on the global side, and one
+      // 128-byte core matrix per chunk on the shared side (at most 4-way bank conflicts)
       for (int idx = tid; idx < TILE * 16; idx += NT) {
-        const int r = idx >> 4, kc = idx & 15;
+        const int r = (idx & 7) + 8 * ((idx >> 5) & 15), kc = ((idx >> 3) & 3) + 4 * (idx >> 9);
         if (r < rows) cp_async16(sm.a[buf] + tile_off(r, kc * 8), src + (long long)r * st + kc * 8);
       }
     }
     asm volatile("cp.async.commit_group;\n" ::);
   };
 
-  int it = 0;
-  issue_tile(blockIdx.x, 0);
-  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, it++) {
-    const int buf = it & 1;
-    issue_tile(tile + gridDim.x, buf ^ 1);       // prefetch the next tile
-    int b, h, win0;
-    tile_coords(tile, b, h, win0);
-    const int wins = min(4, n_win - win0), rows = wins * W;
-
-    // modality of each token of the tile (ids > 2 count as text)
-    if (tid < TILE) {
-      unsigned char m = 255;
-      if (tid < rows) {
-        m = modality[(size_t)b * n_tokens + (size_t)win0 * W + tid];
-        m = m > 2 ? 0 : m;
-      }
-      sm.mod[tid] = m;
+  // the tile being prefetched: coordinates and this thread's modality byte
+  int nb = 0, nh = 0, nwin0 = 0;
+  unsigned char next_mod = 0;
+  auto fetch_next_mod = [&](int tile) {
+    if (tile < n_tiles && tid < TILE) {
+      const int nrows = min(TILE, (n_win - nwin0) * W);
+      unsigned char m = 0;
+      if (tid < nrows) m = modality[(size_t)nb * n_tokens + (size_t)nwin0 * W + tid];
+      next_mod = m > 2 ? 0 : m;
     }
-    asm volatile("cp.async.wait_group 1;\n" ::: "memory");   // this tile has landed (the prefetch may be in flight)
-    __syncthreads();
-    // norms with the exact adjacent-pair summation tree, four threads per token, read from the staged
-    // tile: a 16-byte chunk (8 channels) is three levels of the tree, a thread's four chunks two more,
-    // the four threads of a token the last two (shuffles between neighbouring lanes)
-    {
-      const int r = tid >> 2, q = tid & 3;
-      float part[4];
+  };
+  if (tile_begin < n_tiles) tile_coords(tile_begin, nb, nh, nwin0);
+  fetch_next_mod(tile_begin);
+  issue_tile(tile_begin, 0, nb, nh, nwin0);
+
+  int tile = tile_begin, buf = 1;       // buf flips when a tile is set up
+  int b = 0, h = 0, win0 = 0, wins = 0;
+  unsigned pend = 0;                    // modalities of the current tile not yet issued
+  int jobs = 0;
+  // the previous job, whose accumulator is waiting for its epilogue
+  bool p_valid = false, p_last = false;
+  int p_buf = 0, p_mod = 0, p_acc = 0, p_b = 0, p_h = 0, p_win0 = 0, p_wins = 0;
+
+  while (true) {
+    // ---------------- prepare and issue the next job
+    bool have_job = false;
+    if (pend == 0 && tile < n_tiles) {
+      buf ^= 1;
+      b = nb; h = nh; win0 = nwin0;
+      wins = min(4, n_win - win0);
+      const int rows = wins * W;
+      if (tid < TILE) sm.mod[buf][tid] = tid < rows ? next_mod : 255;
+      const int ntile = tile + 1;
+      if (ntile < n_tiles) {   // next tile of the range: step the coordinates, no divisions
+        nwin0 += 4;
+        if (nwin0 >= tiles_per_unit * 4) { nwin0 = 0; if (++nh == cv.n_kv_heads) { nh = 0; nb++; } }
+      }
+      fetch_next_mod(ntile);
+      issue_tile(ntile, buf ^ 1, nb, nh, nwin0);                 // prefetch
+      asm volatile("cp.async.wait_group 1;\n" ::: "memory");    // this tile has landed
+      __syncthreads();
+      // norms with the exact adjacent-pair summation tree, four threads per token, read from the staged
+      // tile: a 16-byte chunk (8 channels) is three levels of the tree, a thread's four chunks two more,
+      // the four threads of a token the last two (shuffles between neighbouring lanes)
+      if (worker) {
+        const int r = tid >> 2, q = tid & 3;
+        float part[4];
 #pragma unroll
-      for (int i = 0; i < 4; i++) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(sm.a[buf] + tile_off(r, (4 * q + i) * 8));
-        const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-        float2 x0 = __half22float2(h2[0]), x1 = __half22float2(h2[1]), x2 = __half22float2(h2[2]), x3 = __half22float2(h2[3]);
-        float s0 = __fadd_rn(__fmul_rn(x0.x, x0.x), __fmul_rn(x0.y, x0.y));
-        float s1 = __fadd_rn(__fmul_rn(x1.x, x1.x), __fmul_rn(x1.y, x1.y));
-        float s2 = __fadd_rn(__fmul_rn(x2.x, x2.x), __fmul_rn(x2.y, x2.y));
-        float s3 = __fadd_rn(__fmul_rn(x3.x, x3.x), __fmul_rn(x3.y, x3.y));
-        part[i] = __fadd_rn(__fadd_rn(s0, s1), __fadd_rn(s2, s3));
+        for (int i = 0; i < 4; i++) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(sm.a[buf] + tile_off(r, (4 * q + i) * 8));
+          const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+          float2 x0 = __half22float2(h2[0]), x1 = __half22float2(h2[1]), x2 = __half22float2(h2[2]), x3 = __half22float2(h2[3]);
+          float s0 = __fadd_rn(__fmul_rn(x0.x, x0.x), __fmul_rn(x0.y, x0.y));
+          float s1 = __fadd_rn(__fmul_rn(x1.x, x1.x), __fmul_rn(x1.y, x1.y));
+          float s2 = __fadd_rn(__fmul_rn(x2.x, x2.x), __fmul_rn(x2.y, x2.y));
+          float s3 = __fadd_rn(__fmul_rn(x3.x, x3.x), __fmul_rn(x3.y, x3.y));
+          part[i] = __fadd_rn(__fadd_rn(s0, s1), __fadd_rn(s2, s3));
+        }
+        float sum = __fadd_rn(__fadd_rn(part[0], part[1]), __fadd_rn(part[2], part[3]));
+        sum = __fadd_rn(sum, __shfl_xor_sync(0xffffffffu, sum, 1));
+        sum = __fadd_rn(sum, __shfl_xor_sync(0xffffffffu, sum, 2));
+        if (q == 0 && r < rows) {
+          float n = __fsqrt_rn(sum);
+          n = n > 65504.0f ? 65504.0f : n;
+          const __half nh16 = __float2half_rn(n);
+          const float nf = __half2float(nh16);
+          unsigned char* rec = cv.record(layer, b, h, win0 + (r >> 5));
+          reinterpret_cast<__half*>(rec + OFF_VNORM)[norm_pos(r & 31)] = nh16;
+          sm.inv[buf][r] = nf != 0.0f ? __fdiv_rn(1.0f, nf) : 0.0f;
+        }
       }
-      float sum = __fadd_rn(__fadd_rn(part[0], part[1]), __fadd_rn(part[2], part[3]));
-      sum = __fadd_rn(sum, __shfl_xor_sync(0xffffffffu, sum, 1));
-      sum = __fadd_rn(sum, __shfl_xor_sync(0xffffffffu, sum, 2));
-      if (q == 0 && r < rows) {
-        float n = __fsqrt_rn(sum);
-        n = n > 65504.0f ? 65504.0f : n;
-        const __half nh = __float2half_rn(n);
-        const float nf = __half2float(nh);
-        unsigned char* rec = cv.record(layer, b, h, win0 + (r >> 5));
-        reinterpret_cast<__half*>(rec + OFF_VNORM)[norm_pos(r & 31)] = nh;
-        sm.inv[r] = nf != 0.0f ? __fdiv_rn(1.0f, nf) : 0.0f;
+      {
+        const uint32_t m4 = reinterpret_cast<const uint32_t*>(sm.mod[buf])[lane];   // 4 tokens per lane
+        unsigned mine = 0;
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+          const unsigned mm = (m4 >> (8 * u)) & 0xffu;
+          if (mm < 3) mine |= 1u << mm;
+        }
+#pragma unroll
+        for (int d = 16; d; d >>= 1) mine |= __shfl_xor_sync(0xffffffffu, mine, d);
+        pend = mine;
       }
     }
-    __syncthreads();
-    unsigned present = 0;
-    for (int m = 0; m < 3; m++) {
-      int any = 0;
-      for (int r = lane; r < rows; r += 32) any |= (sm.mod[r] == m);
-      if (__any_sync(0xffffffffu, any)) present |= 1u << m;
-    }
-
-    const int rset = n_R == 1 ? 0 : h;
-    for (int m = 0; m < 3; m++) {
-      if (!((present >> m) & 1)) continue;
-      const int key = rset * 3 + m;
+    int m = 0;
+    if (pend) {
+      m = __ffs(pend) - 1;
+      pend &= ~(1u << m);
+      const int key = (n_R == 1 ? 0 : h) * 3 + m;
       int slot = slot_key[0] == key ? 0 : (slot_key[1] == key ? 1 : -1);
       if (slot < 0) {
         // not resident: replace the slot that was not used last.  Split R_m into fp16 hi + lo, laid out
         // as the B operand (row = output channel, K = input channel)
         slot = last_slot ^ 1;
         const float* Rm = R + (size_t)key * D * D;
-        for (int idx = tid; idx < D * D / 8; idx += NT) {
+        for (int idx = tid; idx < (worker ? D * D / 8 : 0); idx += NT) {
           const int n = idx >> 4, kc = idx & 15;
           const float4 x0 = __ldg(reinterpret_cast<const float4*>(Rm + n * D + kc * 8));
           const float4 x1 = __ldg(reinterpret_cast<const float4*>(Rm + n * D + kc * 8 + 4));
@@ -211,8 +247,9 @@ __global__ void __launch_bounds__(NT, 1) k_quantize_values_tc(CacheView cv, int 
       asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // generic-proxy writes -> tensor-core reads
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
       __syncthreads();
-      if (tid == 0) {
+      if (tid == NT) {
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const uint32_t dcol = tmem + (uint32_t)(jobs & 1) * 128;
 #pragma unroll 1
         for (int part = 0; part < 2; part++)
 #pragma unroll 1
@@ -222,73 +259,83 @@ __global__ void __launch_bounds__(NT, 1) k_quantize_values_tc(CacheView cv, int 
             const uint32_t accumulate = (part | s) ? 1u : 0u;
             asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                          "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
-                         ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+                         ::"r"(dcol), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
           }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(&sm.mbar)) : "memory");
       }
-      const bool ok = __syncthreads_and(mbar_wait(smem_u32(&sm.mbar), phase) ? 1 : 0) != 0;   // same answer in every thread
-      phase ^= 1;
-      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-      if (!ok) { failed = true; break; }
-      // epilogue: warp w reads tensor-memory lanes 32*(w&3).. (token rows) and the 32 columns (w>>2)*32..
-      // (output channels).  tcgen05.ld is warp-collective, so every lane reads; only tokens of
-      // modality m keep the result.
-      {
-        const int row = (warp & 3) * 32 + lane, cc = warp >> 2;
-        const bool mine = sm.mod[row] == m;
-        const float inv = sm.inv[row];
-        unsigned char* crow = sm.code + row * CSTRIDE + cc * 32;
-        uint32_t r[32];
-        const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + cc * 32;
-        asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
-                     : "=r"(r[0]),"=r"(r[1]),"=r"(r[2]),"=r"(r[3]),"=r"(r[4]),"=r"(r[5]),"=r"(r[6]),"=r"(r[7]),"=r"(r[8]),"=r"(r[9]),"=r"(r[10]),"=r"(r[11]),"=r"(r[12]),"=r"(r[13]),"=r"(r[14]),"=r"(r[15]),
-                       "=r"(r[16]),"=r"(r[17]),"=r"(r[18]),"=r"(r[19]),"=r"(r[20]),"=r"(r[21]),"=r"(r[22]),"=r"(r[23]),"=r"(r[24]),"=r"(r[25]),"=r"(r[26]),"=r"(r[27]),"=r"(r[28]),"=r"(r[29]),"=r"(r[30]),"=r"(r[31])
-                     : "r"(taddr) : "memory");
-        asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-        if (mine) {
+      have_job = true;
+    }
+
+    // ---------------- epilogue of the previous job, while the tensor cores work on this one
+    if (p_valid && worker) {
+      // warp w reads tensor-memory lanes 32*(w&3).. (token rows) and the 32 columns (w>>2)*32.. (output
+      // channels).  tcgen05.ld is warp-collective, so every lane reads; only tokens of the job's
+      // modality keep the result.
+      const int row = (warp & 3) * 32 + lane, cc = warp >> 2;
+      const bool mine = sm.mod[p_buf][row] == p_mod;
+      const float inv = sm.inv[p_buf][row];
+      uint32_t r[32];
+      const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)p_acc * 128 + cc * 32;
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+                   : "=r"(r[0]),"=r"(r[1]),"=r"(r[2]),"=r"(r[3]),"=r"(r[4]),"=r"(r[5]),"=r"(r[6]),"=r"(r[7]),"=r"(r[8]),"=r"(r[9]),"=r"(r[10]),"=r"(r[11]),"=r"(r[12]),"=r"(r[13]),"=r"(r[14]),"=r"(r[15]),
+                     "=r"(r[16]),"=r"(r[17]),"=r"(r[18]),"=r"(r[19]),"=r"(r[20]),"=r"(r[21]),"=r"(r[22]),"=r"(r[23]),"=r"(r[24]),"=r"(r[25]),"=r"(r[26]),"=r"(r[27]),"=r"(r[28]),"=r"(r[29]),"=r"(r[30]),"=r"(r[31])
+                   : "r"(taddr) : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+      if (mine) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            uint32_t packed = 0;
+        for (int half = 0; half < 2; half++) {
+          uint32_t word = 0;
 #pragma unroll
-            for (int u = 0; u < 4; u++) {
-              const float z = __fmul_rn(__uint_as_float(r[j + u]), inv);
-              packed |= (uint32_t)((z > -CB_THRESH) + (z > 0.0f) + (z > CB_THRESH)) << (8 * u);
-            }
-            *reinterpret_cast<uint32_t*>(crow + j) = packed;
+          for (int u = 0; u < 16; u++) {
+            const float z = __fmul_rn(__uint_as_float(r[16 * half + u]), inv);
+            word |= (uint32_t)((z > -CB_THRESH) + (z > 0.0f) + (z > CB_THRESH)) << (2 * u);
           }
+          sm.cw[p_buf][row][2 * cc + half] = word;
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-      __syncthreads();   // TMEM and the code buffer are consistent before the next MMA / the packing
     }
-
-    if (failed) break;
-    // pack the codes of each window in record order (value codes are the A operand of the decode kernel)
-    for (int wi = tid; wi < wins * 256; wi += NT) {
-      const int wq = wi >> 8, w8 = wi & 255;
-      const int mu = (w8 >> 7) * 4 + (w8 & 3);
-      const int l = (w8 & 127) >> 2;
-      const int g = l >> 2, t = l & 3;
-      uint32_t word = 0;
+    if (p_valid && p_last) {
+      __syncthreads();   // all codes of the tile are in the buffer (every warp, the issuing one included)
+      if (worker) {
+        // pack the codes of each window in record order (value codes are the A operand of the decode kernel)
+        for (int wi = tid; wi < p_wins * 256; wi += NT) {
+          const int wq = wi >> 8, w8 = wi & 255;
+          const int mu = (w8 >> 7) * 4 + (w8 & 3);
+          const int l = (w8 & 127) >> 2;
+          const int g = l >> 2, t = l & 3;
+          uint32_t word = 0;
 #pragma unroll
-      for (int q = 0; q < 8; q++) {
-        const int shf = q >> 2, j = q & 3;
+          for (int j = 0; j < 4; j++) {
 #pragma unroll
-        for (int e = 0; e < 2; e++) {
-          const int i = 16 * (j >> 1) + 8 * (j & 1) + 2 * t + e;
-          const int c = 16 * mu + 8 * shf + g;
-          word |= (uint32_t)sm.code[(wq * W + i) * CSTRIDE + c] << (16 * e + 8 * shf + 2 * j);
+            for (int e = 0; e < 2; e++) {
+              const int i = 16 * (j >> 1) + 8 * (j & 1) + 2 * t + e;
+              const uint32_t src = sm.cw[p_buf][wq * W + i][mu];          // channels 16*mu .. 16*mu+15 of token i
+              word |= ((src >> (2 * g)) & 3u) << (16 * e + 2 * j);       // channel 16*mu + g
+              word |= ((src >> (2 * (8 + g))) & 3u) << (16 * e + 8 + 2 * j);   // channel 16*mu + 8 + g
+            }
+          }
+          reinterpret_cast<uint32_t*>(cv.record(layer, p_b, p_h, p_win0 + wq) + OFF_VCODE)[w8] = word;
         }
       }
-      reinterpret_cast<uint32_t*>(cv.record(layer, b, h, win0 + wq) + OFF_VCODE)[w8] = word;
     }
-    __syncthreads();
+    if (!have_job) break;
+
+    // ---------------- wait for this job's MMAs (warp 0 polls; the block barrier spreads the answer)
+    const bool ok = __syncthreads_and(warp != 0 || mbar_wait(smem_u32(&sm.mbar), phase) ? 1 : 0) != 0;
+    phase ^= 1;
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    if (!ok) { failed = true; break; }
+    p_valid = true; p_last = pend == 0; p_buf = buf; p_mod = m; p_acc = jobs & 1;
+    p_b = b; p_h = h; p_win0 = win0; p_wins = wins;
+    jobs++;
+    if (pend == 0) tile += 1;
   }
   asm volatile("cp.async.wait_group 0;\n" ::: "memory");
   if (tid == 0 && failed) atomicCAS(cv.status, 0, (int)OKQ_ERR_TIMEOUT);
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
   __syncthreads();
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 128;\n" ::"r"(tmem) : "memory");
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;\n" ::"r"(tmem) : "memory");
 }
 
 okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __half* v, const int64_t strides[3],
@@ -305,7 +352,7 @@ okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __hal
   const long long n_tiles = (long long)((n_win + 3) / 4) * cv.n_kv_heads * cv.batch;
   if (n_tiles == 0) return OKQ_OK;
   const int grid = (int)(n_tiles < n_sm ? n_tiles : n_sm);
-  k_quantize_values_tc<<<grid, NT, sizeof(TcSmem) + 1024, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
+  k_quantize_values_tc<<<grid, NT_ALL, sizeof(TcSmem) + 1024, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
                                                                 modality, n_tokens, R, n_R);
   return OKQ_OK;
 }
