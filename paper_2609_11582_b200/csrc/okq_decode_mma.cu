@@ -115,6 +115,9 @@ __device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int p
   const int g = lane >> 2, t = lane & 3;
   const float fsc = sm.fscale[g];
   float run_m = -INFINITY, run_l = 0.f;
+  uint2 qreg[16];
+#pragma unroll
+  for (int r = 0; r < 16; r++) qreg[r] = sm.qf[r][lane];
 
   auto issue = [&](int k) {
     if (k < sg.n_my) {
@@ -158,7 +161,7 @@ __device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int p
 #pragma unroll
         for (int half = 0; half < 2; half++) {
           const int kappa = 2 * kq + half;
-          const uint2 q0 = sm.qf[2 * kappa][lane], q1 = sm.qf[2 * kappa + 1][lane];
+          const uint2 q0 = qreg[2 * kappa], q1 = qreg[2 * kappa + 1];
           uint32_t a0, a1, a2, a3;
           split_product(u2h(q0.x), u2h(q0.y), u2h(half ? m4.z : m4.x), a0, a1);
           split_product(u2h(q1.x), u2h(q1.y), u2h(half ? m4.w : m4.y), a2, a3);

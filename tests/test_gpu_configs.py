@@ -101,3 +101,39 @@ def test_full_7b_step_sampled():
         ref, _ = O.attention(1, qs, kq, vq, modrow, kt, vt, signs[sl].numpy(), R[sl].numpy())
         errs = Hn.assert_attention_close(o[sl, sb], ref.reshape(Hq, D))
         print(f"full step7b layer {sl} seq {sb}: rel-L2 {errs[0]:.2e} worst head {errs[1]:.2e} max-abs {errs[2]:.2e}")
+
+
+def test_ragged_batch_lengths():
+    """Sequences of different lengths in one decode call (lengths set per sequence, tails filled to match):
+    the persistent kernel's partition follows the per-sequence window counts."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=4, n_layers=2, n_tokens=1500)
+    c = Hn.Case(w, capacity=1536)
+    dev = c.cache.device
+    lengths = np.array([[1500, 40, 700, 0], [33, 1499, 31, 1024]])        # [layer][sequence]
+    U = w.batch * w.n_kv_heads
+    kt = c.cache.k_tail.view(2, w.batch, w.n_kv_heads, W, D)
+    vt = c.cache.v_tail.view(2, w.batch, w.n_kv_heads, W, D)
+    for l in range(2):
+        for b in range(w.batch):
+            n = int(lengths[l, b]); npk = (n // W) * W
+            if n > npk:
+                kt[l, b, :, : n - npk] = c.k[l][b, :, npk:n].to(dev)
+                vt[l, b, :, : n - npk] = c.v[l][b, :, npk:n].to(dev)
+    c.cache.seq_len.copy_(torch.from_numpy(lengths.reshape(-1).astype(np.int32)).to(dev))
+    got = c.gpu_decode(0, layer_count=2)
+    got_simt = c.gpu_decode(0, layer_count=2, simt=True)
+    for l in range(2):
+        for b in range(w.batch):
+            n = int(lengths[l, b])
+            if n == 0:
+                assert (got[l, b] == 0).all() and (got_simt[l, b] == 0).all()
+                continue
+            kb = Hn.u16(c.k[l][b, :, :n]); vb = Hn.u16(c.v[l][b, :, :n])
+            mod = c.mod_b[b, :n].numpy()
+            kq, vq, _ = O.quantize_batch(kb, vb, mod, c.signs[l].numpy(), c.R[l].numpy())
+            npk = (n // W) * W
+            q = Hn.u16(c.q[l, b]).reshape(w.n_kv_heads, w.group, D)
+            ref, _ = O.attention(1, q, kq, vq, mod, kb[:, npk:], vb[:, npk:], c.signs[l].numpy(), c.R[l].numpy())
+            ref = ref.reshape(w.n_q_heads, D)
+            Hn.assert_attention_close(got[l, b], ref)
+            Hn.assert_attention_close(got_simt[l, b], ref)
