@@ -478,9 +478,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
 constexpr int CB_SEQ = 4;                 // sequences per combine CTA (one 128-thread group each)
 constexpr int CB_ROWS = CB_SEQ * GP;      // (sequence, head) rows per combine CTA
 
+constexpr int CB_CHUNK = 32;              // rows of a rotation matrix staged per step
+
 struct CombineSmem {
-  __align__(16) float Rm[D][D];  // one modality's rotation matrix, staged with cp.async
-  float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
+  __align__(16) float Rbuf[2][CB_CHUNK][D];   // double-buffered 32-row slices of the rotation matrices
+  __align__(16) float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
+  __align__(16) float rawv[CB_ROWS][D];       // raw-tail contribution, [row][channel]
   float tsc[CB_SEQ][W][GP];     // tail scores (log2 domain)
   float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
   int prefix[MAX_ENTRIES + 1];
@@ -556,7 +559,6 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
     sm.Ls[bs][c] = L;
   }
   __syncthreads();
-  float raw[GP];
 #pragma unroll
   for (int j = 0; j < GP; j++) {
     float v[3] = {0.f, 0.f, 0.f}, a = 0.f;
@@ -579,45 +581,69 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
     sm.vec[0][bs * GP + j][c] = v[0];
     sm.vec[1][bs * GP + j][c] = v[1];
     sm.vec[2][bs * GP + j][c] = v[2];
-    raw[j] = a;
+    sm.rawv[bs * GP + j][c] = a;
   }
-  __syncthreads();
 
-  // out[row][c] = sum_m sum_r R_m[r][c] * vec[m][row][r] for this group's GP rows; each matrix
-  // is staged in shared memory once per CTA
-  float o[GP];
-#pragma unroll
-  for (int j = 0; j < GP; j++) o[j] = 0.f;
+  // out[row][c] = raw[row][c] + sum_m sum_r R_m[r][c] * vec[m][row][r].  Threads 0..255 compute a
+  // 4-row x 4-column tile each; threads 256..511 stream the matrices through shared memory in
+  // 32-row slices, one slice ahead.
+  const bool comp = threadIdx.x < 256;
+  const int rw = (threadIdx.x >> 5) * 4, cl = (threadIdx.x & 31) * 4;   // first row / column of the tile
   const float* Rset = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D;
-  for (int m = 0; m < 3; m++) {
-    __syncthreads();   // everyone is done with the previous matrix
-    {
-      const float* src = Rset + (size_t)m * D * D;
-      float* dst = &sm.Rm[0][0];
-      for (int i = threadIdx.x; i < D * D / 4; i += CB_SEQ * 128) cp_async16(dst + 4 * i, src + 4 * i);
-      cp_async_commit();
-      cp_async_wait<0>();
-    }
-    __syncthreads();
-#pragma unroll 2
-    for (int r = 0; r < D; r += 4) {
-      const float r0 = sm.Rm[r][c], r1 = sm.Rm[r + 1][c], r2 = sm.Rm[r + 2][c], r3 = sm.Rm[r + 3][c];
+  constexpr int N_CHUNK = 3 * D / CB_CHUNK;
+  auto stage = [&](int chunk) {   // rows [32*chunk, 32*chunk+32) of the three stacked matrices
+    const float* src = Rset + (size_t)chunk * CB_CHUNK * D;
+    float* dst = &sm.Rbuf[chunk & 1][0][0];
+    for (int i = threadIdx.x - 256; i < CB_CHUNK * D / 4; i += 256) cp_async16(dst + 4 * i, src + 4 * i);
+    cp_async_commit();
+  };
+  float o[4][4];
 #pragma unroll
-      for (int j = 0; j < GP; j++) {
-        const float4 x = *reinterpret_cast<const float4*>(&sm.vec[m][bs * GP + j][r]);
-        o[j] = fmaf(r0, x.x, o[j]);
-        o[j] = fmaf(r1, x.y, o[j]);
-        o[j] = fmaf(r2, x.z, o[j]);
-        o[j] = fmaf(r3, x.w, o[j]);
+  for (int i = 0; i < 4; i++)
+#pragma unroll
+    for (int k = 0; k < 4; k++) o[i][k] = 0.f;
+  if (!comp) stage(0);
+  for (int chunk = 0; chunk < N_CHUNK; chunk++) {
+    if (!comp) cp_async_wait<0>();
+    __syncthreads();   // slice `chunk` has landed; everyone is done with slice chunk-1 (and, first time, vec is complete)
+    if (!comp) {
+      if (chunk + 1 < N_CHUNK) stage(chunk + 1);
+    } else {
+      const int m = chunk / (D / CB_CHUNK), r0 = (chunk % (D / CB_CHUNK)) * CB_CHUNK;
+#pragma unroll 2
+      for (int r = 0; r < CB_CHUNK; r += 4) {
+        float4 rr[4], x[4];
+#pragma unroll
+        for (int k = 0; k < 4; k++) rr[k] = *reinterpret_cast<const float4*>(&sm.Rbuf[chunk & 1][r + k][cl]);
+#pragma unroll
+        for (int i = 0; i < 4; i++) x[i] = *reinterpret_cast<const float4*>(&sm.vec[m][rw + i][r0 + r]);
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+          o[i][0] = fmaf(rr[0].x, x[i].x, o[i][0]); o[i][1] = fmaf(rr[0].y, x[i].x, o[i][1]);
+          o[i][2] = fmaf(rr[0].z, x[i].x, o[i][2]); o[i][3] = fmaf(rr[0].w, x[i].x, o[i][3]);
+          o[i][0] = fmaf(rr[1].x, x[i].y, o[i][0]); o[i][1] = fmaf(rr[1].y, x[i].y, o[i][1]);
+          o[i][2] = fmaf(rr[1].z, x[i].y, o[i][2]); o[i][3] = fmaf(rr[1].w, x[i].y, o[i][3]);
+          o[i][0] = fmaf(rr[2].x, x[i].z, o[i][0]); o[i][1] = fmaf(rr[2].y, x[i].z, o[i][1]);
+          o[i][2] = fmaf(rr[2].z, x[i].z, o[i][2]); o[i][3] = fmaf(rr[2].w, x[i].z, o[i][3]);
+          o[i][0] = fmaf(rr[3].x, x[i].w, o[i][0]); o[i][1] = fmaf(rr[3].y, x[i].w, o[i][1]);
+          o[i][2] = fmaf(rr[3].z, x[i].w, o[i][2]); o[i][3] = fmaf(rr[3].w, x[i].w, o[i][3]);
+        }
       }
     }
   }
-  if (live) {
+  if (comp) {
 #pragma unroll
-    for (int j = 0; j < GP; j++) {
-      if (j >= G) continue;
-      const float L = sm.Ls[bs][j];
-      P.out[(((size_t)li * cv.batch + b) * cv.n_q_heads + h * G + j) * D + c] = L > 0.f ? (o[j] + raw[j]) / L : 0.f;
+    for (int i = 0; i < 4; i++) {
+      const int row = rw + i, ob = blockIdx.y * CB_SEQ + row / GP, j = row % GP;
+      if (ob >= cv.batch || j >= G) continue;
+      const float L = sm.Ls[row / GP][j];
+      const float4 rv = *reinterpret_cast<const float4*>(&sm.rawv[row][cl]);
+      float4 res = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (L > 0.f) {
+        const float inv = 1.0f / L;
+        res = make_float4((o[i][0] + rv.x) * inv, (o[i][1] + rv.y) * inv, (o[i][2] + rv.z) * inv, (o[i][3] + rv.w) * inv);
+      }
+      *reinterpret_cast<float4*>(&P.out[(((size_t)li * cv.batch + ob) * cv.n_q_heads + h * G + j) * D + cl]) = res;
     }
   }
 }
