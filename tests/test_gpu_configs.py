@@ -137,3 +137,24 @@ def test_ragged_batch_lengths():
             ref = ref.reshape(w.n_q_heads, D)
             Hn.assert_attention_close(got[l, b], ref)
             Hn.assert_attention_close(got_simt[l, b], ref)
+
+
+@pytest.mark.parametrize("n_q,n_kv", [(4, 4), (8, 2), (6, 1)])
+def test_other_gqa_groups(n_q, n_kv):
+    """GQA groups 1, 4 and 6 (the kernels pad the group to 8 heads)."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], n_q_heads=n_q, n_kv_heads=n_kv, batch=2, n_tokens=300 + 11)
+    c = Hn.Case(w)
+    ref, _ = c.oracle_attention(0)
+    Hn.assert_attention_close(c.gpu_decode(0)[0], ref)
+    Hn.assert_attention_close(c.gpu_decode(0, simt=True)[0], ref)
+
+
+def test_layer_offset_and_many_sequences():
+    """A call on layers [1, 3) of a 3-layer cache with more (layer, sequence) pairs than one launch
+    covers (the library then launches layer by layer)."""
+    w = WL.scaled(WL.WORKLOADS["tiny"], n_layers=3, batch=600, n_tokens=40)
+    c = Hn.Case(w, capacity=64)
+    got = c.gpu_decode(1, layer_count=2)
+    for i, l in enumerate((1, 2)):
+        ref, _ = c.oracle_attention(l)
+        Hn.assert_attention_close(got[i], ref)
