@@ -508,6 +508,11 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
   const int per = total > 0 ? (total + n_cta - 1) / n_cta : 1;
   constexpr float ACC_SCALE = (CB_OUTER - CB_INNER) * 262144.0f;  // (b - a) * 2^18
   constexpr float LOG2E = 1.4426950408889634f;
+  // Coefficient of the weight sum S: -b from the codebook identity, plus the mean of what the bit-1
+  // plane loses because its relative weight (3a-b)/(2(b-a)) enters the MMA rounded to fp16 (bit 1 is
+  // set for half of the codes on average); the zero-mean remainder is at the 1e-5 level.
+  constexpr float DELTA_REL = (3.0f * CB_INNER - CB_OUTER) / (2.0f * (CB_OUTER - CB_INNER));
+  const float S_COEF = -CB_OUTER + (CB_OUTER - CB_INNER) * (DELTA_REL - __half2float(__float2half_rn(DELTA_REL)));
 
   const int e = li * cv.batch + bb;
   const int seq = live ? cv.seq_len[layer * cv.batch + bb] : 0;
@@ -573,7 +578,7 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
         for (int m = 0; m < 3; m++) {
           // weight sum of head j: the four lanes of quad j hold partial sums
           const float S = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
-          v[m] = fmaf(fmaf(ACC_SCALE, pp.frag[m][r][l32], -CB_OUTER * S), ef, v[m]);
+          v[m] = fmaf(fmaf(ACC_SCALE, pp.frag[m][r][l32], S_COEF * S), ef, v[m]);
         }
       }
       for (int i = 0; i < n_tail; i++) a = fmaf(exp2f(sm.tsc[bs][i][j] - M), __half2float(vt[i * D + c]), a);
