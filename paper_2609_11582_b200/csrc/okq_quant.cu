@@ -24,31 +24,101 @@ struct WindowSmem {
 };
 
 // Key window: rows(i) = rows + i*stride, i = 0..31.  128 threads.
+//
+// The 128-point transform is done in two in-register halves around one shared-memory transpose:
+// eight threads per token first hold 16 consecutive channels each (stages h = 1, 2, 4, 8, and the
+// first four levels of the norm's summation tree), then each holds the 2 x 8 channels that differ in
+// the three high index bits (stages h = 16, 32, 64).  The stage order, and with it every rounding,
+// is that of the plain butterfly loop.
 __device__ void quantize_key_window(const __half* rows, long long stride, const float* __restrict__ signs,
                                     unsigned char* rec, WindowSmem& sm) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const float4 sg = *reinterpret_cast<const float4*>(signs + 4 * lane);
+  const int tid = threadIdx.x;
   __half* knorm = reinterpret_cast<__half*>(rec + OFF_KNORM);
-  for (int k = 0; k < 8; k++) {
-    int i = warp * 8 + k;
-    float4 x = load_row4(rows + (long long)i * stride, lane);
-    float n = warp_norm(x);
-    __half nh = __float2half_rn(n);
-    float nf = __half2float(nh);
-    float4 y = make_float4(__fmul_rn(sg.x, x.x), __fmul_rn(sg.y, x.y), __fmul_rn(sg.z, x.z), __fmul_rn(sg.w, x.w));
-    y = warp_fwht(y, lane);
-    float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (nf != 0.0f) {
-      float cinv = __fdiv_rn(RSQRT_D, nf);
-      z = make_float4(__fmul_rn(y.x, cinv), __fmul_rn(y.y, cinv), __fmul_rn(y.z, cinv), __fmul_rn(y.w, cinv));
+  const int a = tid & 7;          // which 16-channel block (first half) / which channel pair (second half)
+  float sg[16];
+#pragma unroll
+  for (int q = 0; q < 4; q++) {
+    const float4 s4 = *reinterpret_cast<const float4*>(signs + 16 * a + 4 * q);
+    sg[4 * q] = s4.x; sg[4 * q + 1] = s4.y; sg[4 * q + 2] = s4.z; sg[4 * q + 3] = s4.w;
+  }
+#pragma unroll 1
+  for (int round = 0; round < 2; round++) {
+    const int i = (tid >> 3) + 16 * round;   // token; its eight threads are neighbours in one warp
+    float* zrow = &sm.z[i * ZS];
+    float y[16];
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(rows + (long long)i * stride + 16 * a);
+      const uint4 r0 = src[0], r1 = src[1];
+      const __half2* h0 = reinterpret_cast<const __half2*>(&r0);
+      const __half2* h1 = reinterpret_cast<const __half2*>(&r1);
+#pragma unroll
+      for (int q = 0; q < 4; q++) {
+        const float2 f0 = __half22float2(h0[q]), f1 = __half22float2(h1[q]);
+        y[2 * q] = f0.x; y[2 * q + 1] = f0.y; y[8 + 2 * q] = f1.x; y[8 + 2 * q + 1] = f1.y;
+      }
     }
-    *reinterpret_cast<float4*>(&sm.z[i * ZS + 4 * lane]) = z;
-    if (lane == 0) knorm[norm_pos(i)] = nh;
+    // norm: adjacent-pair tree (4 levels here, 3 across the eight threads)
+    float t[16];
+#pragma unroll
+    for (int c = 0; c < 16; c++) t[c] = __fmul_rn(y[c], y[c]);
+#pragma unroll
+    for (int n = 8; n >= 1; n >>= 1)
+#pragma unroll
+      for (int c = 0; c < n; c++) t[c] = __fadd_rn(t[2 * c], t[2 * c + 1]);
+    float ssum = t[0];
+    ssum = __fadd_rn(ssum, __shfl_xor_sync(0xffffffffu, ssum, 1));
+    ssum = __fadd_rn(ssum, __shfl_xor_sync(0xffffffffu, ssum, 2));
+    ssum = __fadd_rn(ssum, __shfl_xor_sync(0xffffffffu, ssum, 4));
+    float nrm = __fsqrt_rn(ssum);
+    nrm = nrm > 65504.0f ? 65504.0f : nrm;
+    const __half nh = __float2half_rn(nrm);
+    const float nf = __half2float(nh);
+    if (a == 0) knorm[norm_pos(i)] = nh;
+    const float cinv = nf != 0.0f ? __fdiv_rn(RSQRT_D, nf) : 0.0f;
+    // D x, then stages h = 1, 2, 4, 8 inside the 16-channel block
+#pragma unroll
+    for (int c = 0; c < 16; c++) y[c] = __fmul_rn(sg[c], y[c]);
+#pragma unroll
+    for (int hh = 1; hh < 16; hh <<= 1)
+#pragma unroll
+      for (int j = 0; j < 16; j++)
+        if ((j & hh) == 0) {
+          const float p = y[j], q2 = y[j + hh];
+          y[j] = __fadd_rn(p, q2);
+          y[j + hh] = __fsub_rn(p, q2);
+        }
+#pragma unroll
+    for (int q = 0; q < 4; q++)
+      *reinterpret_cast<float4*>(&zrow[16 * a + 4 * q]) = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+    __syncwarp();
+    // second half: channels 16*u + 2*a + e, u = 0..7: stages h = 16, 32, 64 act on u
+    float v0[8], v1[8];
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      const float2 p = *reinterpret_cast<const float2*>(&zrow[16 * u + 2 * a]);
+      v0[u] = p.x; v1[u] = p.y;
+    }
+#pragma unroll
+    for (int hh = 1; hh < 8; hh <<= 1)
+#pragma unroll
+      for (int j = 0; j < 8; j++)
+        if ((j & hh) == 0) {
+          float p = v0[j], q2 = v0[j + hh];
+          v0[j] = __fadd_rn(p, q2); v0[j + hh] = __fsub_rn(p, q2);
+          p = v1[j]; q2 = v1[j + hh];
+          v1[j] = __fadd_rn(p, q2); v1[j + hh] = __fsub_rn(p, q2);
+        }
+    __syncwarp();   // every thread of the token has read the first-half values before they are overwritten
+#pragma unroll
+    for (int u = 0; u < 8; u++)
+      *reinterpret_cast<float2*>(&zrow[16 * u + 2 * a]) =
+          nf != 0.0f ? make_float2(__fmul_rn(v0[u], cinv), __fmul_rn(v1[u], cinv)) : make_float2(0.f, 0.f);
   }
   __syncthreads();
   {  // per channel: window minimum and step (Eq. 4)
     int c = tid;
     float mn = sm.z[c], mx = mn;
+#pragma unroll 8
     for (int i = 1; i < W; i++) {
       float v = sm.z[i * ZS + c];
       if (v < mn) mn = v;
@@ -67,26 +137,37 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
     reinterpret_cast<__half*>(rec + OFF_KS)[p] = sh;
   }
   __syncthreads();
-  uint32_t* words = reinterpret_cast<uint32_t*>(rec + OFF_KCODE);
-  for (int wi = tid; wi < 256; wi += 128) {
-    int h2 = wi >> 7, rem = wi & 127;
-    int l = rem >> 2, tt = (rem >> 1) & 1, ww = rem & 1;
-    int g = l >> 2, t = l & 3;
-    int i = g + 8 * (2 * h2 + tt);
-    uint32_t word = 0;
+  // codes: a thread keeps the (m, 1/s) of the 16 channels of "its" word position (t, ww) in registers
+  // and packs that word for two tokens
+  {
+    uint32_t* words = reinterpret_cast<uint32_t*>(rec + OFF_KCODE);
+    const int t = tid & 3, ww = (tid >> 2) & 1, tg = tid >> 3;   // tg: 16 token pairs
+    float mch[16], rch[16];
 #pragma unroll
     for (int q = 0; q < 8; q++) {
-      int r = ww * 8 + q;
-      int kappa = r >> 1, pair = r & 1;
-#pragma unroll
-      for (int e = 0; e < 2; e++) {
-        int c = 16 * kappa + 8 * pair + 2 * t + e;
-        float qv = rintf(__fmul_rn(__fsub_rn(sm.z[i * ZS + c], sm.a[c]), sm.b[c]));
-        uint32_t code = qv < 0.0f ? 0u : (qv > 3.0f ? 3u : (uint32_t)qv);
-        word |= code << (16 * e + 8 * (q >> 2) + 2 * (q & 3));
-      }
+      const int c0 = 16 * ((ww * 8 + q) >> 1) + 8 * (q & 1) + 2 * t;
+      const float2 m2 = *reinterpret_cast<const float2*>(&sm.a[c0]);
+      const float2 r2 = *reinterpret_cast<const float2*>(&sm.b[c0]);
+      mch[2 * q] = m2.x; mch[2 * q + 1] = m2.y; rch[2 * q] = r2.x; rch[2 * q + 1] = r2.y;
     }
-    words[wi] = word;
+#pragma unroll
+    for (int k = 0; k < 2; k++) {
+      const int i = 2 * tg + k;
+      uint32_t word = 0;
+#pragma unroll
+      for (int q = 0; q < 8; q++) {
+        const int c0 = 16 * ((ww * 8 + q) >> 1) + 8 * (q & 1) + 2 * t;
+        const float2 z2 = *reinterpret_cast<const float2*>(&sm.z[i * ZS + c0]);
+#pragma unroll
+        for (int e = 0; e < 2; e++) {
+          const float qv = rintf(__fmul_rn(__fsub_rn(e ? z2.y : z2.x, mch[2 * q + e]), rch[2 * q + e]));
+          const uint32_t code = (uint32_t)fminf(fmaxf(qv, 0.0f), 3.0f);   // clamp to [0, 3]
+          word |= code << (16 * e + 8 * (q >> 2) + 2 * (q & 3));
+        }
+      }
+      // word index of (token i, t, ww): [i >> 4][lane 4*(i & 7) + t][(i >> 3) & 1][ww]
+      words[(i >> 4) * 128 + (4 * (i & 7) + t) * 4 + ((i >> 3) & 1) * 2 + ww] = word;
+    }
   }
   __syncthreads();
 }
