@@ -180,6 +180,130 @@ void okqo_window_quantize(const float* z, uint16_t* meta, uint8_t* codes) {
   }
 }
 
+/* ---------------------------------------------------------------- MXFP4 (m, s) metadata
+ *
+ * The paper's default metadata format ("MXFP4 metadata by default", Implementation details):
+ * m and s are each stored as 4-bit E2M1 elements sharing one 8-bit power-of-two scale (E8M0) per
+ * block of 32.  The paper does not say how blocks are formed or how values are rounded; the
+ * reading taken here (listed in the design notes):
+ *   - a block is 32 consecutive channels of one window, separately for m and for s;
+ *   - the scale is the smallest power of two 2^k with 6 * 2^k >= max|x| over the block (6 is
+ *     the largest E2M1 magnitude), k clamped to [-23, 12] so that every decoded value
+ *     grid * 2^k is exactly an fp16 number;
+ *   - m is rounded DOWN to the E2M1 grid {0, .5, 1, 1.5, 2, 3, 4, 6} * 2^k (with sign), the
+ *     step s is rounded UP, so the four levels m' + s' * {0,1,2,3} always cover [min, max];
+ *   - codes are computed against the decoded pair (m', s') exactly as in the fp16 format.
+ * 2 * (128 * 4 + 4 * 8) bits per 32-token window = 136 B instead of 512 B: 72.25 B per token per
+ * KV head = 2.258 bits per element, the figure the paper prints for its default.
+ */
+static const float MX_GRID[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+
+int okqo_bytes_per_window_mx(void) { return OKQ_W * ((OKQ_D * 2) / 8 + 2 + (OKQ_D * 2) / 8 + 2) + 2 * (OKQ_D / 2 + OKQ_D / 32); }
+
+/* smallest k in [-23, 12] with 6 * 2^k >= amax */
+int okqo_mx_scale_exp(float amax) {
+  int k = -23;
+  if (amax > 0.0f) {
+    int e;
+    float f = frexpf(amax, &e); /* amax = f * 2^e, f in [0.5, 1); 6 * 2^k = 0.75 * 2^(k+3) */
+    k = (f <= 0.75f) ? e - 3 : e - 2;
+  }
+  if (k < -23) k = -23;
+  if (k > 12) k = 12;
+  return k;
+}
+
+/* nibble (sign << 3 | grid index) of x on the grid * 2^k; mode < 0 rounds down, mode > 0 rounds up */
+uint8_t okqo_mx_encode(float x, int k, int mode) {
+  float q = ldexpf(x, -k); /* exact */
+  int best = -1;
+  float bestv = 0.0f;
+  for (int sgn = 0; sgn < 2; sgn++)
+    for (int i = 0; i < 8; i++) {
+      if (sgn && i == 0) continue; /* no negative zero */
+      float g = sgn ? -MX_GRID[i] : MX_GRID[i];
+      int ok = mode < 0 ? (g <= q) : (g >= q);
+      if (!ok) continue;
+      if (best < 0 || (mode < 0 ? g > bestv : g < bestv)) { best = (sgn << 3) | i; bestv = g; }
+    }
+  if (best < 0) best = mode < 0 ? (1 << 3 | 7) : 7; /* beyond the grid: saturate (cannot happen with the scale above) */
+  return (uint8_t)best;
+}
+
+float okqo_mx_decode(uint8_t nib, int k) {
+  float g = MX_GRID[nib & 7];
+  return ldexpf((nib & 8) ? -g : g, k);
+}
+
+/* Eq. 4 with MXFP4 metadata for one window.  mx: 136 bytes = m nibbles [64] (channel c in byte c/2,
+ * low nibble for even c), s nibbles [64], m scales [4] (k + 127), s scales [4].  meta_dec: the decoded
+ * (m', s') as fp16 [128][2], the same array the fp16 format stores.  codes as okqo_window_quantize. */
+void okqo_window_quantize_mx(const float* z, uint8_t* mx, uint16_t* meta_dec, uint8_t* codes) {
+  float mn[OKQ_D], mxv[OKQ_D], md[OKQ_D], sr[OKQ_D], sd[OKQ_D];
+  memset(codes, 0, OKQ_W * OKQ_D / 4);
+  memset(mx, 0, 136);
+  for (int c = 0; c < OKQ_D; c++) {
+    mn[c] = mxv[c] = z[c];
+    for (int i = 1; i < OKQ_W; i++) {
+      float v = z[i * OKQ_D + c];
+      if (v < mn[c]) mn[c] = v;
+      if (v > mxv[c]) mxv[c] = v;
+    }
+  }
+  for (int b = 0; b < OKQ_D / 32; b++) { /* minima: scale from the block's largest magnitude, round down */
+    float amax = 0.0f;
+    for (int c = 32 * b; c < 32 * b + 32; c++) if (fabsf(mn[c]) > amax) amax = fabsf(mn[c]);
+    int k = okqo_mx_scale_exp(amax);
+    mx[128 + b] = (uint8_t)(k + 127);
+    for (int c = 32 * b; c < 32 * b + 32; c++) {
+      uint8_t nib = okqo_mx_encode(mn[c], k, -1);
+      mx[c / 2] |= (uint8_t)(nib << (4 * (c & 1)));
+      md[c] = okqo_mx_decode(nib, k);
+      float range = mxv[c] - md[c];
+      if (range < 0.0f) range = 0.0f;
+      sr[c] = range / 3.0f;
+    }
+  }
+  for (int b = 0; b < OKQ_D / 32; b++) { /* steps: round up */
+    float amax = 0.0f;
+    for (int c = 32 * b; c < 32 * b + 32; c++) if (sr[c] > amax) amax = sr[c];
+    int k = okqo_mx_scale_exp(amax);
+    mx[132 + b] = (uint8_t)(k + 127);
+    for (int c = 32 * b; c < 32 * b + 32; c++) {
+      uint8_t nib = okqo_mx_encode(sr[c], k, +1);
+      mx[64 + c / 2] |= (uint8_t)(nib << (4 * (c & 1)));
+      sd[c] = okqo_mx_decode(nib, k);
+    }
+  }
+  for (int c = 0; c < OKQ_D; c++) {
+    meta_dec[2 * c] = okqo_float_to_half(md[c]);     /* exact: every decoded value is an fp16 number */
+    meta_dec[2 * c + 1] = okqo_float_to_half(sd[c]);
+    if (!(sd[c] > 0.0f)) continue;
+    float r = 1.0f / sd[c];
+    for (int i = 0; i < OKQ_W; i++) {
+      float q = rintf((z[i * OKQ_D + c] - md[c]) * r);
+      int code = q < 0.0f ? 0 : (q > 3.0f ? 3 : (int)q);
+      codes[i * (OKQ_D / 4) + c / 4] |= (uint8_t)(code << (2 * (c % 4)));
+    }
+  }
+}
+
+/* Key quantiser with MXFP4 metadata over one (layer, sequence, KV head).  mx: [n_windows][136]. */
+int64_t okqo_quantize_keys_mx(const uint16_t* k, int64_t n_tokens, const float* signs, uint8_t* codes,
+                              uint16_t* norms, uint16_t* meta_dec, uint8_t* mx) {
+  int64_t n_win = n_tokens / OKQ_W;
+  float* z = (float*)malloc(sizeof(float) * OKQ_W * OKQ_D);
+  for (int64_t g = 0; g < n_win; g++) {
+    for (int i = 0; i < OKQ_W; i++) {
+      int64_t tok = g * OKQ_W + i;
+      okqo_key_rotate(k + tok * OKQ_D, signs, norms + tok, z + i * OKQ_D);
+    }
+    okqo_window_quantize_mx(z, mx + g * 136, meta_dec + g * OKQ_D * 2, codes + g * OKQ_W * (OKQ_D / 4));
+  }
+  free(z);
+  return n_win * OKQ_W;
+}
+
 /* Key quantiser over one (layer, sequence, KV head): tokens [0, n_tokens); the first
  * floor(n/32)*32 are packed.  Returns the number of packed tokens. */
 int64_t okqo_quantize_keys(const uint16_t* k, int64_t n_tokens, const float* signs,
@@ -451,11 +575,27 @@ int okqo_attention_batch(int path, int U, const uint16_t* q, int G, int64_t n_pa
 }
 
 /* Quantise many units (keys and values) in parallel; inputs [U][n_tokens][128] fp16. */
+int okqo_quantize_batch_fmt(int U, const uint16_t* k, const uint16_t* v, int64_t n_tokens,
+                            const uint8_t* modality, int64_t mod_stride, const int32_t* unit_seq,
+                            const int32_t* unit_rot, const float* signs, const float* R,
+                            uint8_t* k_codes, uint16_t* k_norm, uint16_t* k_meta, uint8_t* v_codes,
+                            uint16_t* v_norm, int meta_format, uint8_t* k_mx);
+
 int okqo_quantize_batch(int U, const uint16_t* k, const uint16_t* v, int64_t n_tokens,
                         const uint8_t* modality, int64_t mod_stride, const int32_t* unit_seq,
                         const int32_t* unit_rot, const float* signs, const float* R,
                         uint8_t* k_codes, uint16_t* k_norm, uint16_t* k_meta, uint8_t* v_codes,
                         uint16_t* v_norm) {
+  return okqo_quantize_batch_fmt(U, k, v, n_tokens, modality, mod_stride, unit_seq, unit_rot, signs, R, k_codes,
+                                 k_norm, k_meta, v_codes, v_norm, 0, NULL);
+}
+
+/* meta_format 0: fp16 (m, s); 1: MXFP4 (k_meta receives the decoded pairs, k_mx [U][n_win][136] the stored bytes) */
+int okqo_quantize_batch_fmt(int U, const uint16_t* k, const uint16_t* v, int64_t n_tokens,
+                            const uint8_t* modality, int64_t mod_stride, const int32_t* unit_seq,
+                            const int32_t* unit_rot, const float* signs, const float* R,
+                            uint8_t* k_codes, uint16_t* k_norm, uint16_t* k_meta, uint8_t* v_codes,
+                            uint16_t* v_norm, int meta_format, uint8_t* k_mx) {
   int threads = 1;
   int64_t np = (n_tokens / OKQ_W) * OKQ_W;
 #ifdef _OPENMP
@@ -463,9 +603,14 @@ int okqo_quantize_batch(int U, const uint16_t* k, const uint16_t* v, int64_t n_t
 #pragma omp parallel for schedule(dynamic, 1)
 #endif
   for (int u = 0; u < U; u++) {
-    okqo_quantize_keys(k + (size_t)u * n_tokens * OKQ_D, n_tokens, signs + (size_t)unit_rot[u] * OKQ_D,
-                       k_codes + (size_t)u * np * 32, k_norm + (size_t)u * np,
-                       k_meta + (size_t)u * (np / OKQ_W) * OKQ_D * 2);
+    if (meta_format == 1)
+      okqo_quantize_keys_mx(k + (size_t)u * n_tokens * OKQ_D, n_tokens, signs + (size_t)unit_rot[u] * OKQ_D,
+                            k_codes + (size_t)u * np * 32, k_norm + (size_t)u * np,
+                            k_meta + (size_t)u * (np / OKQ_W) * OKQ_D * 2, k_mx + (size_t)u * (np / OKQ_W) * 136);
+    else
+      okqo_quantize_keys(k + (size_t)u * n_tokens * OKQ_D, n_tokens, signs + (size_t)unit_rot[u] * OKQ_D,
+                         k_codes + (size_t)u * np * 32, k_norm + (size_t)u * np,
+                         k_meta + (size_t)u * (np / OKQ_W) * OKQ_D * 2);
     okqo_quantize_values(v + (size_t)u * n_tokens * OKQ_D, n_tokens,
                          modality + (size_t)unit_seq[u] * mod_stride,
                          R + (size_t)unit_rot[u] * 3 * OKQ_D * OKQ_D, v_codes + (size_t)u * np * 32,

@@ -42,6 +42,14 @@ def lib():
         L.okqo_quantize_values.restype = C.c_int64
         L.okqo_attention_batch.restype = C.c_int
         L.okqo_quantize_batch.restype = C.c_int
+        L.okqo_quantize_batch_fmt.restype = C.c_int
+        L.okqo_bytes_per_window_mx.restype = C.c_int
+        L.okqo_mx_scale_exp.restype = C.c_int
+        L.okqo_mx_scale_exp.argtypes = [C.c_float]
+        L.okqo_mx_encode.restype = C.c_uint8
+        L.okqo_mx_encode.argtypes = [C.c_float, C.c_int, C.c_int]
+        L.okqo_mx_decode.restype = C.c_float
+        L.okqo_mx_decode.argtypes = [C.c_uint8, C.c_int]
         _lib = L
     return _lib
 
@@ -111,6 +119,24 @@ def window_quantize(z: np.ndarray):
     codes = np.empty((W, D // 4), np.uint8)
     lib().okqo_window_quantize(_p(z), _p(meta), _p(codes))
     return meta, codes
+
+
+def window_quantize_mx(z: np.ndarray):
+    """MXFP4-metadata form of window_quantize: (mx bytes uint8 [136], decoded meta uint16 [128,2], codes [32,32])."""
+    z = _c(z, np.float32)
+    assert z.shape == (W, D)
+    mx = np.empty(136, np.uint8)
+    meta = np.empty((D, 2), np.uint16)
+    codes = np.empty((W, D // 4), np.uint8)
+    lib().okqo_window_quantize_mx(_p(z), _p(mx), _p(meta), _p(codes))
+    return mx, meta, codes
+
+
+def mx_unpack(mx: np.ndarray):
+    """Stored MXFP4 bytes [..., 136] -> (m nibbles [...,128], s nibbles [...,128], m exponents [...,4], s exponents [...,4])."""
+    mx = np.asarray(mx, np.uint8)
+    nib = lambda b: np.stack([b & 15, b >> 4], axis=-1).reshape(*b.shape[:-1], D)
+    return nib(mx[..., :64]), nib(mx[..., 64:128]), mx[..., 128:132].astype(np.int32) - 127, mx[..., 132:136].astype(np.int32) - 127
 
 
 def quantize_keys(k_bits: np.ndarray, signs: np.ndarray):
@@ -194,8 +220,9 @@ def attention(path: int, q_bits, kq, vq, modality, k_tail, v_tail, signs, R, sm_
     return out, th
 
 
-def quantize_batch(k_bits, v_bits, modality, signs, R, unit_seq=None, unit_rot=None):
-    """k_bits, v_bits [U,n,128] u16 -> (kq, vq) stacked dicts, threads used."""
+def quantize_batch(k_bits, v_bits, modality, signs, R, unit_seq=None, unit_rot=None, meta_format=0):
+    """k_bits, v_bits [U,n,128] u16 -> (kq, vq) stacked dicts, threads used.
+    meta_format 1 = MXFP4 metadata: kq["meta"] holds the decoded (m', s') and kq["mx"] the stored bytes."""
     k_bits = _c(k_bits, np.uint16); v_bits = _c(v_bits, np.uint16)
     U, n, _ = k_bits.shape
     npk = (n // W) * W
@@ -209,7 +236,11 @@ def quantize_batch(k_bits, v_bits, modality, signs, R, unit_seq=None, unit_rot=N
     kq = {"codes": np.zeros((U, npk, 32), np.uint8), "norm": np.zeros((U, npk), np.uint16),
           "meta": np.zeros((U, npk // W, D, 2), np.uint16)}
     vq = {"codes": np.zeros((U, npk, 32), np.uint8), "norm": np.zeros((U, npk), np.uint16)}
-    th = lib().okqo_quantize_batch(C.c_int(U), _p(k_bits), _p(v_bits), C.c_int64(n), _p(modality),
-                                   C.c_int64(modality.shape[1]), _p(unit_seq), _p(unit_rot), _p(signs), _p(R),
-                                   _p(kq["codes"]), _p(kq["norm"]), _p(kq["meta"]), _p(vq["codes"]), _p(vq["norm"]))
+    mx = np.zeros((U, npk // W, 136), np.uint8)
+    th = lib().okqo_quantize_batch_fmt(C.c_int(U), _p(k_bits), _p(v_bits), C.c_int64(n), _p(modality),
+                                       C.c_int64(modality.shape[1]), _p(unit_seq), _p(unit_rot), _p(signs), _p(R),
+                                       _p(kq["codes"]), _p(kq["norm"]), _p(kq["meta"]), _p(vq["codes"]), _p(vq["norm"]),
+                                       C.c_int(meta_format), _p(mx))
+    if meta_format == 1:
+        kq["mx"] = mx
     return kq, vq, th

@@ -440,3 +440,76 @@ def test_attention_batch_matches_single_units():
     assert th >= 1
     for u, c in enumerate(cs):
         assert np.abs(out[u] - _run(1, c)).max() < 1e-13
+
+
+# ------------------------------------------------------------------ MXFP4 (m, s) metadata (the paper's default)
+
+E2M1 = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6])
+
+
+def test_mx_storage_rate_matches_paper_table():
+    gold = read_golden("bits_per_elem.txt")
+    L = O.lib()
+    assert L.okqo_bytes_per_window_mx() == 2312                       # 72.25 B per token per KV head
+    assert round(L.okqo_bytes_per_window_mx() * 8 / (W * 2 * D), 3) == gold["omnikvquant_k2v2_mxfp4_meta"]
+
+
+def test_mx_scale_and_rounding_against_brute_force():
+    L = O.lib()
+    rng = np.random.default_rng(21)
+    signed_grid = np.concatenate([-E2M1[:0:-1], E2M1])
+    for amax in np.concatenate([10.0 ** rng.uniform(-9, 0.5, 300), [0.75, 1.5, 6.0, 3.0, 2.0 ** -24, 1e-12, 0.0]]):
+        amax = float(np.float32(amax))
+        k = L.okqo_mx_scale_exp(amax)
+        ks = [kk for kk in range(-23, 13) if 6.0 * 2.0 ** kk >= amax]
+        assert k == (ks[0] if ks else 12)                               # smallest power of two that covers the block
+    for _ in range(400):
+        k = int(rng.integers(-8, 3))
+        x = float(np.float32(rng.uniform(-6, 6) * 2.0 ** k))
+        pts = signed_grid * 2.0 ** k
+        lo = L.okqo_mx_decode(L.okqo_mx_encode(x, k, -1), k)
+        hi = L.okqo_mx_decode(L.okqo_mx_encode(x, k, +1), k)
+        assert lo == pts[pts <= x].max() and hi == pts[pts >= x].min()
+    # nibble layout: sign in bit 3, grid index in bits 0..2; zero is never negative
+    assert L.okqo_mx_encode(0.0, 0, -1) == 0 and L.okqo_mx_encode(-0.0, 0, +1) == 0
+    assert L.okqo_mx_encode(-6.0, 0, -1) == 0b1111 and L.okqo_mx_encode(1.5, 0, +1) == 0b0011
+
+
+def test_mx_window_covers_range_and_is_fp16_exact():
+    rng = np.random.default_rng(22)
+    z = (rng.standard_normal((W, D)) / math.sqrt(D)).astype(np.float32)
+    z[:, 5] *= 10; z[:, 40] = 0.0; z[:, 41] = 1e-7
+    mx, meta, codes = O.window_quantize_mx(z)
+    mn, sn, mk, sk = O.mx_unpack(mx)
+    sign = lambda n: np.where(n & 8, -1.0, 1.0)
+    m_dec = sign(mn) * E2M1[mn & 7] * 2.0 ** np.repeat(mk, 32)
+    s_dec = sign(sn) * E2M1[sn & 7] * 2.0 ** np.repeat(sk, 32)
+    # the decoded pairs are exactly the fp16 numbers in `meta`
+    assert (bits2f(meta[:, 0]) == m_dec).all() and (bits2f(meta[:, 1]) == s_dec).all()
+    assert (s_dec >= 0).all()
+    zmin, zmax = z.min(0).astype(np.float64), z.max(0).astype(np.float64)
+    assert (m_dec <= zmin).all()                                      # m rounds down ...
+    assert (m_dec + 3 * s_dec >= zmax - 1e-7).all()                   # ... s rounds up: the four levels cover the window
+    c = O.unpack_codes(codes)
+    assert c.min() >= 0 and c.max() <= 3
+    zhat = m_dec[None] + s_dec[None] * c
+    assert (np.abs(zhat - z) <= s_dec[None] / 2 + 1e-7).all()          # nothing is clipped
+    # coarser metadata costs accuracy relative to the fp16 format, but not much (the paper's table:
+    # key reconstruction error 0.1833 with MXFP4 metadata against 0.1495 with FP16 metadata)
+    meta16, codes16 = O.window_quantize(z)
+    z16 = bits2f(meta16[:, 0])[None] + bits2f(meta16[:, 1])[None] * O.unpack_codes(codes16)
+    e_mx, e_16 = ((zhat - z) ** 2).mean(), ((z16 - z) ** 2).mean()
+    assert 1.0 < e_mx / e_16 < 2.5
+
+
+def test_mx_attention_paths_agree():
+    """The attention oracle only sees the decoded (m', s'): definition path == rotated-space path."""
+    c = _small_case(139, seed=31)
+    kq, vq, _ = O.quantize_batch(c["kb"][None], c["vb"][None], c["mod"], c["signs"], c["R"], meta_format=1)
+    assert kq["mx"].shape == (1, 4, 136)
+    a, _ = O.attention(0, c["q"][None], kq, vq, c["mod"], c["kt"][None], c["vt"][None], c["signs"], c["R"])
+    b, _ = O.attention(1, c["q"][None], kq, vq, c["mod"], c["kt"][None], c["vt"][None], c["signs"], c["R"])
+    assert np.abs(a - b).max() < 1e-10
+    # and differs measurably from the fp16-metadata cache (it is a different, coarser encoding)
+    ref = _run(0, c)
+    assert np.abs(a[0] - ref).max() > 1e-4 and np.isfinite(a).all()
