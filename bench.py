@@ -211,6 +211,9 @@ def main():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling on a small case)")
+    ap.add_argument("--meta", default="fp16", choices=["fp16", "mxfp4"],
+                    help="(m, s) metadata format of the cache: fp16 = 84 B per token and KV head (the headline "
+                         "configuration), mxfp4 = 72.25 B (secondary measurement; no cpu_baseline, no ncu traffic)")
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
                     help="decode: the headline decode step; prefill: bulk quantisation of a fresh fp16 K/V cache "
                          "(secondary measurement, default workload prefill7b)")
@@ -236,7 +239,9 @@ def main():
 
     # ---- build the packed cache on the device (setup, untimed)
     L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
-    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev)
+    mx = args.meta == "mxfp4"
+    bytes_th = 72.25 if mx else BYTES_PER_TOKEN_HEAD
+    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev, meta_format=B.META_MXFP4 if mx else B.META_FP16)
     mod = WL.modality_layout(w).unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
     signs = torch.stack([WL.gen_signs(w, l) for l in range(L)]).to(dev)
     R = torch.stack([WL.gen_rotations(w, l) for l in range(L)]).unsqueeze(1).contiguous().to(dev)
@@ -259,7 +264,7 @@ def main():
     q_dev = q_host.to(dev); kn_dev = kn_host.to(dev); vn_dev = vn_host.to(dev); mn_dev = mn_host.to(dev)
     out = torch.empty(L, Bn, Hq, 128, dtype=torch.float32, device=dev)
     ws = torch.empty(max(16, B.decode_workspace_bytes(cache, L, args.splits)), dtype=torch.uint8, device=dev)
-    packed_bytes = L * Bn * H * N * BYTES_PER_TOKEN_HEAD
+    packed_bytes = int(L * Bn * H * N * bytes_th)
 
     def step_resident(s):
         B.append(cache, 0, L, kn_dev[s], vn_dev[s], mn_dev, signs, R)
@@ -319,12 +324,12 @@ def main():
     e2e_value = world * packed_bytes / (ms_e2e / args.steps * 1e-3) / 1e9
     peak, peak_kind = measured_peaks()
     achieved = packed_bytes / (kernel_ms * 1e-3) / 1e9
-    traffic = None if NCU_DRAM_BYTES_PER_TOKEN_HEAD is None else NCU_DRAM_BYTES_PER_TOKEN_HEAD * L * Bn * H * N
+    traffic = None if NCU_DRAM_BYTES_PER_TOKEN_HEAD is None or mx else NCU_DRAM_BYTES_PER_TOKEN_HEAD * L * Bn * H * N
 
     if rank != 0:
         return
     cpu = None
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and not mx:
         n_l, n_s = min(2, L), min(8, Bn)
         oargs, unit_rot, th_units = oracle_prepare(w, n_l, n_s)
         passes = [oracle_pass(oargs, unit_rot) for _ in range(3)]
@@ -337,8 +342,9 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "n_layers": L, "batch": Bn, "n_q_heads": Hq, "n_kv_heads": H, "context": N,
+                       "meta_format": args.meta, "bytes_per_token_head": bytes_th,
                        "step": "okq_append(1 text token/seq, all layers) + okq_decode_attention(all layers), one call each",
-                       "packed_kv_bytes_per_step": packed_bytes, "l2": "inputs (1.2 GB of records per step) exceed L2",
+                       "packed_kv_bytes_per_step": packed_bytes, "l2": f"inputs ({packed_bytes / 1e9:.2f} GB of records per step) exceed L2",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "GB/s", "ms_per_step": ms_e2e / args.steps,

@@ -28,6 +28,12 @@
  *     [ 576,  640)  value norms, fp16 x 32 tokens
  *     [ 640, 1664)  key codes,   2 bits x 32 tokens x 128 channels
  *     [1664, 2688)  value codes, 2 bits x 32 tokens x 128 channels
+ * With OKQ_META_MXFP4 (the paper's default metadata: 2.258 bits/element) the first 512 bytes shrink to
+ * 136: m and s as 4-bit E2M1 elements with one power-of-two E8M0 scale per 32 consecutive channels
+ * (m rounded down, s rounded up, so the four levels still cover the window; the scale is the smallest
+ * power of two whose 6-fold reaches the block maximum, clamped to [2^-23, 2^12] so that every decoded
+ * value is an fp16 number), OKQ_RECORD_BYTES_MX = 2312 bytes per record, 72.25 per token per KV head.
+ * Codes are computed against the decoded pair, exactly as with fp16 metadata.
  * Inside a record the channel / token order is the one the decode kernel's tensor-core
  * fragments want; okq_cache_export / okq_cache_import convert to and from the canonical
  * arrays (token-major codes with channel c of a token in byte c/4 at bits 2*(c%4);
@@ -45,7 +51,10 @@ extern "C" {
 
 #define OKQ_HEAD_DIM 128
 #define OKQ_WINDOW 32
-#define OKQ_RECORD_BYTES 2688
+#define OKQ_RECORD_BYTES 2688    /* window record with fp16 (m, s) metadata */
+#define OKQ_RECORD_BYTES_MX 2312 /* window record with MXFP4 (m, s) metadata */
+#define OKQ_META_FP16 0
+#define OKQ_META_MXFP4 1
 #define OKQ_MAX_GROUP 8
 #define OKQ_NOALLOC_SCRATCH_BYTES (32u << 20) /* fixed scratch of okq_decode_attention_noalloc */
 
@@ -71,8 +80,8 @@ typedef struct okq_cache {
   int32_t head_dim;  /* 128 */
   int32_t window;    /* 32 */
   int32_t capacity;  /* max tokens per sequence, multiple of 32 */
-  int32_t reserved;  /* 0 */
-  void* records;     /* [n_layers][batch][n_kv_heads][capacity/32][OKQ_RECORD_BYTES] */
+  int32_t meta_format; /* OKQ_META_FP16 (0) or OKQ_META_MXFP4 (1): how the key (m, s) pairs are stored */
+  void* records;     /* [n_layers][batch][n_kv_heads][capacity/32][record bytes of the format]; 16-byte aligned */
   uint8_t* modality; /* [batch][capacity], shared by all layers and heads */
   void* k_tail;      /* [n_layers][batch][n_kv_heads][32][128] fp16: raw keys not yet in a full window */
   void* v_tail;      /* same for values */
@@ -234,6 +243,18 @@ okq_status okq_cache_export(const okq_cache* cache, int32_t layer, uint8_t* k_co
 okq_status okq_cache_import(const okq_cache* cache, int32_t layer, const uint8_t* k_codes,
                             const void* k_norm, const void* k_meta, const uint8_t* v_codes,
                             const void* v_norm, void* stream);
+/*
+ * With OKQ_META_MXFP4, okq_cache_export writes the DECODED (m, s) pairs into k_meta and
+ * okq_cache_import returns OKQ_ERR_UNSUPPORTED (fp16 pairs need not lie on the MX grid).
+ * okq_cache_export_mx (OKQ_META_MXFP4 caches only, else OKQ_ERR_UNSUPPORTED) also writes the
+ * stored metadata bytes in natural channel order:
+ *   k_mx   device uint8 [batch][n_kv_heads][capacity/32][136]:
+ *          [0, 64) m elements, channel c in byte c/2 (even c in the low nibble; bit 3 = sign,
+ *          bits 0-2 index {0, .5, 1, 1.5, 2, 3, 4, 6}); [64, 128) s elements likewise;
+ *          [128, 132) m block exponents k + 127 for channels [32 j, 32 j + 32); [132, 136) s exponents.
+ */
+okq_status okq_cache_export_mx(const okq_cache* cache, int32_t layer, uint8_t* k_codes, void* k_norm,
+                               void* k_meta, uint8_t* k_mx, uint8_t* v_codes, void* v_norm, void* stream);
 
 #ifdef __cplusplus
 }

@@ -14,13 +14,15 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libokq.so")
 
 HEAD_DIM, WINDOW, RECORD_BYTES, MAX_GROUP = 128, 32, 2688, 8
+RECORD_BYTES_MX, MX_META_BYTES = 2312, 136
+META_FP16, META_MXFP4 = 0, 1
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(8)
 
 
 class okq_cache(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("batch", C.c_int32), ("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32),
-                ("head_dim", C.c_int32), ("window", C.c_int32), ("capacity", C.c_int32), ("reserved", C.c_int32),
+                ("head_dim", C.c_int32), ("window", C.c_int32), ("capacity", C.c_int32), ("meta_format", C.c_int32),
                 ("records", C.c_void_p), ("modality", C.c_void_p), ("k_tail", C.c_void_p), ("v_tail", C.c_void_p),
                 ("seq_len", C.c_void_p), ("status", C.c_void_p)]
 
@@ -76,6 +78,8 @@ def lib():
         L.okq_profile_events.argtypes = [C.c_void_p, C.c_void_p]
         L.okq_cache_export.restype = C.c_int
         L.okq_cache_export.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 6
+        L.okq_cache_export_mx.restype = C.c_int
+        L.okq_cache_export_mx.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 7
         L.okq_cache_import.restype = C.c_int
         L.okq_cache_import.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 6
         _lib = L
@@ -86,7 +90,7 @@ def exported_symbols():
     return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
             "okq_cache_import", "okq_profile_events", "okq_decode_attention_simt",
-            "okq_decode_attention_noalloc", "okq_quantize_values_bulk"]
+            "okq_decode_attention_noalloc", "okq_quantize_values_bulk", "okq_cache_export_mx"]
 
 
 def _ptr(t) -> int:
@@ -103,8 +107,9 @@ def _check(st: int, where: str):
         raise OkqError(st, where)
 
 
-def cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, head_dim=HEAD_DIM, window=WINDOW):
-    shape = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, head_dim, window, capacity, 0)
+def cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, head_dim=HEAD_DIM, window=WINDOW,
+                meta_format=META_FP16):
+    shape = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, head_dim, window, capacity, meta_format)
     out = (C.c_size_t * 6)()
     _check(lib().okq_cache_sizes(C.byref(shape), out), "okq_cache_sizes")
     return list(out)
@@ -113,8 +118,9 @@ def cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, head_dim=HEAD_
 class Cache:
     """Device buffers of a 2-bit KV cache plus the C struct that describes them."""
 
-    def __init__(self, n_layers, batch, n_kv_heads, n_q_heads, capacity, device="cuda"):
-        sizes = cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity)
+    def __init__(self, n_layers, batch, n_kv_heads, n_q_heads, capacity, device="cuda", meta_format=META_FP16):
+        sizes = cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, meta_format=meta_format)
+        self.meta_format = meta_format
         self.n_layers, self.batch, self.n_kv_heads, self.n_q_heads, self.capacity = (
             n_layers, batch, n_kv_heads, n_q_heads, capacity)
         self.device = torch.device(device)
@@ -124,7 +130,7 @@ class Cache:
         self.v_tail = torch.zeros(sizes[3] // 2, dtype=torch.float16, device=device)
         self.seq_len = torch.zeros(n_layers * batch, dtype=torch.int32, device=device)
         self.status = torch.zeros(4, dtype=torch.int32, device=device)
-        self.c = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, HEAD_DIM, WINDOW, capacity, 0,
+        self.c = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, HEAD_DIM, WINDOW, capacity, meta_format,
                            self.records.data_ptr(), self.modality.data_ptr(), self.k_tail.data_ptr(),
                            self.v_tail.data_ptr(), self.seq_len.data_ptr(), self.status.data_ptr())
 
@@ -134,7 +140,8 @@ class Cache:
 
     def packed_bytes(self, n_tokens):
         """Bytes of packed records a decode step over n_tokens per sequence must read."""
-        return self.n_layers * self.batch * self.n_kv_heads * (n_tokens // WINDOW) * RECORD_BYTES
+        return self.n_layers * self.batch * self.n_kv_heads * (n_tokens // WINDOW) * (
+            RECORD_BYTES_MX if self.meta_format == META_MXFP4 else RECORD_BYTES)
 
     def device_status(self) -> int:
         return int(self.status[0].item())
@@ -206,6 +213,12 @@ def cache_export(cache: Cache, layer: int, stream=None):
            "k_meta": torch.empty(B, H, cap // WINDOW, HEAD_DIM, 2, dtype=torch.float16, device=dev),
            "v_codes": torch.empty(B, H, cap, 32, dtype=torch.uint8, device=dev),
            "v_norm": torch.empty(B, H, cap, dtype=torch.float16, device=dev)}
+    if cache.meta_format == META_MXFP4:   # k_meta = decoded pairs, k_mx = the stored bytes
+        out["k_mx"] = torch.empty(B, H, cap // WINDOW, MX_META_BYTES, dtype=torch.uint8, device=dev)
+        _check(lib().okq_cache_export_mx(C.byref(cache.c), layer, _ptr(out["k_codes"]), _ptr(out["k_norm"]),
+                                         _ptr(out["k_meta"]), _ptr(out["k_mx"]), _ptr(out["v_codes"]),
+                                         _ptr(out["v_norm"]), _stream(stream)), "okq_cache_export_mx")
+        return out
     _check(lib().okq_cache_export(C.byref(cache.c), layer, _ptr(out["k_codes"]), _ptr(out["k_norm"]),
                                   _ptr(out["k_meta"]), _ptr(out["v_codes"]), _ptr(out["v_norm"]), _stream(stream)),
            "okq_cache_export")

@@ -88,9 +88,20 @@ __global__ void __launch_bounds__(128) k_decode_simt(DecodeParams P) {
   const float cb[4] = {-CB_OUTER, -CB_INNER, CB_INNER, CB_OUTER};
 
   for (int win = w_begin + warp; win < w_end; win += 4) {
-    const unsigned char* rec = cv.record(layer, b, h, win);
-    for (int i = lane; i < RECORD_BYTES / 16; i += 32)
-      reinterpret_cast<uint4*>(ws.rec)[i] = __ldg(reinterpret_cast<const uint4*>(rec) + i);
+    if (cv.fmt == FMT_FP16) {
+      const unsigned char* rec = cv.meta(layer, b, h, win);
+      for (int i = lane; i < RECORD_BYTES / 16; i += 32)
+        reinterpret_cast<uint4*>(ws.rec)[i] = __ldg(reinterpret_cast<const uint4*>(rec) + i);
+    } else {
+      // same staged image as with fp16 metadata: the body behind 512 bytes of decoded (m, s)
+      const unsigned char* body = cv.body(layer, b, h, win);
+      for (int i = lane; i < BODY_BYTES / 16; i += 32)
+        reinterpret_cast<uint4*>(ws.rec + META_BYTES_FP16)[i] = __ldg(reinterpret_cast<const uint4*>(body) + i);
+      uint2 m4, s4;
+      mx_decode_lane(cv.meta(layer, b, h, win), lane, m4, s4);
+      *reinterpret_cast<uint2*>(ws.rec + OFF_KM + 8 * lane) = m4;
+      *reinterpret_cast<uint2*>(ws.rec + OFF_KS + 8 * lane) = s4;
+    }
     ws.mod[lane] = cv.modality[(size_t)b * cv.capacity + (size_t)win * W + lane];
     __syncwarp();
     // per-window weights and bias

@@ -34,7 +34,10 @@ constexpr int NPAIR = 8;                        // warp pairs per CTA
 constexpr int NTHREADS = NPAIR * 64;
 constexpr int NSTAGE = 4;                       // record ring per pair
 constexpr int PREFETCH = 2;                     // windows in flight ahead of the score warp
-constexpr int STAGE_BYTES = RECORD_BYTES + 32;  // record + the window's 32 modality bytes
+// staged window image: the fp16-metadata record, the window's 32 modality bytes and, with MXFP4
+// metadata, the 136 stored metadata bytes (decoded into the first 512 bytes by the score warp)
+constexpr int STAGE_MOD = RECORD_BYTES, STAGE_MX = RECORD_BYTES + 32;
+template <int FMT> constexpr int stage_bytes() { return FMT == FMT_MXFP4 ? STAGE_MX + 144 : STAGE_MX; }
 constexpr float RESCALE_LOG2 = 3.0f;            // numerators stay below 2^3 * 2^6 * vnorm in fp16
 constexpr int SPILL_REGS = 33;                  // 32 accumulator registers + the running weight sum
 
@@ -46,8 +49,9 @@ struct Handoff {
   int pad[15];
 };
 
+template <int FMT>
 struct MmaSmem {
-  __align__(16) unsigned char stage[NPAIR][NSTAGE][STAGE_BYTES];
+  __align__(16) unsigned char stage[NPAIR][NSTAGE][stage_bytes<FMT>()];
   __align__(16) Handoff hand[NPAIR][2];
   float spill[NPAIR][3][SPILL_REGS][32];
   float spill_m[NPAIR][3][GP];
@@ -68,6 +72,10 @@ __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
   uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
+}
+__device__ __forceinline__ void cp_async8(void* smem, const void* gmem) {
+  uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(s), "l"(gmem));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
 template <int N>
@@ -110,7 +118,8 @@ struct Segment {
 };
 
 // ---------------------------------------------------------------- score warp
-__device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int pair, int lane, float& run_m_out,
+template <int FMT>
+__device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, int pair, int lane, float& run_m_out,
                                            float& run_l_out) {
   const int g = lane >> 2, t = lane & 3;
   const float fsc = sm.fscale[g];
@@ -123,13 +132,26 @@ __device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int p
     if (k < sg.n_my) {
       const int win = sg.w0 + k;
       unsigned char* dst = sm.stage[pair][k % NSTAGE];
-      const unsigned char* src = sg.rec0 + (size_t)win * RECORD_BYTES;
+      if (FMT == FMT_FP16) {
+        const unsigned char* src = sg.rec0 + (size_t)win * RECORD_BYTES;
 #pragma unroll
-      for (int i = 0; i < 6; i++) {
-        int c16 = lane + 32 * i;
-        if (c16 < RECORD_BYTES / 16) cp_async16(dst + 16 * c16, src + 16 * c16);
+        for (int i = 0; i < 6; i++) {
+          int c16 = lane + 32 * i;
+          if (c16 < RECORD_BYTES / 16) cp_async16(dst + 16 * c16, src + 16 * c16);
+        }
+      } else {
+        // body (16-byte aligned) behind the 512 bytes the decoded (m, s) will occupy; the 136
+        // metadata bytes are only 8-byte aligned
+        const unsigned char* body = sg.rec0 + mx_body_off(win);
+        const unsigned char* meta = sg.rec0 + mx_meta_off(win);
+#pragma unroll
+        for (int i = 0; i < 5; i++) {
+          int c16 = lane + 32 * i;
+          if (c16 < BODY_BYTES / 16) cp_async16(dst + META_BYTES_FP16 + 16 * c16, body + 16 * c16);
+        }
+        if (lane < MX_META_BYTES / 8) cp_async8(dst + STAGE_MX + 8 * lane, meta + 8 * lane);
       }
-      if (lane < 2) cp_async16(dst + RECORD_BYTES + 16 * lane, sg.mod0 + (size_t)win * W + 16 * lane);
+      if (lane < 2) cp_async16(dst + STAGE_MOD + 16 * lane, sg.mod0 + (size_t)win * W + 16 * lane);
     }
     cp_async_commit();
   };
@@ -141,7 +163,14 @@ __device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int p
       issue(k + PREFETCH);
       cp_async_wait<PREFETCH>();
       __syncwarp();
-      const unsigned char* st = sm.stage[pair][k % NSTAGE];
+      unsigned char* st = sm.stage[pair][k % NSTAGE];
+      if (FMT == FMT_MXFP4) {   // decode the stored (m, s) into the fp16 planes of the staged image
+        uint2 m4, s4;
+        mx_decode_lane(st + STAGE_MX, lane, m4, s4);
+        *reinterpret_cast<uint2*>(st + OFF_KM + 8 * lane) = m4;
+        *reinterpret_cast<uint2*>(st + OFF_KS + 8 * lane) = s4;
+        __syncwarp();
+      }
       const uint4* mp = reinterpret_cast<const uint4*>(st + OFF_KM + 64 * t);
       const uint4* sp = reinterpret_cast<const uint4*>(st + OFF_KS + 64 * t);
       // bias sum_c q'_c m_c (against the constant operand 4^j 2^-24, two independent chains)
@@ -225,7 +254,8 @@ __device__ __forceinline__ void score_warp(MmaSmem& sm, const Segment& sg, int p
 }
 
 // ---------------------------------------------------------------- value warp
-__device__ __forceinline__ void value_warp(MmaSmem& sm, const Segment& sg, int pair, int lane) {
+template <int FMT>
+__device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, int pair, int lane) {
   const int g = lane >> 2, t = lane & 3;
   float acc[8][4];
 #pragma unroll
@@ -259,7 +289,7 @@ __device__ __forceinline__ void value_warp(MmaSmem& sm, const Segment& sg, int p
         run_S *= ho.alpha[g];
       }
       cur_m = ho.m[g];
-      const unsigned char* wmod = st + RECORD_BYTES;
+      const unsigned char* wmod = st + STAGE_MOD;
       const int mymod = wmod[lane];
       const int first = __shfl_sync(0xffffffffu, mymod, 0);
       const bool uniform = __all_sync(0xffffffffu, mymod == first);
@@ -352,9 +382,10 @@ __device__ __forceinline__ void value_warp(MmaSmem& sm, const Segment& sg, int p
 }  // namespace
 
 // grid = n_cta (persistent), 512 threads
+template <int FMT>
 __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  MmaSmem& sm = *reinterpret_cast<MmaSmem*>(smem_raw);
+  MmaSmem<FMT>& sm = *reinterpret_cast<MmaSmem<FMT>*>(smem_raw);
   const CacheView& cv = P.cv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int pair = warp & (NPAIR - 1);
@@ -423,19 +454,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
     __syncthreads();
 
     Segment sg;
-    sg.rec0 = cv.record(layer, b, h, 0);
+    sg.rec0 = cv.unit(layer, b, h);
     sg.mod0 = cv.modality + (size_t)b * cv.capacity;
     const int cnt = (seg + NPAIR - 1) / NPAIR;   // contiguous ranges: few modality changes per pair
     sg.w0 = w0 + pair * cnt;
     sg.n_my = max(0, min(cnt, seg - pair * cnt));
     if (is_score) {
       float run_m, run_l;
-      score_warp(sm, sg, pair, lane, run_m, run_l);
+      score_warp<FMT>(sm, sg, pair, lane, run_m, run_l);
       run_l += __shfl_xor_sync(0xffffffffu, run_l, 1);
       run_l += __shfl_xor_sync(0xffffffffu, run_l, 2);
       if ((lane & 3) == 0) { sm.wm[pair][lane >> 2] = run_m; sm.wl[pair][lane >> 2] = run_l; }
     } else {
-      value_warp(sm, sg, pair, lane);
+      value_warp<FMT>(sm, sg, pair, lane);
     }
     __syncthreads();
 
@@ -656,14 +687,19 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
 okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, cudaEvent_t before, cudaEvent_t after) {
   static thread_local bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_decode_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MmaSmem));
+    cudaError_t e = cudaFuncSetAttribute(k_decode_mma<FMT_FP16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)sizeof(MmaSmem<FMT_FP16>));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_decode_mma<FMT_MXFP4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)sizeof(MmaSmem<FMT_MXFP4>));
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k_combine_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem));
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
     attr_set = true;
   }
   if (before) cudaEventRecord(before, s);
-  k_decode_mma<<<n_cta, NTHREADS, sizeof(MmaSmem), s>>>(P);
+  if (P.cv.fmt == FMT_MXFP4) k_decode_mma<FMT_MXFP4><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_MXFP4>), s>>>(P);
+  else k_decode_mma<FMT_FP16><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_FP16>), s>>>(P);
   if (after) cudaEventRecord(after, s);
   k_combine_mma<<<dim3(P.cv.n_kv_heads, (P.cv.batch + CB_SEQ - 1) / CB_SEQ, P.layer_count), CB_SEQ * 128,
                   sizeof(CombineSmem), s>>>(P, n_cta);

@@ -69,8 +69,30 @@ __host__ __device__ inline void vcode_pos(int i, int c, int& word, int& bit) {
   bit = 16 * e + 8 * sh + 2 * j;
 }
 
+// A record = metadata (m, s) followed by a "body" [key norms 64 | value norms 64 | key codes 1024 |
+// value codes 1024] whose layout is the same for both metadata formats.
+//   Format 0 (fp16 (m, s)): 512 metadata bytes, records back to back (the offsets above).
+//   Format 1 (MXFP4 (m, s), the paper's default): 136 metadata bytes [m nibbles 64 | s nibbles 64 |
+//   m scales 4 | s scales 4], nibbles in meta_pos order (even position in the low nibble), one E8M0
+//   scale per 32 consecutive channels.  2312 bytes per window; so that every body starts on a 16-byte
+//   boundary, two consecutive windows share one 4624-byte block [meta 0 | meta 1 | body 0 | body 1].
+constexpr int FMT_FP16 = 0, FMT_MXFP4 = 1;
+constexpr int MX_META_BYTES = 136;
+constexpr int META_BYTES_FP16 = 512;
+constexpr int BODY_BYTES = 2176;
+constexpr int B_KNORM = 0, B_VNORM = 64, B_KCODE = 128, B_VCODE = 1152;   // offsets inside a body
+constexpr int MX_PAIR_BYTES = 2 * (MX_META_BYTES + BODY_BYTES);
+static_assert(META_BYTES_FP16 + BODY_BYTES == RECORD_BYTES && OFF_KNORM == META_BYTES_FP16 + B_KNORM &&
+              OFF_VCODE == META_BYTES_FP16 + B_VCODE, "record layout");
+
+__host__ __device__ inline size_t mx_meta_off(size_t win) { return (win >> 1) * MX_PAIR_BYTES + (win & 1) * MX_META_BYTES; }
+__host__ __device__ inline size_t mx_body_off(size_t win) {
+  return (win >> 1) * MX_PAIR_BYTES + 2 * MX_META_BYTES + (win & 1) * BODY_BYTES;
+}
+
 struct CacheView {
   int n_layers, batch, n_kv_heads, n_q_heads, capacity;
+  int fmt;
   unsigned char* records;
   unsigned char* modality;
   __half* k_tail;
@@ -78,8 +100,18 @@ struct CacheView {
   int* seq_len;
   int* status;
   __host__ __device__ inline size_t n_windows() const { return (size_t)capacity / W; }
-  __host__ __device__ inline unsigned char* record(int layer, int b, int h, size_t win) const {
-    return records + ((((size_t)layer * batch + b) * n_kv_heads + h) * n_windows() + win) * RECORD_BYTES;
+  // bytes of the records of one (layer, sequence, KV head)
+  __host__ __device__ inline size_t unit_bytes() const {
+    return fmt == FMT_MXFP4 ? ((n_windows() + 1) / 2) * (size_t)MX_PAIR_BYTES : n_windows() * (size_t)RECORD_BYTES;
+  }
+  __host__ __device__ inline unsigned char* unit(int layer, int b, int h) const {
+    return records + (((size_t)layer * batch + b) * n_kv_heads + h) * unit_bytes();
+  }
+  __host__ __device__ inline unsigned char* meta(int layer, int b, int h, size_t win) const {
+    return unit(layer, b, h) + (fmt == FMT_MXFP4 ? mx_meta_off(win) : win * RECORD_BYTES);
+  }
+  __host__ __device__ inline unsigned char* body(int layer, int b, int h, size_t win) const {
+    return unit(layer, b, h) + (fmt == FMT_MXFP4 ? mx_body_off(win) : win * RECORD_BYTES + META_BYTES_FP16);
   }
   __host__ __device__ inline size_t tail_off(int layer, int b, int h) const {
     return (((size_t)layer * batch + b) * n_kv_heads + h) * (size_t)(W * D);

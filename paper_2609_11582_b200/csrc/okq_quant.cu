@@ -31,9 +31,9 @@ struct WindowSmem {
 // the three high index bits (stages h = 16, 32, 64).  The stage order, and with it every rounding,
 // is that of the plain butterfly loop.
 __device__ void quantize_key_window(const __half* rows, long long stride, const float* __restrict__ signs,
-                                    unsigned char* rec, WindowSmem& sm) {
+                                    unsigned char* rec, unsigned char* body, int fmt, WindowSmem& sm) {
   const int tid = threadIdx.x;
-  __half* knorm = reinterpret_cast<__half*>(rec + OFF_KNORM);
+  __half* knorm = reinterpret_cast<__half*>(body + B_KNORM);
   const int a = tid & 7;          // which 16-channel block (first half) / which channel pair (second half)
   float sg[16];
 #pragma unroll
@@ -124,23 +124,53 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
       if (v < mn) mn = v;
       if (v > mx) mx = v;
     }
-    __half mh = __float2half_rn(mn);
-    float mf = __half2float(mh);
-    float range = __fsub_rn(mx, mf);
-    if (range < 0.0f) range = 0.0f;
-    __half sh = __float2half_rn(__fdiv_rn(range, 3.0f));
-    float sf = __half2float(sh);
-    sm.a[c] = mf;
-    sm.b[c] = sf > 0.0f ? __fdiv_rn(1.0f, sf) : 0.0f;
-    int p = meta_pos(c);
-    reinterpret_cast<__half*>(rec + OFF_KM)[p] = mh;
-    reinterpret_cast<__half*>(rec + OFF_KS)[p] = sh;
+    if (fmt == FMT_FP16) {
+      __half mh = __float2half_rn(mn);
+      float mf = __half2float(mh);
+      float range = __fsub_rn(mx, mf);
+      if (range < 0.0f) range = 0.0f;
+      __half sh = __float2half_rn(__fdiv_rn(range, 3.0f));
+      float sf = __half2float(sh);
+      sm.a[c] = mf;
+      sm.b[c] = sf > 0.0f ? __fdiv_rn(1.0f, sf) : 0.0f;
+      int p = meta_pos(c);
+      reinterpret_cast<__half*>(rec + OFF_KM)[p] = mh;
+      reinterpret_cast<__half*>(rec + OFF_KS)[p] = sh;
+    } else {
+      // MXFP4: a warp is one block of 32 consecutive channels.  m rounds down, s rounds up.
+      const int lane = tid & 31, blk = tid >> 5;
+      float amax = fabsf(mn);
+#pragma unroll
+      for (int d = 16; d; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+      const int km = mx_scale_exp(amax);
+      const unsigned mnib = mx_encode(mn, km, false);
+      const float mf = mx_decode(mnib, km);
+      float range = __fsub_rn(mx, mf);
+      if (range < 0.0f) range = 0.0f;
+      const float sraw = __fdiv_rn(range, 3.0f);
+      float smax = sraw;
+#pragma unroll
+      for (int d = 16; d; d >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, d));
+      const int ks = mx_scale_exp(smax);
+      const unsigned snib = mx_encode(sraw, ks, true);
+      const float sf = mx_decode(snib, ks);
+      sm.a[c] = mf;
+      sm.b[c] = sf > 0.0f ? __fdiv_rn(1.0f, sf) : 0.0f;
+      const int p = meta_pos(c);
+      sm.code[p] = (unsigned char)mnib;          // nibbles in record order, packed two per byte below
+      sm.code[D + p] = (unsigned char)snib;
+      if (lane == 0) { rec[128 + blk] = (unsigned char)(km + 127); rec[132 + blk] = (unsigned char)(ks + 127); }
+    }
   }
   __syncthreads();
+  if (fmt == FMT_MXFP4) {
+    // 128 bytes: m nibbles [0, 64), s nibbles [64, 128)
+    rec[tid] = (unsigned char)(sm.code[2 * tid] | (sm.code[2 * tid + 1] << 4));
+  }
   // codes: a thread keeps the (m, 1/s) of the 16 channels of "its" word position (t, ww) in registers
   // and packs that word for two tokens
   {
-    uint32_t* words = reinterpret_cast<uint32_t*>(rec + OFF_KCODE);
+    uint32_t* words = reinterpret_cast<uint32_t*>(body + B_KCODE);
     const int t = tid & 3, ww = (tid >> 2) & 1, tg = tid >> 3;   // tg: 16 token pairs
     float mch[16], rch[16];
 #pragma unroll
@@ -174,9 +204,9 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
 
 // Value window.  mod[] must already be in sm.mod and sm.uniform set.  Rset = R + rsel*3*D*D.
 __device__ void quantize_value_window(const __half* rows, long long stride, const float* __restrict__ Rset,
-                                      unsigned char* rec, WindowSmem& sm) {
+                                      unsigned char* body, WindowSmem& sm) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  __half* vnorm = reinterpret_cast<__half*>(rec + OFF_VNORM);
+  __half* vnorm = reinterpret_cast<__half*>(body + B_VNORM);
   for (int k = 0; k < 8; k++) {
     int i = warp * 8 + k;
     float4 x = load_row4(rows + (long long)i * stride, lane);
@@ -233,7 +263,7 @@ __device__ void quantize_value_window(const __half* rows, long long stride, cons
     }
   }
   __syncthreads();
-  uint32_t* words = reinterpret_cast<uint32_t*>(rec + OFF_VCODE);
+  uint32_t* words = reinterpret_cast<uint32_t*>(body + B_VCODE);
   for (int wi = tid; wi < 256; wi += 128) {
     int mu = (wi >> 7) * 4 + (wi & 3);
     int l = (wi & 127) >> 2;
@@ -274,7 +304,7 @@ __global__ void __launch_bounds__(128) k_quantize_keys(CacheView cv, int layer, 
   __shared__ WindowSmem sm;
   int win = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const __half* rows = k + b * sb + h * sh + (long long)win * W * st;
-  quantize_key_window(rows, st, signs, cv.record(layer, b, h, win), sm);
+  quantize_key_window(rows, st, signs, cv.meta(layer, b, h, win), cv.body(layer, b, h, win), cv.fmt, sm);
 }
 
 __global__ void __launch_bounds__(128) k_quantize_values(CacheView cv, int layer, const __half* __restrict__ v,
@@ -286,7 +316,7 @@ __global__ void __launch_bounds__(128) k_quantize_values(CacheView cv, int layer
   stage_modality(modality + (size_t)b * n_tokens + (size_t)win * W, sm);
   const __half* rows = v + b * sb + h * sh + (long long)win * W * st;
   const float* Rset = R + (size_t)(n_R == 1 ? 0 : h) * 3 * D * D;
-  quantize_value_window(rows, st, Rset, cv.record(layer, b, h, win), sm);
+  quantize_value_window(rows, st, Rset, cv.body(layer, b, h, win), sm);
 }
 
 // raw tail copy + seq_len (+ modality for the value call); grid (n_kv_heads, batch), 128 threads
@@ -337,8 +367,8 @@ __global__ void __launch_bounds__(128) k_append(CacheView cv, int layer0, const 
   if (h == 0 && threadIdx.x == 32) cv.modality[(size_t)b * cv.capacity + pos] = mnew;
   if (slot != W - 1) return;
   __syncthreads();  // the 32nd token of the window is now visible to the whole block
-  unsigned char* rec = cv.record(layer, b, h, pos / W);
-  quantize_key_window(kt, D, signs + (size_t)li * D, rec, sm);
+  unsigned char* body = cv.body(layer, b, h, pos / W);
+  quantize_key_window(kt, D, signs + (size_t)li * D, cv.meta(layer, b, h, pos / W), body, cv.fmt, sm);
   if (threadIdx.x < 32) {
     unsigned char m = threadIdx.x == W - 1 ? mnew : cv.modality[(size_t)b * cv.capacity + (pos - (W - 1)) + threadIdx.x];
     sm.mod[threadIdx.x] = m;
@@ -348,7 +378,7 @@ __global__ void __launch_bounds__(128) k_append(CacheView cv, int layer0, const 
   }
   __syncthreads();
   const float* Rset = R + ((size_t)li * n_R + (n_R == 1 ? 0 : h)) * 3 * D * D;
-  quantize_value_window(vt, D, Rset, rec, sm);
+  quantize_value_window(vt, D, Rset, body, sm);
 }
 
 __global__ void k_advance(CacheView cv, int layer0, int layer_count) {
@@ -362,13 +392,14 @@ __global__ void k_advance(CacheView cv, int layer0, int layer_count) {
 
 // grid (capacity/32, n_kv_heads, batch), 128 threads
 __global__ void k_export(CacheView cv, int layer, unsigned char* k_codes, __half* k_norm, __half* k_meta,
-                         unsigned char* v_codes, __half* v_norm) {
+                         unsigned char* v_codes, __half* v_norm, unsigned char* k_mx) {
   int win = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const unsigned char* rec = cv.record(layer, b, h, win);
+  const unsigned char* rec = cv.meta(layer, b, h, win);
+  const unsigned char* body = cv.body(layer, b, h, win);
   size_t unit = (size_t)b * cv.n_kv_heads + h;
   size_t tok0 = unit * cv.capacity + (size_t)win * W;
-  const uint32_t* kw = reinterpret_cast<const uint32_t*>(rec + OFF_KCODE);
-  const uint32_t* vw = reinterpret_cast<const uint32_t*>(rec + OFF_VCODE);
+  const uint32_t* kw = reinterpret_cast<const uint32_t*>(body + B_KCODE);
+  const uint32_t* vw = reinterpret_cast<const uint32_t*>(body + B_VCODE);
   for (int idx = threadIdx.x; idx < W * 32; idx += blockDim.x) {
     int i = idx >> 5, byte = idx & 31;
     unsigned kb = 0, vb = 0;
@@ -383,21 +414,35 @@ __global__ void k_export(CacheView cv, int layer, unsigned char* k_codes, __half
     v_codes[(tok0 + i) * 32 + byte] = (unsigned char)vb;
   }
   if (threadIdx.x < W) {
-    k_norm[tok0 + threadIdx.x] = reinterpret_cast<const __half*>(rec + OFF_KNORM)[norm_pos(threadIdx.x)];
-    v_norm[tok0 + threadIdx.x] = reinterpret_cast<const __half*>(rec + OFF_VNORM)[norm_pos(threadIdx.x)];
+    k_norm[tok0 + threadIdx.x] = reinterpret_cast<const __half*>(body + B_KNORM)[norm_pos(threadIdx.x)];
+    v_norm[tok0 + threadIdx.x] = reinterpret_cast<const __half*>(body + B_VNORM)[norm_pos(threadIdx.x)];
   }
   {
     int c = threadIdx.x, p = meta_pos(c);
     size_t o = ((unit * cv.n_windows() + win) * D + c) * 2;
-    k_meta[o] = reinterpret_cast<const __half*>(rec + OFF_KM)[p];
-    k_meta[o + 1] = reinterpret_cast<const __half*>(rec + OFF_KS)[p];
+    if (cv.fmt == FMT_FP16) {
+      k_meta[o] = reinterpret_cast<const __half*>(rec + OFF_KM)[p];
+      k_meta[o + 1] = reinterpret_cast<const __half*>(rec + OFF_KS)[p];
+    } else {   // decode the MXFP4 pair; every decoded value is an fp16 number
+      const unsigned mnib = (rec[p >> 1] >> (4 * (p & 1))) & 15u, snib = (rec[64 + (p >> 1)] >> (4 * (p & 1))) & 15u;
+      k_meta[o] = __float2half_rn(mx_decode(mnib, (int)rec[128 + (c >> 5)] - 127));
+      k_meta[o + 1] = __float2half_rn(mx_decode(snib, (int)rec[132 + (c >> 5)] - 127));
+      if (k_mx) {   // stored bytes in natural channel order: nibble of channel c in byte c/2
+        unsigned char* dst = k_mx + (unit * cv.n_windows() + win) * MX_META_BYTES;
+        __shared__ unsigned char nb[2 * D];
+        nb[c] = (unsigned char)mnib; nb[D + c] = (unsigned char)snib;
+        __syncthreads();
+        dst[c] = (unsigned char)(nb[2 * c] | (nb[2 * c + 1] << 4));
+        if (c < 8) dst[128 + c] = rec[128 + c];
+      }
+    }
   }
 }
 
 __global__ void k_import(CacheView cv, int layer, const unsigned char* k_codes, const __half* k_norm,
                          const __half* k_meta, const unsigned char* v_codes, const __half* v_norm) {
   int win = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  unsigned char* rec = cv.record(layer, b, h, win);
+  unsigned char* rec = cv.meta(layer, b, h, win);   // fp16 metadata only
   size_t unit = (size_t)b * cv.n_kv_heads + h;
   size_t tok0 = unit * cv.capacity + (size_t)win * W;
   __shared__ uint32_t kw[256], vw[256];
@@ -538,7 +583,21 @@ okq_status okq_cache_export(const okq_cache* cache, int32_t layer, uint8_t* k_co
   CacheView cv = make_view(cache);
   k_export<<<dim3(cv.capacity / W, cv.n_kv_heads, cv.batch), 128, 0, static_cast<cudaStream_t>(stream)>>>(
       cv, layer, k_codes, static_cast<__half*>(k_norm), static_cast<__half*>(k_meta), v_codes,
-      static_cast<__half*>(v_norm));
+      static_cast<__half*>(v_norm), nullptr);
+  return launch_status();
+}
+
+okq_status okq_cache_export_mx(const okq_cache* cache, int32_t layer, uint8_t* k_codes, void* k_norm, void* k_meta,
+                               uint8_t* k_mx, uint8_t* v_codes, void* v_norm, void* stream) {
+  okq_status st = check_cache(cache, true);
+  if (st != OKQ_OK) return st;
+  if (cache->meta_format != OKQ_META_MXFP4) return OKQ_ERR_UNSUPPORTED;
+  if (layer < 0 || layer >= cache->n_layers || !k_codes || !k_norm || !k_meta || !k_mx || !v_codes || !v_norm)
+    return OKQ_ERR_INVALID_ARG;
+  CacheView cv = make_view(cache);
+  k_export<<<dim3(cv.capacity / W, cv.n_kv_heads, cv.batch), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+      cv, layer, k_codes, static_cast<__half*>(k_norm), static_cast<__half*>(k_meta), v_codes,
+      static_cast<__half*>(v_norm), k_mx);
   return launch_status();
 }
 
@@ -546,6 +605,7 @@ okq_status okq_cache_import(const okq_cache* cache, int32_t layer, const uint8_t
                             const void* k_meta, const uint8_t* v_codes, const void* v_norm, void* stream) {
   okq_status st = check_cache(cache, true);
   if (st != OKQ_OK) return st;
+  if (cache->meta_format != OKQ_META_FP16) return OKQ_ERR_UNSUPPORTED;   // fp16 (m, s) need not lie on the MX grid
   if (layer < 0 || layer >= cache->n_layers || !k_codes || !k_norm || !k_meta || !v_codes || !v_norm)
     return OKQ_ERR_INVALID_ARG;
   CacheView cv = make_view(cache);

@@ -197,8 +197,8 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(CacheView cv, 
           n = n > 65504.0f ? 65504.0f : n;
           const __half nh16 = __float2half_rn(n);
           const float nf = __half2float(nh16);
-          unsigned char* rec = cv.record(layer, b, h, win0 + (r >> 5));
-          reinterpret_cast<__half*>(rec + OFF_VNORM)[norm_pos(r & 31)] = nh16;
+          unsigned char* body = cv.body(layer, b, h, win0 + (r >> 5));
+          reinterpret_cast<__half*>(body + B_VNORM)[norm_pos(r & 31)] = nh16;
           sm.inv[buf][r] = nf != 0.0f ? __fdiv_rn(1.0f, nf) : 0.0f;
         }
       }
@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(CacheView cv, 
               word |= ((src >> (2 * (8 + g))) & 3u) << (16 * e + 8 + 2 * j);   // channel 16*mu + 8 + g
             }
           }
-          reinterpret_cast<uint32_t*>(cv.record(layer, p_b, p_h, p_win0 + wq) + OFF_VCODE)[w8] = word;
+          reinterpret_cast<uint32_t*>(cv.body(layer, p_b, p_h, p_win0 + wq) + B_VCODE)[w8] = word;
         }
       }
     }

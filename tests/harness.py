@@ -21,11 +21,14 @@ def u16(t: torch.Tensor) -> np.ndarray:
 class Case:
     """One workload instantiated on the GPU (all layers) with per-layer inputs kept on the host."""
 
-    def __init__(self, w: WL.Workload, n_tokens=None, capacity=None, device="cuda", gen_device="cpu"):
+    def __init__(self, w: WL.Workload, n_tokens=None, capacity=None, device="cuda", gen_device="cpu",
+                 meta_format=0, bulk_values=False):
         self.w = w
+        self.meta_format = meta_format
         self.n = w.n_tokens if n_tokens is None else n_tokens
         cap = capacity if capacity is not None else ((self.n + W - 1) // W + 2) * W
-        self.cache = B.Cache(w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, cap, device=device)
+        self.cache = B.Cache(w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, cap, device=device,
+                             meta_format=meta_format)
         self.mod = WL.modality_layout(w, self.n)                           # [n]
         self.mod_b = self.mod.unsqueeze(0).repeat(w.batch, 1).contiguous()  # [B, n]
         self.signs = torch.stack([WL.gen_signs(w, l) for l in range(w.n_layers)])      # [L,128]
@@ -40,7 +43,7 @@ class Case:
             k, v = WL.gen_kv(w, l, device=gen_device, n_tokens=self.n)
             self.k.append(k.cpu()); self.v.append(v.cpu())
             B.quantize_keys(self.cache, l, k.to(device), self.d_signs[l])
-            B.quantize_values(self.cache, l, v.to(device), self.d_mod, self.d_R[l])
+            B.quantize_values(self.cache, l, v.to(device), self.d_mod, self.d_R[l], bulk=bulk_values)
         torch.cuda.synchronize()
 
     # ---- oracle side
@@ -51,7 +54,7 @@ class Case:
         vb = u16(self.v[layer]).reshape(U, self.n, D)
         unit_seq = np.repeat(np.arange(w.batch), w.n_kv_heads)
         kq, vq, _ = O.quantize_batch(kb, vb, self.mod_b.numpy(), self.signs[layer].numpy(), self.R[layer].numpy(),
-                                     unit_seq=unit_seq)
+                                     unit_seq=unit_seq, meta_format=self.meta_format)
         return kq, vq, kb, vb
 
     def oracle_attention(self, layer, path=1, extra_k=None, extra_v=None):
@@ -101,6 +104,9 @@ def compare_cache(case: Case, layer: int, exp: dict, kq: dict, vq: dict):
     assert (kc == kq["codes"]).all(), f"key codes differ: {(kc != kq['codes']).sum()} bytes"
     assert (vn == vq["norm"]).all(), "value norms differ"
     assert (vc == vq["codes"]).all(), f"value codes differ: {(vc != vq['codes']).sum()} bytes"
+    if "mx" in kq:   # stored MXFP4 metadata bytes
+        mx = g["k_mx"].numpy().reshape(U, cap // W, 136)[:, :npk // W]
+        assert (mx == kq["mx"]).all(), f"stored MXFP4 metadata differs at {np.argwhere(mx != kq['mx'])[:4]}"
 
 
 def attention_errors(got: np.ndarray, ref: np.ndarray):
