@@ -322,22 +322,24 @@ __global__ void __launch_bounds__(128) k_quantize_values(CacheView cv, int layer
 // raw tail copy + seq_len (+ modality for the value call); grid (n_kv_heads, batch), 128 threads
 __global__ void k_bulk_tail(CacheView cv, int layer, const __half* __restrict__ src, long long sb, long long sh,
                             long long st, int n_tokens, __half* tail, const unsigned char* __restrict__ modality) {
-  int h = blockIdx.x, b = blockIdx.y;
-  int n_packed = n_tokens & ~(W - 1);
-  int n_tail = n_tokens - n_packed;
-  __half* dst = tail + cv.tail_off(layer, b, h);
-  for (int idx = threadIdx.x; idx < n_tail * (D / 8); idx += blockDim.x) {
-    int i = idx / (D / 8), c8 = idx % (D / 8);
-    reinterpret_cast<uint4*>(dst + i * D)[c8] =
-        *reinterpret_cast<const uint4*>(src + b * sb + h * sh + (long long)(n_packed + i) * st + c8 * 8);
+  const int h = blockIdx.x, b = blockIdx.y;
+  if (blockIdx.z == 0) {
+    const int n_packed = n_tokens & ~(W - 1);
+    const int n_tail = n_tokens - n_packed;
+    __half* dst = tail + cv.tail_off(layer, b, h);
+    for (int idx = threadIdx.x; idx < n_tail * (D / 8); idx += blockDim.x) {
+      int i = idx / (D / 8), c8 = idx % (D / 8);
+      reinterpret_cast<uint4*>(dst + i * D)[c8] =
+          *reinterpret_cast<const uint4*>(src + b * sb + h * sh + (long long)(n_packed + i) * st + c8 * 8);
+    }
+    if (h == 0 && threadIdx.x == 0) cv.seq_len[layer * cv.batch + b] = n_tokens;
   }
-  if (h == 0) {
-    if (threadIdx.x == 0) cv.seq_len[layer * cv.batch + b] = n_tokens;
-    if (modality)
-      for (int i = threadIdx.x; i < n_tokens; i += blockDim.x) {
-        unsigned char m = modality[(size_t)b * n_tokens + i];
-        cv.modality[(size_t)b * cv.capacity + i] = m > 2 ? 0 : m;
-      }
+  if (modality) {   // the sequence's modality bytes, spread over the (head, slice) blocks of the sequence
+    const int stride = gridDim.x * gridDim.z * blockDim.x;
+    for (int i = (h * gridDim.z + blockIdx.z) * blockDim.x + threadIdx.x; i < n_tokens; i += stride) {
+      const unsigned char m = modality[(size_t)b * n_tokens + i];
+      cv.modality[(size_t)b * cv.capacity + i] = m > 2 ? 0 : m;
+    }
   }
 }
 
@@ -480,6 +482,8 @@ okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __hal
                                      const unsigned char* modality, int n_tokens, const float* R, int n_R,
                                      int n_sm, cudaStream_t s);
 
+constexpr int TAIL_SLICES = 16;   // blocks per (sequence, head) that share the copy of the modality bytes
+
 static okq_status check_bulk(const okq_cache* c, int32_t layer, const void* x, const int64_t strides[3],
                              int32_t n_tokens) {
   okq_status st = check_cache(c, true);
@@ -533,8 +537,8 @@ okq_status okq_quantize_values(const okq_cache* cache, int32_t layer, const void
     k_quantize_values<<<grid, 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2], modality, n_tokens, R,
                                            n_R);
   }
-  k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
-                                                           n_tokens, cv.v_tail, n_tokens > 0 ? modality : nullptr);
+  k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch, TAIL_SLICES), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
+                                                                        n_tokens, cv.v_tail, n_tokens > 0 ? modality : nullptr);
   return launch_status();
 }
 
@@ -551,8 +555,8 @@ okq_status okq_quantize_values_bulk(const okq_cache* cache, int32_t layer, const
   const __half* v = static_cast<const __half*>(v_fp16);
   st = launch_quantize_values_tc(cv, layer, v, strides, modality, n_tokens, R, n_R, sm_count(), s);
   if (st != OKQ_OK) return st;
-  k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
-                                                           n_tokens, cv.v_tail, n_tokens > 0 ? modality : nullptr);
+  k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch, TAIL_SLICES), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
+                                                                        n_tokens, cv.v_tail, n_tokens > 0 ? modality : nullptr);
   return launch_status();
 }
 
