@@ -37,6 +37,7 @@ BYTES_PER_TOKEN_HEAD = 84          # 32 B key codes + 2 B key norm + 16 B (m, s)
 # 4-layer slice of the workload (176 MB of records, larger than L2) and divided by its token-heads;
 # traffic grows in proportion to the token-heads (profiles/decode_mma_layers4_ncu_full.md).
 NCU_DRAM_BYTES_PER_TOKEN_HEAD = 86.99
+NCU_DRAM_BYTES_PER_TOKEN_HEAD_MX = 75.30   # same capture with --meta mxfp4
 
 
 def measured_peaks():
@@ -213,7 +214,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling on a small case)")
     ap.add_argument("--meta", default="fp16", choices=["fp16", "mxfp4"],
                     help="(m, s) metadata format of the cache: fp16 = 84 B per token and KV head (the headline "
-                         "configuration), mxfp4 = 72.25 B (secondary measurement; no cpu_baseline, no ncu traffic)")
+                         "configuration), mxfp4 = 72.25 B (secondary measurement; no cpu_baseline)")
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
                     help="decode: the headline decode step; prefill: bulk quantisation of a fresh fp16 K/V cache "
                          "(secondary measurement, default workload prefill7b)")
@@ -324,7 +325,7 @@ def main():
     e2e_value = world * packed_bytes / (ms_e2e / args.steps * 1e-3) / 1e9
     peak, peak_kind = measured_peaks()
     achieved = packed_bytes / (kernel_ms * 1e-3) / 1e9
-    traffic = None if NCU_DRAM_BYTES_PER_TOKEN_HEAD is None or mx else NCU_DRAM_BYTES_PER_TOKEN_HEAD * L * Bn * H * N
+    traffic = (NCU_DRAM_BYTES_PER_TOKEN_HEAD_MX if mx else NCU_DRAM_BYTES_PER_TOKEN_HEAD) * L * Bn * H * N
 
     if rank != 0:
         return

@@ -43,11 +43,12 @@ def test_long_context_batch1():
     Hn.assert_attention_close(got4, ref)
 
 
-def test_full_7b_step_sampled():
+@pytest.mark.parametrize("meta_format", [B.META_FP16, B.META_MXFP4])
+def test_full_7b_step_sampled(meta_format):
     w = WL.WORKLOADS["step7b"]
     dev = torch.device("cuda")
     L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
-    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev)
+    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev, meta_format=meta_format)
     mod_cpu = WL.modality_layout(w)
     mod = mod_cpu.unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
     signs = torch.stack([WL.gen_signs(w, l) for l in range(L)])
@@ -84,13 +85,15 @@ def test_full_7b_step_sampled():
     for (sl, sb) in samples:
         kc, vc = kept[(sl, sb)]
         kb = Hn.u16(kc).reshape(H, N, D); vb = Hn.u16(vc).reshape(H, N, D)
-        kq, vq, _ = O.quantize_batch(kb, vb, mod_cpu.numpy(), signs[sl].numpy(), R[sl].numpy())
+        kq, vq, _ = O.quantize_batch(kb, vb, mod_cpu.numpy(), signs[sl].numpy(), R[sl].numpy(), meta_format=meta_format)
         e = B.cache_export(cache, sl)
         torch.cuda.synchronize()
         cap = cache.capacity
         assert (e["k_codes"][sb].cpu().numpy()[:, :N] == kq["codes"]).all()
         assert (Hn.u16(e["k_norm"][sb])[:, :N] == kq["norm"]).all()
         assert (Hn.u16(e["k_meta"][sb])[:, :N // W] == kq["meta"]).all()
+        if meta_format == B.META_MXFP4:
+            assert (e["k_mx"][sb].cpu().numpy()[:, :N // W] == kq["mx"]).all()
         assert (e["v_codes"][sb].cpu().numpy()[:, :N] == vq["codes"]).all()
         assert (Hn.u16(e["v_norm"][sb])[:, :N] == vq["norm"]).all()
         del e
@@ -100,7 +103,7 @@ def test_full_7b_step_sampled():
         modrow = np.concatenate([mod_cpu.numpy(), np.zeros(1, np.uint8)])
         ref, _ = O.attention(1, qs, kq, vq, modrow, kt, vt, signs[sl].numpy(), R[sl].numpy())
         errs = Hn.assert_attention_close(o[sl, sb], ref.reshape(Hq, D))
-        print(f"full step7b layer {sl} seq {sb}: rel-L2 {errs[0]:.2e} worst head {errs[1]:.2e} max-abs {errs[2]:.2e}")
+        print(f"full step7b (meta format {meta_format}) layer {sl} seq {sb}: rel-L2 {errs[0]:.2e} worst head {errs[1]:.2e} max-abs {errs[2]:.2e}")
 
 
 def test_ragged_batch_lengths():
