@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(128) k_decode_simt(DecodeParams P) {
 #pragma unroll
       for (int k = 0; k < 4; k++) {
         int p = 4 * lane + k;
-        float mf = __half2float(mp[p]), sf = __half2float(sp[p]);
+        float mf = __half2float(mp[p]) * (1.0f / (float)(1 << (2 * meta_shift_pos(p)))), sf = __half2float(sp[p]);
         float wv[GP];
 #pragma unroll
         for (int j = 0; j < GP; j++) {

@@ -173,7 +173,7 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
       }
       const uint4* mp = reinterpret_cast<const uint4*>(st + OFF_KM + 64 * t);
       const uint4* sp = reinterpret_cast<const uint4*>(st + OFF_KS + 64 * t);
-      // bias sum_c q'_c m_c (against the constant operand 4^j 2^-24, two independent chains)
+      // bias sum_c q'_c m_c (two independent chains)
       // and scores sum_c q'_c s_c code_c, one k-step (16 channels) at a time
       float dbA[4] = {0.f, 0.f, 0.f, 0.f}, dbB[4] = {0.f, 0.f, 0.f, 0.f};
       float d[4][4];
@@ -192,10 +192,10 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
           const int kappa = 2 * kq + half;
           const uint2 q0 = qreg[2 * kappa], q1 = qreg[2 * kappa + 1];
           uint32_t a0, a1, a2, a3;
-          split_product(u2h(q0.x), u2h(q0.y), u2h(half ? m4.z : m4.x), a0, a1);
-          split_product(u2h(q1.x), u2h(q1.y), u2h(half ? m4.w : m4.y), a2, a3);
-          if (half) mma16816(dbB, a0, a1, a2, a3, 0x00100010u, 0x00400040u);
-          else mma16816(dbA, a0, a1, a2, a3, 0x00010001u, 0x00040004u);
+          // bias: the stored m * 4^j is the B operand as it is (every column the same), the query fragments
+          // (hi rows, lo rows) the A operand
+          if (half) mma16816(dbB, q0.x, q0.y, q1.x, q1.y, m4.z, m4.w);
+          else mma16816(dbA, q0.x, q0.y, q1.x, q1.y, m4.x, m4.y);
           split_product(u2h(q0.x), u2h(q0.y), u2h(half ? s4.z : s4.x), a0, a1);
           split_product(u2h(q1.x), u2h(q1.y), u2h(half ? s4.w : s4.y), a2, a3);
           const int ww = kappa >> 2, sh = (kappa >> 1) & 1;
@@ -212,7 +212,8 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
       const uint4 kn4 = *reinterpret_cast<const uint4*>(st + OFF_KNORM + 16 * t);
       const uint4 vn4 = *reinterpret_cast<const uint4*>(st + OFF_VNORM + 16 * t);
       const uint32_t knu[4] = {kn4.x, kn4.y, kn4.z, kn4.w}, vnu[4] = {vn4.x, vn4.y, vn4.z, vn4.w};
-      const float bias0 = (dbA[0] + dbB[0]) + (dbA[2] + dbB[2]), bias1 = (dbA[1] + dbB[1]) + (dbA[3] + dbB[3]);
+      // the code sums carry 2^-24 (subnormal code operands), the bias sum does not
+      const float bias0 = ((dbA[0] + dbB[0]) + (dbA[2] + dbB[2])) * 0x1p-24f, bias1 = bias0;
       float sc[4][2];
       float mx = -INFINITY;
 #pragma unroll

@@ -87,8 +87,8 @@ __device__ __forceinline__ uint32_t pow2_half2(int k) {
   return h | (h << 16);
 }
 
-// Decoded (m, s) of record positions 4*lane .. 4*lane+3 from the 136 MXFP4 metadata bytes
-// (global or shared, 2-byte aligned): four fp16 each, exact.
+// Decoded (m * 4^j, s) of record positions 4*lane .. 4*lane+3 from the 136 MXFP4 metadata bytes
+// (global or shared, 2-byte aligned): four fp16 each, exact; m with the position scale of the fp16 layout.
 __device__ __forceinline__ void mx_decode_lane(const unsigned char* meta, int lane, uint2& m4, uint2& s4) {
   const uint32_t xm = *reinterpret_cast<const unsigned short*>(meta + 2 * lane);
   const uint32_t xs = *reinterpret_cast<const unsigned short*>(meta + 64 + 2 * lane);
@@ -98,6 +98,11 @@ __device__ __forceinline__ void mx_decode_lane(const unsigned char* meta, int la
   e2m1x4_to_half2(xm, a, b);
   __half2 r0 = __hmul2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<const __half2*>(&pm));
   __half2 r1 = __hmul2(*reinterpret_cast<__half2*>(&b), *reinterpret_cast<const __half2*>(&pm));
+  // the staged m plane carries the position scale 4^j: positions 4*lane + {0,1} have j = 2*(lane & 1), the
+  // other two j + 1 (a second exact multiply: 2^k * 4^j alone may leave the fp16 range)
+  const uint32_t q0 = pow2_half2(4 * (lane & 1)), q1 = pow2_half2(4 * (lane & 1) + 2);
+  r0 = __hmul2(r0, *reinterpret_cast<const __half2*>(&q0));
+  r1 = __hmul2(r1, *reinterpret_cast<const __half2*>(&q1));
   m4 = make_uint2(*reinterpret_cast<uint32_t*>(&r0), *reinterpret_cast<uint32_t*>(&r1));
   e2m1x4_to_half2(xs, a, b);
   r0 = __hmul2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<const __half2*>(&ps));

@@ -17,7 +17,7 @@
 //  * The 32 key norms (and value norms) are stored in the order norm_pos(i), which puts the
 //    eight tokens whose scores a lane receives next to each other.
 //  * (m, s) are stored as two planes of 128 fp16 in the order pi(c) that makes each
-//    lane's 32 channels contiguous.
+//    lane's 32 channels contiguous; the m plane is pre-multiplied by a power of four (meta_shift).
 #pragma once
 #include <cstdint>
 #include <cuda_fp16.h>
@@ -41,6 +41,12 @@ __host__ __device__ inline int meta_pos(int c) {
   int pair = slot >> 3, t = (slot & 7) >> 1, e = slot & 1;
   return t * 32 + kappa * 4 + pair * 2 + e;
 }
+
+// The m plane holds m_c * 4^j(c), j = (2*kappa + pair) & 3 (exact in fp16: |m| <= 1): 4^j is the position
+// scale of the matching key-code field, which the decode kernel's query fragments are pre-divided by, so the
+// stored value is the tensor-core operand of the bias sum as it is.  log4 of the factor, by channel / position:
+__host__ __device__ inline int meta_shift(int c) { return (2 * (c >> 4) + ((c >> 3) & 1)) & 3; }
+__host__ __device__ inline int meta_shift_pos(int p) { return (2 * ((p >> 2) & 7) + ((p >> 1) & 1)) & 3; }
 
 // position of token i inside the key-norm / value-norm arrays: the four lanes of a quad each
 // find the norms of "their" tokens {8*nu + 2*t + e} in 16 contiguous bytes

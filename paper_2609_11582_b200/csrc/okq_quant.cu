@@ -134,7 +134,7 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
       sm.a[c] = mf;
       sm.b[c] = sf > 0.0f ? __fdiv_rn(1.0f, sf) : 0.0f;
       int p = meta_pos(c);
-      reinterpret_cast<__half*>(rec + OFF_KM)[p] = mh;
+      reinterpret_cast<__half*>(rec + OFF_KM)[p] = __float2half_rn(mf * (float)(1 << (2 * meta_shift(c))));   // exact
       reinterpret_cast<__half*>(rec + OFF_KS)[p] = sh;
     } else {
       // MXFP4: a warp is one block of 32 consecutive channels.  m rounds down, s rounds up.
@@ -423,7 +423,8 @@ __global__ void k_export(CacheView cv, int layer, unsigned char* k_codes, __half
     int c = threadIdx.x, p = meta_pos(c);
     size_t o = ((unit * cv.n_windows() + win) * D + c) * 2;
     if (cv.fmt == FMT_FP16) {
-      k_meta[o] = reinterpret_cast<const __half*>(rec + OFF_KM)[p];
+      k_meta[o] = __float2half_rn(__half2float(reinterpret_cast<const __half*>(rec + OFF_KM)[p]) /
+                                  (float)(1 << (2 * meta_shift(c))));   // exact
       k_meta[o + 1] = reinterpret_cast<const __half*>(rec + OFF_KS)[p];
     } else {   // decode the MXFP4 pair; every decoded value is an fp16 number
       const unsigned mnib = (rec[p >> 1] >> (4 * (p & 1))) & 15u, snib = (rec[64 + (p >> 1)] >> (4 * (p & 1))) & 15u;
@@ -473,7 +474,7 @@ __global__ void k_import(CacheView cv, int layer, const unsigned char* k_codes, 
   {
     int c = threadIdx.x, p = meta_pos(c);
     size_t o = ((unit * cv.n_windows() + win) * D + c) * 2;
-    reinterpret_cast<__half*>(rec + OFF_KM)[p] = k_meta[o];
+    reinterpret_cast<__half*>(rec + OFF_KM)[p] = __float2half_rn(__half2float(k_meta[o]) * (float)(1 << (2 * meta_shift(c))));
     reinterpret_cast<__half*>(rec + OFF_KS)[p] = k_meta[o + 1];
   }
 }
