@@ -202,6 +202,47 @@ def run_prefill(args, w, B, dev, rank):
         print(json.dumps(line), flush=True)
 
 
+def run_calib(args, B, dev, rank):
+    """Secondary measurement: the offline calibration of the value rotations of one (layer, KV head) on a
+    synthetic calibration sequence of 8192 tokens (7 query heads): attention weights, weighted moments, three
+    eigen-decompositions.  One JSON line."""
+    n, G = 8192, 7
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=1, n_tokens=n)
+    k, v = WL.gen_kv(w, 0, device=dev, n_tokens=n)
+    k, v = k[0, 0].contiguous(), v[0, 0].contiguous()
+    q = torch.randn(G, n, 128, generator=torch.Generator(device=dev).manual_seed(7), device=dev).to(torch.float16)
+    mod = WL.modality_layout(w, n).to(dev)
+    signs = WL.gen_signs(w, 0).to(dev)
+    ws = B.calib_workspace(G, n, device=dev)
+
+    def timed(fn):
+        for _ in range(args.warmup):
+            fn()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in ev:
+            a.record(); fn(); b.record()
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in ev) / args.steps
+
+    wts = B.calib_attention_weights(q, k, ws)
+    Cm = B.calib_moments(v, wts, mod, ws)
+    ms_w = timed(lambda: B.calib_attention_weights(q, k, ws))
+    ms_c = timed(lambda: B.calib_moments(v, wts, mod, ws))
+    ms_r = timed(lambda: [B.calib_rotation(Cm[m].contiguous(), signs, ws) for m in range(3)])
+    peak, peak_kind = measured_peaks()
+    # causal scores, computed in both passes: 2 passes x G x n (n + 64) / 2 x 128 multiply-adds (64-key tiles)
+    flops_w = 2.0 * 2 * G * n * (n + 64) / 2 * 128
+    line = {"metric": "calibration of the value rotations: ms per (layer, KV head)", "phase": "calib",
+            "value": ms_w + ms_c + ms_r, "unit": "ms", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "higher_is_better": False, "dtype": "f16-mma/f32/f64", "data": "synthetic",
+            "config": {"workload": "calibration sequence", "tokens": n, "group": G},
+            "attention_weights_ms": ms_w, "attention_weights_tflops": flops_w / (ms_w * 1e-3) / 1e12,
+            "moments_ms": ms_c, "rotations_ms": ms_r}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -215,9 +256,10 @@ def main():
     ap.add_argument("--meta", default="fp16", choices=["fp16", "mxfp4"],
                     help="(m, s) metadata format of the cache: fp16 = 84 B per token and KV head (the headline "
                          "configuration), mxfp4 = 72.25 B (secondary measurement; no cpu_baseline)")
-    ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
+    ap.add_argument("--phase", default="decode", choices=["decode", "prefill", "calib"],
                     help="decode: the headline decode step; prefill: bulk quantisation of a fresh fp16 K/V cache "
-                         "(secondary measurement, default workload prefill7b)")
+                         "(secondary measurement, default workload prefill7b); calib: offline calibration of the "
+                         "value rotations (secondary measurement)")
     args = ap.parse_args()
     if args.workload is None:
         args.workload = "prefill7b" if args.phase == "prefill" else "step7b"
@@ -237,6 +279,8 @@ def main():
 
     if args.phase == "prefill":
         return run_prefill(args, w, B, dev, rank)
+    if args.phase == "calib":
+        return run_calib(args, B, dev, rank)
 
     # ---- build the packed cache on the device (setup, untimed)
     L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens

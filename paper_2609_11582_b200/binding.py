@@ -80,6 +80,17 @@ def lib():
         L.okq_cache_export.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 6
         L.okq_cache_export_mx.restype = C.c_int
         L.okq_cache_export_mx.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 7
+        L.okq_calib_workspace_bytes.restype = C.c_size_t
+        L.okq_calib_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
+        L.okq_calib_attention_weights.restype = C.c_int
+        L.okq_calib_attention_weights.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_int32,
+                                                  C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.okq_calib_moments.restype = C.c_int
+        L.okq_calib_moments.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t,
+                                        C.c_void_p, C.c_void_p]
+        L.okq_calib_rotation.restype = C.c_int
+        L.okq_calib_rotation.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_void_p]
         L.okq_cache_import.restype = C.c_int
         L.okq_cache_import.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 6
         _lib = L
@@ -90,7 +101,8 @@ def exported_symbols():
     return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
             "okq_cache_import", "okq_profile_events", "okq_decode_attention_simt",
-            "okq_decode_attention_noalloc", "okq_quantize_values_bulk", "okq_cache_export_mx"]
+            "okq_decode_attention_noalloc", "okq_quantize_values_bulk", "okq_cache_export_mx",
+            "okq_calib_workspace_bytes", "okq_calib_attention_weights", "okq_calib_moments", "okq_calib_rotation"]
 
 
 def _ptr(t) -> int:
@@ -229,3 +241,40 @@ def cache_import(cache: Cache, layer: int, arrays: dict, stream=None):
     a = {k: v.contiguous() for k, v in arrays.items()}
     _check(lib().okq_cache_import(C.byref(cache.c), layer, _ptr(a["k_codes"]), _ptr(a["k_norm"]), _ptr(a["k_meta"]),
                                   _ptr(a["v_codes"]), _ptr(a["v_norm"]), _stream(stream)), "okq_cache_import")
+
+
+# ---- offline calibration of the value rotations (okq_calib.h)
+
+def calib_workspace(group: int, n: int, device="cuda") -> torch.Tensor:
+    return torch.empty(lib().okq_calib_workspace_bytes(group, n), dtype=torch.uint8, device=device)
+
+
+def calib_attention_weights(q, k, workspace, sm_scale=None, causal=True, stream=None):
+    """q: fp16 [group, n, 128], k: fp16 [n, 128] (contiguous) -> w float32 [n]."""
+    assert q.dtype == torch.float16 and k.dtype == torch.float16 and q.is_contiguous() and k.is_contiguous()
+    group, n = q.shape[0], q.shape[1]
+    w = torch.empty(n, dtype=torch.float32, device=q.device)
+    scale = HEAD_DIM ** -0.5 if sm_scale is None else sm_scale
+    _check(lib().okq_calib_attention_weights(_ptr(q), _ptr(k), group, n, scale, 1 if causal else 0, _ptr(workspace),
+                                             workspace.numel(), _ptr(w), _stream(stream)), "okq_calib_attention_weights")
+    return w
+
+
+def calib_moments(v, w, modality, workspace, stream=None):
+    """v: fp16 [n, 128], w: float32 [n], modality: uint8 [n] -> C float32 [3, 128, 128]."""
+    assert v.dtype == torch.float16 and v.is_contiguous() and w.dtype == torch.float32 and modality.dtype == torch.uint8
+    Cm = torch.empty(3, HEAD_DIM, HEAD_DIM, dtype=torch.float32, device=v.device)
+    _check(lib().okq_calib_moments(_ptr(v), _ptr(w), _ptr(modality), v.shape[0], _ptr(workspace), workspace.numel(),
+                                   _ptr(Cm), _stream(stream)), "okq_calib_moments")
+    return Cm
+
+
+def calib_rotation(Cm, signs, workspace, stream=None):
+    """Cm: float32 [128, 128] symmetric, signs: float32 [128] -> (R float32 [128, 128], eigenvalues [128], sweeps)."""
+    assert Cm.dtype == torch.float32 and Cm.is_contiguous() and signs.dtype == torch.float32
+    R = torch.empty(HEAD_DIM, HEAD_DIM, dtype=torch.float32, device=Cm.device)
+    lam = torch.empty(HEAD_DIM, dtype=torch.float32, device=Cm.device)
+    sweeps = torch.zeros(1, dtype=torch.int32, device=Cm.device)
+    _check(lib().okq_calib_rotation(_ptr(Cm), _ptr(signs), _ptr(workspace), workspace.numel(), _ptr(R), _ptr(lam),
+                                    _ptr(sweeps), _stream(stream)), "okq_calib_rotation")
+    return R, lam, sweeps

@@ -19,9 +19,11 @@ def L():
 
 
 def test_every_declared_symbol_is_exported(L):
-    hdr = open(os.path.join(ROOT, "include", "okq.h")).read()
-    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    declared = set(re.findall(r"\b(okq_[a-z_]+)\s*\(", hdr))
+    declared = set()
+    for name in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        hdr = open(os.path.join(ROOT, "include", name)).read()
+        hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+        declared |= set(re.findall(r"\b(okq_[a-z_]+)\s*\(", hdr))
     assert declared == set(B.exported_symbols())
     for s in declared:
         assert hasattr(L, s), s
@@ -78,3 +80,18 @@ def test_pointer_validation_before_any_launch(L):
     assert L.okq_decode_workspace_bytes(C.byref(c), 0, 3) == 0
     c8 = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, fake + 8, fake, fake, fake, fake, fake)
     assert L.okq_append(C.byref(c8), 0, 1, fake, fake, fake, fake, fake, 1, None) == B.ERR_ALIGNMENT
+
+
+def test_calibration_argument_checks(L):
+    assert L.okq_calib_workspace_bytes(0, 16) == 0 and L.okq_calib_workspace_bytes(7, 0) == 0
+    # the largest of: row statistics + per-(query tile, head) column sums; 64 partial moment sets; 128 x 128 fp64
+    assert L.okq_calib_workspace_bytes(7, 4096) >= max((7 * 4096 * 2 + 64 * 7 * 4096) * 4, 64 * 3 * 128 * 128 * 4, 128 * 128 * 8)
+    assert L.okq_calib_workspace_bytes(1, 8) >= 64 * 3 * 128 * 128 * 4
+    null = C.c_void_p(0)
+    assert L.okq_calib_attention_weights(null, null, 7, 64, C.c_float(1.0), 1, null, 0, null, null) == B.ERR_INVALID_ARG
+    assert L.okq_calib_moments(null, null, null, 64, null, 0, null, null) == B.ERR_INVALID_ARG
+    assert L.okq_calib_rotation(null, null, null, 0, null, null, null, null) == B.ERR_INVALID_ARG
+    fake = C.c_void_p(4096)      # aligned, never dereferenced: the size checks come first
+    assert L.okq_calib_attention_weights(fake, fake, 7, 64, C.c_float(1.0), 1, fake, 16, fake, null) == B.ERR_WORKSPACE
+    assert L.okq_calib_attention_weights(C.c_void_p(4100), fake, 7, 64, C.c_float(1.0), 1, fake, 1 << 30, fake, null) == B.ERR_ALIGNMENT
+    assert L.okq_calib_rotation(fake, fake, fake, 1024, fake, fake, null, null) == B.ERR_WORKSPACE
