@@ -158,6 +158,7 @@ def quantize_values(v_bits: np.ndarray, modality: np.ndarray, R: np.ndarray):
     npk = (n // W) * W
     codes = np.zeros((npk, D // 4), np.uint8)
     norm = np.zeros(npk, np.uint16)
+    assert np.asarray(modality).max(initial=0) <= 2, "modality ids are 0 text, 1 audio, 2 video"
     r = lib().okqo_quantize_values(_p(v_bits), C.c_int64(n), _p(_c(modality, np.uint8)), _p(_c(R, np.float32)),
                                    _p(codes), _p(norm))
     assert r == npk
@@ -199,6 +200,7 @@ def attention(path: int, q_bits, kq, vq, modality, k_tail, v_tail, signs, R, sm_
     npk = kc.shape[1]
     assert kc.shape == (U, npk, 32) and vc.shape == (U, npk, 32)
     modality = _c(modality, np.uint8)
+    assert modality.max(initial=0) <= 2, "modality ids are 0 text, 1 audio, 2 video"
     if modality.ndim == 1:
         modality = modality[None]
     k_tail = _c(k_tail, np.uint16); v_tail = _c(v_tail, np.uint16)
@@ -227,6 +229,7 @@ def quantize_batch(k_bits, v_bits, modality, signs, R, unit_seq=None, unit_rot=N
     U, n, _ = k_bits.shape
     npk = (n // W) * W
     modality = _c(modality, np.uint8)
+    assert modality.max(initial=0) <= 2, "modality ids are 0 text, 1 audio, 2 video"
     if modality.ndim == 1:
         modality = modality[None]
     signs = _c(signs, np.float32).reshape(-1, D)

@@ -22,15 +22,17 @@ class Case:
     """One workload instantiated on the GPU (all layers) with per-layer inputs kept on the host."""
 
     def __init__(self, w: WL.Workload, n_tokens=None, capacity=None, device="cuda", gen_device="cpu",
-                 meta_format=0, bulk_values=False):
+                 meta_format=0, bulk_values=False, modality=None):
         self.w = w
         self.meta_format = meta_format
         self.n = w.n_tokens if n_tokens is None else n_tokens
         cap = capacity if capacity is not None else ((self.n + W - 1) // W + 2) * W
         self.cache = B.Cache(w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, cap, device=device,
                              meta_format=meta_format)
-        self.mod = WL.modality_layout(w, self.n)                           # [n]
-        self.mod_b = self.mod.unsqueeze(0).repeat(w.batch, 1).contiguous()  # [B, n]
+        self.mod = WL.modality_layout(w, self.n) if modality is None else modality   # [n]
+        self.mod_b = self.mod.unsqueeze(0).repeat(w.batch, 1).contiguous()  # [B, n], as the caller passes it
+        # the oracle takes ids in {0, 1, 2}: ids > 2 count as text
+        self.mod_o = torch.where(self.mod_b > 2, torch.zeros_like(self.mod_b), self.mod_b).numpy()
         self.signs = torch.stack([WL.gen_signs(w, l) for l in range(w.n_layers)])      # [L,128]
         self.R = torch.stack([WL.gen_rotations(w, l) for l in range(w.n_layers)])      # [L,3,128,128]
         self.q = torch.stack([WL.gen_queries(w, l) for l in range(w.n_layers)])        # [L,B,Hq,128]
@@ -53,7 +55,7 @@ class Case:
         kb = u16(self.k[layer]).reshape(U, self.n, D)
         vb = u16(self.v[layer]).reshape(U, self.n, D)
         unit_seq = np.repeat(np.arange(w.batch), w.n_kv_heads)
-        kq, vq, _ = O.quantize_batch(kb, vb, self.mod_b.numpy(), self.signs[layer].numpy(), self.R[layer].numpy(),
+        kq, vq, _ = O.quantize_batch(kb, vb, self.mod_o, self.signs[layer].numpy(), self.R[layer].numpy(),
                                      unit_seq=unit_seq, meta_format=self.meta_format)
         return kq, vq, kb, vb
 
@@ -66,7 +68,7 @@ class Case:
         G = w.group
         q = u16(self.q[layer]).reshape(w.batch, w.n_kv_heads, G, D).reshape(U, G, D)
         unit_seq = np.repeat(np.arange(w.batch), w.n_kv_heads)
-        out, th = O.attention(path, q, kq, vq, self.mod_b.numpy(), kb[:, npk:], vb[:, npk:], self.signs[layer].numpy(),
+        out, th = O.attention(path, q, kq, vq, self.mod_o, kb[:, npk:], vb[:, npk:], self.signs[layer].numpy(),
                               self.R[layer].numpy(), unit_seq=unit_seq)
         return out.reshape(w.batch, w.n_q_heads, D), th
 

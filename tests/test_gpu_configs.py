@@ -106,6 +106,32 @@ def test_full_7b_step_sampled(meta_format):
         print(f"full step7b (meta format {meta_format}) layer {sl} seq {sb}: rel-L2 {errs[0]:.2e} worst head {errs[1]:.2e} max-abs {errs[2]:.2e}")
 
 
+@pytest.mark.parametrize("meta_format", [B.META_FP16, B.META_MXFP4])
+def test_every_window_holds_all_three_modalities(meta_format):
+    """Worst case for the per-modality bookkeeping: modality ids drawn per token, so every 32-token window
+    (and every 128-token tile of the bulk value quantiser) mixes text, audio and video; a few ids > 2, which
+    count as text."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=2)
+    n = 1024 + 13
+    g = torch.Generator().manual_seed(99)
+    mod = torch.randint(0, 3, (n,), generator=g, dtype=torch.uint8)
+    mod[::97] = 7
+    c = Hn.Case(w, n_tokens=n, meta_format=meta_format, modality=mod)
+    kq, vq, _, _ = c.oracle_quantize(0)
+    Hn.compare_cache(c, 0, c.gpu_export(0), kq, vq)
+    assert (c.cache.modality.view(w.batch, -1)[:, :n].cpu() == torch.where(mod > 2, torch.zeros_like(mod), mod)).all()
+    ref, _ = c.oracle_attention(0)
+    print("mixed windows:", Hn.assert_attention_close(c.gpu_decode(0)[0], ref))
+    Hn.assert_attention_close(c.gpu_decode(0, simt=True)[0], ref)
+    # the tensor-core value quantiser on the same input: two jobs per tile (three modalities, two accumulators)
+    b = Hn.Case(w, n_tokens=n, meta_format=meta_format, modality=mod, bulk_values=True)
+    ea, eb = c.gpu_export(0), b.gpu_export(0)
+    assert b.cache.device_status() == 0
+    assert torch.equal(ea["v_norm"], eb["v_norm"])
+    assert (ea["v_codes"] != eb["v_codes"]).sum().item() <= 8      # only coordinates that sit on a threshold may differ
+    Hn.assert_attention_close(b.gpu_decode(0)[0], ref)
+
+
 def test_ragged_batch_lengths():
     """Sequences of different lengths in one decode call (lengths set per sequence, tails filled to match):
     the persistent kernel's partition follows the per-sequence window counts."""
