@@ -11,7 +11,15 @@
 
 namespace okq {
 
-constexpr int ZS = 132;  // row stride (floats) of the per-window staging buffers
+constexpr int ZS = 144;  // row stride (floats) of the per-window staging buffers: neighbouring rows 16 banks apart
+
+// Position of channel c inside a staged key row: the four 4-float chunks of every 16-channel block are
+// rotated by (block >> 1), which makes the three access patterns of the key quantiser (16-byte stores of a
+// block per thread, 8-byte accesses with stride 16 channels, 8-byte reads of the code-word order) free of
+// shared-memory bank conflicts.
+__device__ __forceinline__ int zpos(int c) {
+  return (c & ~15) + 4 * ((((c >> 2) & 3) + ((c >> 5) & 3)) & 3) + (c & 3);
+}
 
 struct WindowSmem {
   float z[W * ZS];        // rotated keys, or fp32 values
@@ -89,13 +97,13 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
         }
 #pragma unroll
     for (int q = 0; q < 4; q++)
-      *reinterpret_cast<float4*>(&zrow[16 * a + 4 * q]) = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+      *reinterpret_cast<float4*>(&zrow[zpos(16 * a + 4 * q)]) = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
     __syncwarp();
     // second half: channels 16*u + 2*a + e, u = 0..7: stages h = 16, 32, 64 act on u
     float v0[8], v1[8];
 #pragma unroll
     for (int u = 0; u < 8; u++) {
-      const float2 p = *reinterpret_cast<const float2*>(&zrow[16 * u + 2 * a]);
+      const float2 p = *reinterpret_cast<const float2*>(&zrow[zpos(16 * u + 2 * a)]);
       v0[u] = p.x; v1[u] = p.y;
     }
 #pragma unroll
@@ -111,16 +119,17 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
     __syncwarp();   // every thread of the token has read the first-half values before they are overwritten
 #pragma unroll
     for (int u = 0; u < 8; u++)
-      *reinterpret_cast<float2*>(&zrow[16 * u + 2 * a]) =
+      *reinterpret_cast<float2*>(&zrow[zpos(16 * u + 2 * a)]) =
           nf != 0.0f ? make_float2(__fmul_rn(v0[u], cinv), __fmul_rn(v1[u], cinv)) : make_float2(0.f, 0.f);
   }
   __syncthreads();
   {  // per channel: window minimum and step (Eq. 4)
     int c = tid;
-    float mn = sm.z[c], mx = mn;
+    const int cp = zpos(c);
+    float mn = sm.z[cp], mx = mn;
 #pragma unroll 8
     for (int i = 1; i < W; i++) {
-      float v = sm.z[i * ZS + c];
+      float v = sm.z[i * ZS + cp];
       if (v < mn) mn = v;
       if (v > mx) mx = v;
     }
@@ -171,7 +180,7 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
   // and packs that word for two tokens
   {
     uint32_t* words = reinterpret_cast<uint32_t*>(body + B_KCODE);
-    const int t = tid & 3, ww = (tid >> 2) & 1, tg = tid >> 3;   // tg: 16 token pairs
+    const int t = tid & 3, ww = (tid >> 2) & 1, tg = tid >> 3;   // tokens tg and tg + 16
     float mch[16], rch[16];
 #pragma unroll
     for (int q = 0; q < 8; q++) {
@@ -182,12 +191,12 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
     }
 #pragma unroll
     for (int k = 0; k < 2; k++) {
-      const int i = 2 * tg + k;
+      const int i = tg + 16 * k;
       uint32_t word = 0;
 #pragma unroll
       for (int q = 0; q < 8; q++) {
         const int c0 = 16 * ((ww * 8 + q) >> 1) + 8 * (q & 1) + 2 * t;
-        const float2 z2 = *reinterpret_cast<const float2*>(&sm.z[i * ZS + c0]);
+        const float2 z2 = *reinterpret_cast<const float2*>(&sm.z[i * ZS + zpos(c0)]);
 #pragma unroll
         for (int e = 0; e < 2; e++) {
           const float qv = rintf(__fmul_rn(__fsub_rn(e ? z2.y : z2.x, mch[2 * q + e]), rch[2 * q + e]));
