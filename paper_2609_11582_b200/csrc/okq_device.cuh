@@ -72,41 +72,47 @@ __device__ __forceinline__ float mx_decode(unsigned nib, int k) {
 }
 
 
-// Four E2M1 nibbles (low nibble first) -> two fp16 pairs of the unscaled grid values.  The byte LUT
-// holds the high bytes of fp16 {0, .5, 1, 1.5, 2, 3, 4, 6}; their low bytes are zero.
-__device__ __forceinline__ void e2m1x4_to_half2(uint32_t x, uint32_t& h01, uint32_t& h23) {
-  const uint32_t hb = __byte_perm(0x3E3C3800u, 0x46444240u, x & 0x7777u);
-  const uint32_t sg = x & 0x8888u;
-  h01 = __byte_perm(hb, 0u, 0x1404u) | ((sg << 12) & 0x8000u) | ((sg << 24) & 0x80000000u);
-  h23 = __byte_perm(hb, 0u, 0x3424u) | ((sg << 4) & 0x8000u) | ((sg << 16) & 0x80000000u);
-}
+// E2M1 decode by byte permute: a nibble's low three bits select the high byte of the fp16 value
+// {0, .5, 1, 1.5, 2, 3, 4, 6} * 4^j (low byte zero; 4^j adds 2 j to the exponent, i.e. 8 j to the high byte
+// of the non-zero entries).
+__device__ __forceinline__ uint32_t e2m1_lut_lo(int j) { return 0x3E3C3800u + 0x08080800u * (uint32_t)j; }
+__device__ __forceinline__ uint32_t e2m1_lut_hi(int j) { return 0x46444240u + 0x08080808u * (uint32_t)j; }
 
-// fp16 pair (2^k, 2^k) for k in [-24, 15]
-__device__ __forceinline__ uint32_t pow2_half2(int k) {
-  const uint32_t h = k >= -14 ? (uint32_t)(k + 15) << 10 : 1u << (k + 24);
-  return h | (h << 16);
+// fp16 pair (2^k, 2^k) from the stored exponent byte k + 127 (k in [-24, 15]): the byte is the exponent
+// field of the fp32 number 2^k
+__device__ __forceinline__ __half2 pow2_half2(uint32_t byte) {
+  const float f = __uint_as_float(byte << 23);
+  return __floats2half2_rn(f, f);
 }
 
 // Decoded (m * 4^j, s) of record positions 4*lane .. 4*lane+3 from the 136 MXFP4 metadata bytes
-// (global or shared, 2-byte aligned): four fp16 each, exact; m with the position scale of the fp16 layout.
+// (global or shared, 2-byte aligned): four fp16 each, exact.  m carries the position scale of the fp16
+// layout's m plane: positions 4*lane + {0, 1} have j = 2*(lane & 1), the other two j + 1 (folded into the
+// lookup: grid * 4^j <= 384, and the product with 2^k, |m| * 4^j <= 64, is an fp16 number).
 __device__ __forceinline__ void mx_decode_lane(const unsigned char* meta, int lane, uint2& m4, uint2& s4) {
   const uint32_t xm = *reinterpret_cast<const unsigned short*>(meta + 2 * lane);
   const uint32_t xs = *reinterpret_cast<const unsigned short*>(meta + 64 + 2 * lane);
   const int blk = (lane >> 1) & 3;   // positions 8j .. 8j+7 (mod 32) belong to channel block j
-  const uint32_t pm = pow2_half2((int)meta[128 + blk] - 127), ps = pow2_half2((int)meta[132 + blk] - 127);
-  uint32_t a, b;
-  e2m1x4_to_half2(xm, a, b);
-  __half2 r0 = __hmul2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<const __half2*>(&pm));
-  __half2 r1 = __hmul2(*reinterpret_cast<__half2*>(&b), *reinterpret_cast<const __half2*>(&pm));
-  // the staged m plane carries the position scale 4^j: positions 4*lane + {0,1} have j = 2*(lane & 1), the
-  // other two j + 1 (a second exact multiply: 2^k * 4^j alone may leave the fp16 range)
-  const uint32_t q0 = pow2_half2(4 * (lane & 1)), q1 = pow2_half2(4 * (lane & 1) + 2);
-  r0 = __hmul2(r0, *reinterpret_cast<const __half2*>(&q0));
-  r1 = __hmul2(r1, *reinterpret_cast<const __half2*>(&q1));
+  const __half2 pm = pow2_half2(meta[128 + blk]), ps = pow2_half2(meta[132 + blk]);
+  const int j0 = 2 * (lane & 1);
+  // magnitudes: bytes 0, 1 of the first lookup (scale 4^j0), bytes 2, 3 of the second (4^(j0+1))
+  const uint32_t im = xm & 0x7777u;
+  const uint32_t ma = __byte_perm(e2m1_lut_lo(j0), e2m1_lut_hi(j0), im);
+  const uint32_t mb = __byte_perm(e2m1_lut_lo(j0 + 1), e2m1_lut_hi(j0 + 1), im);
+  // signs: nibble bit 3 of values 0 / 1 -> bits 15 / 31, of values 2 / 3 likewise (the products spread the
+  // four sign bits; stray carries stay below the masked bits)
+  const uint32_t sg = xm & 0x8888u;
+  uint32_t h01 = __byte_perm(ma, 0u, 0x1404u) | ((sg * 0x01001000u) & 0x80008000u);
+  uint32_t h23 = __byte_perm(mb, 0u, 0x3424u) | ((sg * 0x00010010u) & 0x80008000u);
+  __half2 r0 = __hmul2(*reinterpret_cast<__half2*>(&h01), pm);
+  __half2 r1 = __hmul2(*reinterpret_cast<__half2*>(&h23), pm);
   m4 = make_uint2(*reinterpret_cast<uint32_t*>(&r0), *reinterpret_cast<uint32_t*>(&r1));
-  e2m1x4_to_half2(xs, a, b);
-  r0 = __hmul2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<const __half2*>(&ps));
-  r1 = __hmul2(*reinterpret_cast<__half2*>(&b), *reinterpret_cast<const __half2*>(&ps));
+  // s is never negative
+  const uint32_t sa = __byte_perm(e2m1_lut_lo(0), e2m1_lut_hi(0), xs & 0x7777u);
+  h01 = __byte_perm(sa, 0u, 0x1404u);
+  h23 = __byte_perm(sa, 0u, 0x3424u);
+  r0 = __hmul2(*reinterpret_cast<__half2*>(&h01), ps);
+  r1 = __hmul2(*reinterpret_cast<__half2*>(&h23), ps);
   s4 = make_uint2(*reinterpret_cast<uint32_t*>(&r0), *reinterpret_cast<uint32_t*>(&r1));
 }
 
