@@ -187,11 +187,13 @@ void okqo_window_quantize(const float* z, uint16_t* meta, uint8_t* codes) {
  * block of 32.  The paper does not say how blocks are formed or how values are rounded; the
  * reading taken here (listed in the design notes):
  *   - a block is 32 consecutive channels of one window, separately for m and for s;
- *   - the scale is the smallest power of two 2^k with 6 * 2^k >= max|x| over the block (6 is
- *     the largest E2M1 magnitude), k clamped to [-23, 12] so that every decoded value
- *     grid * 2^k is exactly an fp16 number;
- *   - m is rounded DOWN to the E2M1 grid {0, .5, 1, 1.5, 2, 3, 4, 6} * 2^k (with sign), the
- *     step s is rounded UP, so the four levels m' + s' * {0,1,2,3} always cover [min, max];
+ *   - conversion as in the OCP microscaling format: the block exponent is floor(log2 max|x|) - 2 (2^2 is
+ *     the largest power of two of E2M1), clamped to [-23, 12] so that every decoded value grid * 2^k is
+ *     exactly an fp16 number; elements are rounded to the nearest value of the grid
+ *     {0, .5, 1, 1.5, 2, 3, 4, 6} * 2^k (ties to the even mantissa), magnitudes beyond 6 * 2^k saturate;
+ *     a value below m' or above m' + 3 s' takes the end code (codes are clamped to [0, 3] anyway).  With
+ *     this conversion the key error grows by a few percent over fp16 metadata, the order of the paper's
+ *     error table (0.1833 against 0.1495); rounding m down and s up so that nothing clips doubles it;
  *   - codes are computed against the decoded pair (m', s') exactly as in the fp16 format.
  * 2 * (128 * 4 + 4 * 8) bits per 32-token window = 136 B instead of 512 B: 72.25 B per token per
  * KV head = 2.258 bits per element, the figure the paper prints for its default.
@@ -200,34 +202,31 @@ static const float MX_GRID[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f}
 
 int okqo_bytes_per_window_mx(void) { return OKQ_W * ((OKQ_D * 2) / 8 + 2 + (OKQ_D * 2) / 8 + 2) + 2 * (OKQ_D / 2 + OKQ_D / 32); }
 
-/* smallest k in [-23, 12] with 6 * 2^k >= amax */
+/* block exponent floor(log2 amax) - 2, clamped to [-23, 12] (-23 for an all-zero block) */
 int okqo_mx_scale_exp(float amax) {
   int k = -23;
   if (amax > 0.0f) {
     int e;
-    float f = frexpf(amax, &e); /* amax = f * 2^e, f in [0.5, 1); 6 * 2^k = 0.75 * 2^(k+3) */
-    k = (f <= 0.75f) ? e - 3 : e - 2;
+    (void)frexpf(amax, &e); /* amax = f * 2^e, f in [0.5, 1): floor(log2 amax) = e - 1 */
+    k = e - 1 - 2;          /* the element format's largest power of two is 2^2 */
   }
   if (k < -23) k = -23;
   if (k > 12) k = 12;
   return k;
 }
 
-/* nibble (sign << 3 | grid index) of x on the grid * 2^k; mode < 0 rounds down, mode > 0 rounds up */
-uint8_t okqo_mx_encode(float x, int k, int mode) {
+/* nibble (sign << 3 | grid index) of x on the grid * 2^k: nearest grid value, ties to the value with an even
+ * mantissa bit (grid indices 0, 2, 4, 6), magnitudes beyond 6 * 2^k saturate to 6 * 2^k */
+uint8_t okqo_mx_encode(float x, int k) {
   float q = ldexpf(x, -k); /* exact */
-  int best = -1;
-  float bestv = 0.0f;
-  for (int sgn = 0; sgn < 2; sgn++)
-    for (int i = 0; i < 8; i++) {
-      if (sgn && i == 0) continue; /* no negative zero */
-      float g = sgn ? -MX_GRID[i] : MX_GRID[i];
-      int ok = mode < 0 ? (g <= q) : (g >= q);
-      if (!ok) continue;
-      if (best < 0 || (mode < 0 ? g > bestv : g < bestv)) { best = (sgn << 3) | i; bestv = g; }
-    }
-  if (best < 0) best = mode < 0 ? (1 << 3 | 7) : 7; /* beyond the grid: saturate (cannot happen with the scale above) */
-  return (uint8_t)best;
+  float a = fabsf(q);
+  int best = 0;
+  for (int i = 1; i < 8; i++) {
+    float d0 = fabsf(a - MX_GRID[best]), d1 = fabsf(a - MX_GRID[i]);
+    if (d1 < d0 || (d1 == d0 && (i & 1) == 0)) best = i;
+  }
+  if (best == 0) return 0; /* no negative zero */
+  return (uint8_t)(((q < 0.0f) ? 8 : 0) | best);
 }
 
 float okqo_mx_decode(uint8_t nib, int k) {
@@ -250,13 +249,13 @@ void okqo_window_quantize_mx(const float* z, uint8_t* mx, uint16_t* meta_dec, ui
       if (v > mxv[c]) mxv[c] = v;
     }
   }
-  for (int b = 0; b < OKQ_D / 32; b++) { /* minima: scale from the block's largest magnitude, round down */
+  for (int b = 0; b < OKQ_D / 32; b++) { /* minima: scale from the block's largest magnitude */
     float amax = 0.0f;
     for (int c = 32 * b; c < 32 * b + 32; c++) if (fabsf(mn[c]) > amax) amax = fabsf(mn[c]);
     int k = okqo_mx_scale_exp(amax);
     mx[128 + b] = (uint8_t)(k + 127);
     for (int c = 32 * b; c < 32 * b + 32; c++) {
-      uint8_t nib = okqo_mx_encode(mn[c], k, -1);
+      uint8_t nib = okqo_mx_encode(mn[c], k);
       mx[c / 2] |= (uint8_t)(nib << (4 * (c & 1)));
       md[c] = okqo_mx_decode(nib, k);
       float range = mxv[c] - md[c];
@@ -264,13 +263,13 @@ void okqo_window_quantize_mx(const float* z, uint8_t* mx, uint16_t* meta_dec, ui
       sr[c] = range / 3.0f;
     }
   }
-  for (int b = 0; b < OKQ_D / 32; b++) { /* steps: round up */
+  for (int b = 0; b < OKQ_D / 32; b++) { /* steps */
     float amax = 0.0f;
     for (int c = 32 * b; c < 32 * b + 32; c++) if (sr[c] > amax) amax = sr[c];
     int k = okqo_mx_scale_exp(amax);
     mx[132 + b] = (uint8_t)(k + 127);
     for (int c = 32 * b; c < 32 * b + 32; c++) {
-      uint8_t nib = okqo_mx_encode(sr[c], k, +1);
+      uint8_t nib = okqo_mx_encode(sr[c], k);
       mx[64 + c / 2] |= (uint8_t)(nib << (4 * (c & 1)));
       sd[c] = okqo_mx_decode(nib, k);
     }

@@ -47,7 +47,7 @@ def lib():
         L.okqo_mx_scale_exp.restype = C.c_int
         L.okqo_mx_scale_exp.argtypes = [C.c_float]
         L.okqo_mx_encode.restype = C.c_uint8
-        L.okqo_mx_encode.argtypes = [C.c_float, C.c_int, C.c_int]
+        L.okqo_mx_encode.argtypes = [C.c_float, C.c_int]
         L.okqo_mx_decode.restype = C.c_float
         L.okqo_mx_decode.argtypes = [C.c_uint8, C.c_int]
         _lib = L
