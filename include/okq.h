@@ -30,9 +30,10 @@
  *     [1664, 2688)  value codes, 2 bits x 32 tokens x 128 channels
  * With OKQ_META_MXFP4 (the paper's default metadata: 2.258 bits/element) the first 512 bytes shrink to
  * 136: m and s as 4-bit E2M1 elements with one power-of-two E8M0 scale per 32 consecutive channels
- * (m rounded down, s rounded up, so the four levels still cover the window; the scale is the smallest
- * power of two whose 6-fold reaches the block maximum, clamped to [2^-23, 2^12] so that every decoded
- * value is an fp16 number), OKQ_RECORD_BYTES_MX = 2312 bytes per record, 72.25 per token per KV head.
+ * (converted as in the OCP microscaling format: block exponent floor(log2 max|x|) - 2, clamped to
+ * [-23, 12] so that every decoded value is an fp16 number; elements rounded to the nearest grid value,
+ * ties to even, saturating at 6 * 2^k), OKQ_RECORD_BYTES_MX = 2312 bytes per record, 72.25 per token per
+ * KV head.  A key coordinate outside [m', m' + 3 s'] takes the end code.
  * Codes are computed against the decoded pair, exactly as with fp16 metadata.
  * Inside a record the channel / token order is the one the decode kernel's tensor-core
  * fragments want; okq_cache_export / okq_cache_import convert to and from the canonical

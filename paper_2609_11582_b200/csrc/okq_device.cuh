@@ -37,15 +37,16 @@ __device__ __forceinline__ float4 warp_fwht(float4 y, int lane) {
   return make_float4(v[0], v[1], v[2], v[3]);
 }
 
-// ---- MXFP4 metadata: E2M1 elements {0, .5, 1, 1.5, 2, 3, 4, 6} (sign in bit 3) times 2^k
+// ---- MXFP4 metadata: E2M1 elements {0, .5, 1, 1.5, 2, 3, 4, 6} (sign in bit 3) times 2^k, converted as in
+// the OCP microscaling format
 
-// smallest k in [-23, 12] with 6 * 2^k >= amax  (6 * 2^k = 0.75 * 2^(k+3))
+// block exponent floor(log2 amax) - 2, clamped to [-23, 12] (-23 for an all-zero block)
 __device__ __forceinline__ int mx_scale_exp(float amax) {
   int k = -23;
   if (amax > 0.0f) {
     int e;
-    const float f = frexpf(amax, &e);
-    k = f <= 0.75f ? e - 3 : e - 2;
+    (void)frexpf(amax, &e);   // amax = f * 2^e, f in [0.5, 1)
+    k = e - 3;
   }
   return max(-23, min(12, k));
 }
@@ -54,16 +55,14 @@ __device__ __forceinline__ float mx_grid(int idx) {
   return idx < 4 ? 0.5f * (float)idx : (idx == 4 ? 2.0f : (idx == 5 ? 3.0f : (idx == 6 ? 4.0f : 6.0f)));
 }
 
-// nibble of x on the grid * 2^k, rounded down (up = false) or up (up = true); |x| <= 6 * 2^k
-__device__ __forceinline__ unsigned mx_encode(float x, int k, bool up) {
+// nibble of x on the grid * 2^k: nearest grid value, ties to the even mantissa bit (0, 1, 2, 4), magnitudes
+// beyond 6 * 2^k saturate.  The decision points are the midpoints of neighbouring grid values; a tie goes up
+// exactly when the upper neighbour has the even mantissa bit.
+__device__ __forceinline__ unsigned mx_encode(float x, int k) {
   const float q = ldexpf(x, -k);   // exact
   const float a = fabsf(q);
-  // magnitude index: largest grid value <= a, or smallest grid value >= a
-  const int lo = (a >= 0.5f) + (a >= 1.0f) + (a >= 1.5f) + (a >= 2.0f) + (a >= 3.0f) + (a >= 4.0f) + (a >= 6.0f);
-  const int hi = min(7, (a > 0.0f) + (a > 0.5f) + (a > 1.0f) + (a > 1.5f) + (a > 2.0f) + (a > 3.0f) + (a > 4.0f));
-  const bool neg = q < 0.0f;
-  const int idx = (up != neg) ? hi : lo;   // rounding up a negative number shrinks its magnitude
-  return idx == 0 ? 0u : ((neg ? 8u : 0u) | (unsigned)idx);
+  const int idx = (a > 0.25f) + (a >= 0.75f) + (a > 1.25f) + (a >= 1.75f) + (a > 2.5f) + (a >= 3.5f) + (a > 5.0f);
+  return idx == 0 ? 0u : ((q < 0.0f ? 8u : 0u) | (unsigned)idx);
 }
 
 __device__ __forceinline__ float mx_decode(unsigned nib, int k) {

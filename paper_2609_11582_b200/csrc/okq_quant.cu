@@ -146,13 +146,13 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
       reinterpret_cast<__half*>(rec + OFF_KM)[p] = __float2half_rn(mf * (float)(1 << (2 * meta_shift(c))));   // exact
       reinterpret_cast<__half*>(rec + OFF_KS)[p] = sh;
     } else {
-      // MXFP4: a warp is one block of 32 consecutive channels.  m rounds down, s rounds up.
+      // MXFP4: a warp is one block of 32 consecutive channels; nearest-even conversion of m, then of s
       const int lane = tid & 31, blk = tid >> 5;
       float amax = fabsf(mn);
 #pragma unroll
       for (int d = 16; d; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
       const int km = mx_scale_exp(amax);
-      const unsigned mnib = mx_encode(mn, km, false);
+      const unsigned mnib = mx_encode(mn, km);
       const float mf = mx_decode(mnib, km);
       float range = __fsub_rn(mx, mf);
       if (range < 0.0f) range = 0.0f;
@@ -161,7 +161,7 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
 #pragma unroll
       for (int d = 16; d; d >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, d));
       const int ks = mx_scale_exp(smax);
-      const unsigned snib = mx_encode(sraw, ks, true);
+      const unsigned snib = mx_encode(sraw, ks);
       const float sf = mx_decode(snib, ks);
       sm.a[c] = mf;
       sm.b[c] = sf > 0.0f ? __fdiv_rn(1.0f, sf) : 0.0f;

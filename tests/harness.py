@@ -59,10 +59,17 @@ class Case:
                                      unit_seq=unit_seq, meta_format=self.meta_format)
         return kq, vq, kb, vb
 
-    def oracle_attention(self, layer, path=1, extra_k=None, extra_v=None):
-        """Oracle output [B, Hq, 128] for the bulk-built cache of `layer`."""
+    def oracle_attention(self, layer, path=1, extra_k=None, extra_v=None, v_codes=None):
+        """Oracle output [B, Hq, 128] for the bulk-built cache of `layer`.  `v_codes` (canonical value codes
+        [B, Hkv, capacity, 32] as exported) replaces the oracle's own value codes: the tensor-core value
+        quantiser may move a coordinate that sits on a codebook threshold to the neighbouring level."""
         w = self.w
         kq, vq, kb, vb = self.oracle_quantize(layer)
+        if v_codes is not None:
+            npk_ = (self.n // W) * W
+            vq = dict(vq)
+            vq["codes"] = np.ascontiguousarray(
+                v_codes.cpu().numpy().reshape(w.batch * w.n_kv_heads, -1, 32)[:, :npk_])
         npk = (self.n // W) * W
         U = w.batch * w.n_kv_heads
         G = w.group

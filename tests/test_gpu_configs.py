@@ -129,7 +129,8 @@ def test_every_window_holds_all_three_modalities(meta_format):
     assert b.cache.device_status() == 0
     assert torch.equal(ea["v_norm"], eb["v_norm"])
     assert (ea["v_codes"] != eb["v_codes"]).sum().item() <= 8      # only coordinates that sit on a threshold may differ
-    Hn.assert_attention_close(b.gpu_decode(0)[0], ref)
+    ref_b, _ = b.oracle_attention(0, v_codes=eb["v_codes"])       # the oracle over the codes this cache holds
+    Hn.assert_attention_close(b.gpu_decode(0)[0], ref_b)
 
 
 def test_ragged_batch_lengths():
