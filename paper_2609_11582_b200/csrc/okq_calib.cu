@@ -427,11 +427,12 @@ okq_status okq_calib_rotation(const float* C, const float* signs, void* workspac
   if (!C || !signs || !workspace || !R_out || !lambda_out) return OKQ_ERR_INVALID_ARG;
   if (!aligned16(C) || !aligned16(workspace) || !aligned16(R_out)) return OKQ_ERR_ALIGNMENT;
   if (workspace_bytes < EIGEN_BYTES) return OKQ_ERR_WORKSPACE;
-  static thread_local bool attr_set = false;
-  if (!attr_set) {
+  static thread_local unsigned long long attr_mask = 0;
+  int attr_dev = 0;
+  if (attr_needed(attr_mask, attr_dev)) {
     cudaError_t e = cudaFuncSetAttribute(k_calib_eigen, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EIGEN_BYTES);
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
-    attr_set = true;
+    attr_done(attr_mask, attr_dev);
   }
   k_calib_eigen<<<1, EIG_THREADS, EIGEN_BYTES, static_cast<cudaStream_t>(stream)>>>(C, signs, static_cast<double*>(workspace), R_out,
                                                                                   lambda_out, sweeps_out);

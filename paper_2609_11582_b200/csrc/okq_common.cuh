@@ -30,6 +30,18 @@ inline CacheView make_view(const okq_cache* c) {
   return v;
 }
 
+// Function attributes (dynamic shared memory size) are per device: `mask` remembers, per calling thread and
+// call site, the devices on which they have been set.  Returns true when the current device still needs them.
+inline bool attr_needed(unsigned long long& mask, int& dev_out) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  dev_out = dev;
+  return dev < 0 || dev >= 64 || !((mask >> dev) & 1ull);
+}
+inline void attr_done(unsigned long long& mask, int dev) {
+  if (dev >= 0 && dev < 64) mask |= 1ull << dev;
+}
+
 inline okq_status launch_status() {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {

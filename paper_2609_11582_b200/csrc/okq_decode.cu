@@ -514,11 +514,12 @@ okq_status okq_decode_attention_simt(const okq_cache* cache, int32_t layer, int3
   P.n_splits = num_splits > 0 ? num_splits : auto_splits(cache, layer_count);
   P.partials = static_cast<Partial*>(workspace);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  static thread_local bool attr_set = false;
-  if (!attr_set) {
+  static thread_local unsigned long long attr_mask = 0;
+  int attr_dev = 0;
+  if (attr_needed(attr_mask, attr_dev)) {
     cudaError_t e = cudaFuncSetAttribute(k_decode_simt, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecodeSmem));
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
-    attr_set = true;
+    attr_done(attr_mask, attr_dev);
   }
   dim3 grid(P.n_splits, cache->n_kv_heads, cache->batch * layer_count);
   if (g_ev_before) cudaEventRecord(g_ev_before, s);

@@ -686,8 +686,9 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
 }
 
 okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, cudaEvent_t before, cudaEvent_t after) {
-  static thread_local bool attr_set = false;
-  if (!attr_set) {
+  static thread_local unsigned long long attr_mask = 0;
+  int attr_dev = 0;
+  if (attr_needed(attr_mask, attr_dev)) {
     cudaError_t e = cudaFuncSetAttribute(k_decode_mma<FMT_FP16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)sizeof(MmaSmem<FMT_FP16>));
     if (e == cudaSuccess)
@@ -696,7 +697,7 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k_combine_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem));
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
-    attr_set = true;
+    attr_done(attr_mask, attr_dev);
   }
   if (before) cudaEventRecord(before, s);
   if (P.cv.fmt == FMT_MXFP4) k_decode_mma<FMT_MXFP4><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_MXFP4>), s>>>(P);

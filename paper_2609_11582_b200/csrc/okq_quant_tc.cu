@@ -510,12 +510,13 @@ EncodeTiledFn encode_tiled() {
 okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __half* v, const int64_t strides[3],
                                      const unsigned char* modality, int n_tokens, const float* R, int n_R,
                                      int n_sm, cudaStream_t s) {
-  static thread_local bool attr_set = false;
-  if (!attr_set) {
+  static thread_local unsigned long long attr_mask = 0;
+  int attr_dev = 0;
+  if (attr_needed(attr_mask, attr_dev)) {
     cudaError_t e = cudaFuncSetAttribute(k_quantize_values_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)sizeof(TcSmem) + 1024);
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
-    attr_set = true;
+    attr_done(attr_mask, attr_dev);
   }
   const int n_win = n_tokens / W;
   const long long n_tiles = (long long)((n_win + 3) / 4) * cv.n_kv_heads * cv.batch;
