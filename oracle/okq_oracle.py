@@ -247,3 +247,39 @@ def quantize_batch(k_bits, v_bits, modality, signs, R, unit_seq=None, unit_rot=N
     if meta_format == 1:
         kq["mx"] = mx
     return kq, vq, th
+
+
+# ---------------------------------------------------------------- streaming schedules
+
+def packed_counts(n: int, schedule: int):
+    """(packed keys, packed values) of a sequence of n tokens.
+
+    schedule 0: both are packed as soon as a 32-token window is complete.
+    schedule 1, the paper's captioning schedule (Implementation details): keys are quantised every 128 tokens,
+    in groups of 32; values stay behind a 128-token sliding fp16 window before they are quantised (window by
+    window, since a value record holds 32 tokens)."""
+    if schedule == 0:
+        return (n // W) * W, (n // W) * W
+    return (n // 128) * 128, (((n - 128) // W) * W if n >= 128 else 0)
+
+
+def attention_scheduled(q_bits, kq, vq, modality, k_bits, v_bits, signs, R, k_packed: int, v_packed: int,
+                        sm_scale=None):
+    """Attention of one (layer, sequence, KV head) by definition, in fp64, when the first `k_packed` keys and the
+    first `v_packed` values are read from the packed cache and the rest are still raw fp16:
+    out_h = softmax(q_h K_hat^T * scale) V_hat with K_hat / V_hat the dequantised (Eq. 2-4, Eq. 6) or raw rows.
+
+    q_bits [G,128] u16; kq / vq: one unit's packed arrays (codes [np,32], norm [np], meta [np/32,128,2]);
+    modality [n] u8; k_bits / v_bits [n,128] u16 raw tokens.  Returns fp64 [G,128]."""
+    k = half_to_float(_c(k_bits, np.uint16)).astype(np.float64).reshape(-1, D)
+    v = half_to_float(_c(v_bits, np.uint16)).astype(np.float64).reshape(-1, D)
+    for t in range(k_packed):
+        k[t] = dequant_key(kq["codes"][t], kq["norm"][t], kq["meta"][t // W], signs)
+    for t in range(v_packed):
+        v[t] = dequant_value(vq["codes"][t], vq["norm"][t], R[int(modality[t])])
+    q = half_to_float(_c(q_bits, np.uint16)).astype(np.float64).reshape(-1, D)
+    scale = D ** -0.5 if sm_scale is None else sm_scale
+    s = (q @ k.T) * scale
+    s -= s.max(axis=1, keepdims=True)
+    p = np.exp(s)
+    return (p / p.sum(axis=1, keepdims=True)) @ v

@@ -524,3 +524,37 @@ def test_mx_attention_paths_agree():
     # and differs measurably from the fp16-metadata cache (it is a different, coarser encoding)
     ref = _run(0, c)
     assert np.abs(a[0] - ref).max() > 1e-4 and np.isfinite(a).all()
+
+
+# ------------------------------------------------------------------ streaming schedules
+
+def test_packed_counts_follow_the_stated_schedules():
+    # window schedule: whole 32-token windows
+    assert [O.packed_counts(n, 0) for n in (0, 31, 32, 100)] == [(0, 0), (0, 0), (32, 32), (96, 96)]
+    # captioning schedule: keys every 128 tokens, values behind a 128-token fp16 window
+    want = {0: (0, 0), 127: (0, 0), 128: (128, 0), 159: (128, 0), 160: (128, 32), 191: (128, 32), 192: (128, 64),
+            255: (128, 96), 256: (256, 128), 2048 + 77: (2048, 1984)}
+    for n, kv in want.items():
+        assert O.packed_counts(n, 1) == kv
+    for n in range(0, 700):
+        kp, vp = O.packed_counts(n, 1)
+        assert kp % 128 == 0 and vp % 32 == 0 and 0 <= n - kp < 128 and vp <= kp
+        assert (n < 128 and vp == 0) or 128 <= n - vp < 160       # the raw values are the last 128 .. 159 tokens
+
+
+def test_scheduled_attention_reduces_to_known_cases():
+    c = _small_case(139, seed=41)
+    kq1, vq1 = c["kq"], c["vq"]
+    # the window schedule is the attention oracle's definition path
+    ref = _run(0, c)
+    got = O.attention_scheduled(c["q"], kq1, vq1, c["mod"], c["kb"], c["vb"], c["signs"], c["R"], 128, 128)
+    assert np.abs(got - ref).max() < 1e-12
+    # nothing packed: plain fp16 attention
+    q = torch.from_numpy(bits2f(c["q"])); k = torch.from_numpy(bits2f(c["kb"])); v = torch.from_numpy(bits2f(c["vb"]))
+    plain = torch.nn.functional.scaled_dot_product_attention(q[None], k[None], v[None])[0].numpy()
+    got = O.attention_scheduled(c["q"], kq1, vq1, c["mod"], c["kb"], c["vb"], c["signs"], c["R"], 0, 0)
+    assert np.abs(got - plain).max() < 1e-12
+    # captioning schedule at n = 139: keys of the first 128 tokens packed, every value raw
+    kp, vp = O.packed_counts(139, 1)
+    got = O.attention_scheduled(c["q"], kq1, vq1, c["mod"], c["kb"], c["vb"], c["signs"], c["R"], kp, vp)
+    assert (kp, vp) == (128, 0) and np.abs(got - ref).max() > 1e-4 and np.abs(got - plain).max() > 1e-4
