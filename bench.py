@@ -256,6 +256,10 @@ def main():
     ap.add_argument("--meta", default="fp16", choices=["fp16", "mxfp4"],
                     help="(m, s) metadata format of the cache: fp16 = 84 B per token and KV head (the headline "
                          "configuration), mxfp4 = 72.25 B (secondary measurement; no cpu_baseline)")
+    ap.add_argument("--schedule", default="window", choices=["window", "caption"],
+                    help="streaming schedule of the cache: window = pack every 32 tokens (the headline configuration), "
+                         "caption = the paper's captioning schedule (keys every 128 tokens, values behind a 128-token "
+                         "fp16 window; secondary measurement, no cpu_baseline)")
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill", "calib"],
                     help="decode: the headline decode step; prefill: bulk quantisation of a fresh fp16 K/V cache "
                          "(secondary measurement, default workload prefill7b); calib: offline calibration of the "
@@ -286,7 +290,9 @@ def main():
     L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
     mx = args.meta == "mxfp4"
     bytes_th = 72.25 if mx else BYTES_PER_TOKEN_HEAD
-    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev, meta_format=B.META_MXFP4 if mx else B.META_FP16)
+    caption = args.schedule == "caption"
+    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev, meta_format=B.META_MXFP4 if mx else B.META_FP16,
+                    schedule=B.SCHEDULE_CAPTION if caption else B.SCHEDULE_WINDOW)
     mod = WL.modality_layout(w).unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
     signs = torch.stack([WL.gen_signs(w, l) for l in range(L)]).to(dev)
     R = torch.stack([WL.gen_rotations(w, l) for l in range(L)]).unsqueeze(1).contiguous().to(dev)
@@ -432,7 +438,7 @@ def main():
     if rank != 0:
         return
     cpu = None
-    if world == 1 and not args.no_cpu_baseline and not mx:
+    if world == 1 and not args.no_cpu_baseline and not mx and not caption:
         n_l, n_s = min(2, L), min(8, Bn)
         oargs, unit_rot, th_units = oracle_prepare(w, n_l, n_s)
         passes = [oracle_pass(oargs, unit_rot) for _ in range(3)]
@@ -445,7 +451,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "n_layers": L, "batch": Bn, "n_q_heads": Hq, "n_kv_heads": H, "context": N,
-                       "meta_format": args.meta, "bytes_per_token_head": bytes_th,
+                       "meta_format": args.meta, "bytes_per_token_head": bytes_th, "schedule": args.schedule,
                        "step": "okq_append(1 text token/seq, all layers) + okq_decode_attention(all layers), one call each",
                        "packed_kv_bytes_per_step": packed_bytes, "l2": f"inputs ({packed_bytes / 1e9:.2f} GB of records per step) exceed L2",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},

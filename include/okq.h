@@ -82,13 +82,29 @@ typedef struct okq_cache {
   int32_t window;    /* 32 */
   int32_t capacity;  /* max tokens per sequence, multiple of 32 */
   int32_t meta_format; /* OKQ_META_FP16 (0) or OKQ_META_MXFP4 (1): how the key (m, s) pairs are stored */
+  int32_t schedule;    /* OKQ_SCHEDULE_WINDOW (0) or OKQ_SCHEDULE_CAPTION (1): when raw tokens are packed, see below */
+  int32_t reserved;    /* 0 */
   void* records;     /* [n_layers][batch][n_kv_heads][capacity/32][record bytes of the format]; 16-byte aligned */
   uint8_t* modality; /* [batch][capacity], shared by all layers and heads */
-  void* k_tail;      /* [n_layers][batch][n_kv_heads][32][128] fp16: raw keys not yet in a full window */
-  void* v_tail;      /* same for values */
-  int32_t* seq_len;  /* [n_layers][batch] tokens held; the first (seq_len & ~31) are packed */
+  void* k_tail;      /* [n_layers][batch][n_kv_heads][32 | 128][128] fp16: raw keys not packed yet (token t in slot t mod 32 | 128) */
+  void* v_tail;      /* [n_layers][batch][n_kv_heads][32 | 160][128] fp16: raw values not packed yet (slot t mod 32 | 160) */
+  int32_t* seq_len;  /* [n_layers][batch] tokens held; how many of them are packed follows from the schedule */
   int32_t* status;   /* [1] sticky first device-side error, 0 = none */
 } okq_cache;
+
+/*
+ * Streaming schedules (the paper's "Implementation details").  With n tokens in a sequence:
+ *   OKQ_SCHEDULE_WINDOW   keys and values are packed as soon as a 32-token window is complete: the first
+ *                         32 * floor(n / 32) tokens of both are packed, at most 31 are raw fp16.
+ *   OKQ_SCHEDULE_CAPTION  the paper's captioning schedule: keys are packed every 128 tokens, in four groups of
+ *                         32 (the first 128 * floor(n / 128) keys are packed, at most 127 are raw), values stay
+ *                         behind a sliding window of 128 raw fp16 tokens (the first 32 * floor((n - 128) / 32)
+ *                         values are packed once n >= 128, 128 to 159 are raw).  A window's packed content is the
+ *                         same under both schedules; only which recent tokens are still fp16 differs.
+ *                         okq_decode_attention_simt returns OKQ_ERR_UNSUPPORTED for such a cache.
+ */
+#define OKQ_SCHEDULE_WINDOW 0
+#define OKQ_SCHEDULE_CAPTION 1
 
 /* Byte sizes of the six device buffers of a cache with the given shape fields (pointers
  * are ignored), in the order records, modality, k_tail, v_tail, seq_len, status.

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libokq.so")
 HEAD_DIM, WINDOW, RECORD_BYTES, MAX_GROUP = 128, 32, 2688, 8
 RECORD_BYTES_MX, MX_META_BYTES = 2312, 136
 META_FP16, META_MXFP4 = 0, 1
+SCHEDULE_WINDOW, SCHEDULE_CAPTION = 0, 1
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(8)
 
@@ -23,6 +24,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CAPACITY, ERR_WORKSPACE
 class okq_cache(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("batch", C.c_int32), ("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("window", C.c_int32), ("capacity", C.c_int32), ("meta_format", C.c_int32),
+                ("schedule", C.c_int32), ("reserved", C.c_int32),
                 ("records", C.c_void_p), ("modality", C.c_void_p), ("k_tail", C.c_void_p), ("v_tail", C.c_void_p),
                 ("seq_len", C.c_void_p), ("status", C.c_void_p)]
 
@@ -120,8 +122,8 @@ def _check(st: int, where: str):
 
 
 def cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, head_dim=HEAD_DIM, window=WINDOW,
-                meta_format=META_FP16):
-    shape = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, head_dim, window, capacity, meta_format)
+                meta_format=META_FP16, schedule=SCHEDULE_WINDOW):
+    shape = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, head_dim, window, capacity, meta_format, schedule, 0)
     out = (C.c_size_t * 6)()
     _check(lib().okq_cache_sizes(C.byref(shape), out), "okq_cache_sizes")
     return list(out)
@@ -130,9 +132,10 @@ def cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, head_dim=HEAD_
 class Cache:
     """Device buffers of a 2-bit KV cache plus the C struct that describes them."""
 
-    def __init__(self, n_layers, batch, n_kv_heads, n_q_heads, capacity, device="cuda", meta_format=META_FP16):
-        sizes = cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, meta_format=meta_format)
-        self.meta_format = meta_format
+    def __init__(self, n_layers, batch, n_kv_heads, n_q_heads, capacity, device="cuda", meta_format=META_FP16,
+                 schedule=SCHEDULE_WINDOW):
+        sizes = cache_sizes(n_layers, batch, n_kv_heads, n_q_heads, capacity, meta_format=meta_format, schedule=schedule)
+        self.meta_format, self.schedule = meta_format, schedule
         self.n_layers, self.batch, self.n_kv_heads, self.n_q_heads, self.capacity = (
             n_layers, batch, n_kv_heads, n_q_heads, capacity)
         self.device = torch.device(device)
@@ -142,7 +145,7 @@ class Cache:
         self.v_tail = torch.zeros(sizes[3] // 2, dtype=torch.float16, device=device)
         self.seq_len = torch.zeros(n_layers * batch, dtype=torch.int32, device=device)
         self.status = torch.zeros(4, dtype=torch.int32, device=device)
-        self.c = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, HEAD_DIM, WINDOW, capacity, meta_format,
+        self.c = okq_cache(n_layers, batch, n_kv_heads, n_q_heads, HEAD_DIM, WINDOW, capacity, meta_format, schedule, 0,
                            self.records.data_ptr(), self.modality.data_ptr(), self.k_tail.data_ptr(),
                            self.v_tail.data_ptr(), self.seq_len.data_ptr(), self.status.data_ptr())
 

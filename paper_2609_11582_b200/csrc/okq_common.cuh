@@ -21,6 +21,7 @@ inline CacheView make_view(const okq_cache* c) {
   v.n_layers = c->n_layers; v.batch = c->batch; v.n_kv_heads = c->n_kv_heads; v.n_q_heads = c->n_q_heads;
   v.capacity = c->capacity;
   v.fmt = c->meta_format;
+  v.sched = c->schedule;
   v.records = static_cast<unsigned char*>(c->records);
   v.modality = c->modality;
   v.k_tail = static_cast<__half*>(c->k_tail);

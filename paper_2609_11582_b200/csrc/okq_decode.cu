@@ -226,8 +226,8 @@ __global__ void __launch_bounds__(128) k_decode_simt(DecodeParams P) {
 
   // raw fp16 tail: last split, warp 0
   if (split == P.n_splits - 1 && warp == 0 && n_tail > 0) {
-    const __half* kt = cv.k_tail + cv.tail_off(layer, b, h);
-    const __half* vt = cv.v_tail + cv.tail_off(layer, b, h);
+    const __half* kt = cv.k_tail + cv.k_tail_off(layer, b, h);
+    const __half* vt = cv.v_tail + cv.v_tail_off(layer, b, h);
     float s[GP];
 #pragma unroll
     for (int j = 0; j < GP; j++) s[j] = 0.f;
@@ -510,6 +510,7 @@ okq_status okq_decode_attention_simt(const okq_cache* cache, int32_t layer, int3
                                      void* stream) {
   okq_status st = check_decode(cache, layer, layer_count, q, signs, R, n_R, workspace, workspace_bytes, num_splits, out);
   if (st != OKQ_OK) return st;
+  if (cache->schedule != OKQ_SCHEDULE_WINDOW) return OKQ_ERR_UNSUPPORTED;   // the cross-check kernels know one schedule
   DecodeParams P = make_params(cache, layer, layer_count, q, sm_scale, signs, R, n_R, out);
   P.n_splits = num_splits > 0 ? num_splits : auto_splits(cache, layer_count);
   P.partials = static_cast<Partial*>(workspace);

@@ -512,22 +512,37 @@ constexpr int CB_ROWS = CB_SEQ * GP;      // (sequence, head) rows per combine C
 
 constexpr int CB_CHUNK = 32;              // rows of a rotation matrix staged per step
 
+// CAPTION: the captioning schedule keeps up to 159 raw values (and up to 127 raw keys) per sequence, and
+// the keys of the raw values' tokens may already be packed
+template <bool CAPTION>
 struct CombineSmem {
+  static constexpr int TAIL = CAPTION ? CAPTION_V_SLOTS : W;   // most raw-value tokens of a sequence
   __align__(16) float Rbuf[2][CB_CHUNK][D];   // double-buffered 32-row slices of the rotation matrices
   __align__(16) float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
   __align__(16) float rawv[CB_ROWS][D];       // raw-tail contribution, [row][channel]
-  float tsc[CB_SEQ][W][GP];     // tail scores (log2 domain)
+  // q' = H q in the order of the (m, s) planes, for the scores of packed keys: [0] multiplies s * code, [1] the
+  // stored m (divided by the m plane's position scale when that plane carries it)
+  __align__(16) float qrot[2][CAPTION ? CB_ROWS : 1][D];
+  __align__(16) float tsc[CB_SEQ][TAIL][GP];  // tail scores (log2 domain), then softmax numerators
   float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
   int prefix[MAX_ENTRIES + 1];
 };
 
-// grid (n_kv_heads, ceil(batch / CB_SEQ), layer_count), 4 x 128 threads (group = sequence,
-// thread = channel): merge the partials of each (sequence, head), add the raw tail tokens, apply
-// R_m^T (the four groups read the same matrix elements, so they come from L1 after the first
-// touch) and normalise.
+// (stored m, s) at position p of a window's (m, s) planes, from its metadata in either format; the fp16 format's
+// m carries its position scale, the MXFP4 format decodes to the plain value
+__device__ __forceinline__ float2 window_meta_pos(const unsigned char* meta, int fmt, int p) {
+  if (fmt == FMT_FP16)
+    return make_float2(__half2float(reinterpret_cast<const __half*>(meta + OFF_KM)[p]),
+                       __half2float(reinterpret_cast<const __half*>(meta + OFF_KS)[p]));
+  const unsigned mn = (meta[p >> 1] >> (4 * (p & 1))) & 15u, sn = (meta[64 + (p >> 1)] >> (4 * (p & 1))) & 15u;
+  const int blk = (p >> 3) & 3;
+  return make_float2(mx_decode(mn, (int)meta[128 + blk] - 127), mx_decode(sn, (int)meta[132 + blk] - 127));
+}
+
+template <bool CAPTION>
 __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, int n_cta) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  CombineSmem& sm = *reinterpret_cast<CombineSmem*>(smem_raw);
+  CombineSmem<CAPTION>& sm = *reinterpret_cast<CombineSmem<CAPTION>*>(smem_raw);
   const CacheView& cv = P.cv;
   const int h = blockIdx.x, li = blockIdx.z, layer = P.layer0 + li;
   const int bs = threadIdx.x >> 7, c = threadIdx.x & 127;
@@ -548,38 +563,90 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
 
   const int e = li * cv.batch + bb;
   const int seq = live ? cv.seq_len[layer * cv.batch + bb] : 0;
-  const int nwin = seq / W, n_tail = seq - nwin * W;
+  // tokens [0, v_pk) have packed values (and keys): they are in the split-K partials; tokens [v_pk, seq) have raw
+  // values; of those, [v_pk, k_pk) have packed keys (captioning schedule only), the rest raw keys
+  const int v_pk = cv.v_packed(seq), k_pk = cv.k_packed(seq);
+  const int nwin = v_pk / W, n_tail = seq - v_pk;
   const int unit = e * Hkv + h;
   const int start = sm.prefix[e] + h * nwin, end = start + nwin;
   const int cta_lo = nwin > 0 ? start / per : 0, cta_hi = nwin > 0 ? (end - 1) / per : -1;
   const __half* qbase = P.q + (((size_t)li * cv.batch + bb) * cv.n_q_heads + h * G) * D;
-  const __half* kt = cv.k_tail + cv.tail_off(layer, bb, h);
-  const __half* vt = cv.v_tail + cv.tail_off(layer, bb, h);
-  // tail scores: thread -> (token = c & 31, heads (c >> 5) * 2 + {0, 1})
-  {
-    const int tok = c & 31;
+  const __half* kt = cv.k_tail + cv.k_tail_off(layer, bb, h);
+  const __half* vt = cv.v_tail + cv.v_tail_off(layer, bb, h);
+  if (CAPTION) {   // q' = H q for the scores of packed keys: one warp per (sequence, head) row
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int row = warp; row < CB_ROWS; row += CB_SEQ * 4) {
+      const int rb = blockIdx.y * CB_SEQ + row / GP, j = row % GP;
+      float4 qr = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (rb < cv.batch && j < G) {
+        const float4 x = load_row4(P.q + (((size_t)li * cv.batch + rb) * cv.n_q_heads + h * G + j) * D, lane);
+        const float4 sg = *reinterpret_cast<const float4*>(P.signs + (size_t)li * D + 4 * lane);
+        qr = warp_fwht(make_float4(x.x * sg.x, x.y * sg.y, x.z * sg.z, x.w * sg.w), lane);
+      }
+      const float v4[4] = {qr.x * RSQRT_D, qr.y * RSQRT_D, qr.z * RSQRT_D, qr.w * RSQRT_D};
 #pragma unroll
-    for (int hh = 0; hh < 2; hh++) {
-      const int j = (c >> 5) * 2 + hh;
-      float s = -INFINITY;
-      if (tok < n_tail && j < G) {
-        float a = 0.f;
+      for (int u = 0; u < 4; u++) {
+        const int ch = 4 * lane + u, pp = meta_pos(ch);
+        sm.qrot[0][row][pp] = v4[u];
+        sm.qrot[1][row][pp] = cv.fmt == FMT_FP16 ? v4[u] * (1.0f / (float)(1 << (2 * meta_shift(ch)))) : v4[u];
+      }
+    }
+    __syncthreads();
+  }
+  // tail scores: thread -> (token = c & 31 of a 32-token chunk, heads (c >> 5) * 2 + {0, 1})
+  for (int chunk = 0; chunk * W < n_tail; chunk++) {
+    const int tok = chunk * W + (c & 31), t = v_pk + tok;
+    float s2[2] = {-INFINITY, -INFINITY};
+    const int j0 = (c >> 5) * 2;
+    if (tok < n_tail && j0 < G) {
+      float a2[2] = {0.f, 0.f};
+      if (!CAPTION || t >= k_pk) {   // raw key
+        const __half* krow = kt + cv.k_slot(t) * D;
         for (int k = 0; k < D; k += 8) {
-          const uint4 qv = *reinterpret_cast<const uint4*>(qbase + j * D + k);
-          const uint4 kv = *reinterpret_cast<const uint4*>(kt + tok * D + k);
-          const __half2* q2 = reinterpret_cast<const __half2*>(&qv);
+          const uint4 kv = *reinterpret_cast<const uint4*>(krow + k);
           const __half2* k2 = reinterpret_cast<const __half2*>(&kv);
 #pragma unroll
-          for (int u = 0; u < 4; u++) {
-            const float2 qf = __half22float2(q2[u]), kf = __half22float2(k2[u]);
-            a = fmaf(qf.x, kf.x, a);
-            a = fmaf(qf.y, kf.y, a);
+          for (int hh = 0; hh < 2; hh++) {
+            if (j0 + hh >= G) continue;
+            const uint4 qv = *reinterpret_cast<const uint4*>(qbase + (j0 + hh) * D + k);
+            const __half2* q2 = reinterpret_cast<const __half2*>(&qv);
+#pragma unroll
+            for (int u = 0; u < 4; u++) {
+              const float2 qf = __half22float2(q2[u]), kf = __half22float2(k2[u]);
+              a2[hh] = fmaf(qf.x, kf.x, a2[hh]);
+              a2[hh] = fmaf(qf.y, kf.y, a2[hh]);
+            }
           }
         }
-        s = a * P.sm_scale * LOG2E;
+      } else {   // packed key: q . k_hat = norm * sum_c q'_c (m_c + s_c code_c)
+        // the 16 codes of word (tt, ww) of a token belong to the consecutive positions 32 tt + 16 ww .. + 15 of
+        // the (m, s) planes
+        const int win = t / W, ti = t % W;
+        const unsigned char* meta = cv.meta(layer, bb, h, win);
+        const unsigned char* body = cv.body(layer, bb, h, win);
+        const uint32_t* kw = reinterpret_cast<const uint32_t*>(body + B_KCODE) + (ti >> 4) * 128 + (ti & 7) * 16 + ((ti >> 3) & 1) * 2;
+        const int r0 = bs * GP + j0, r1 = bs * GP + min(j0 + 1, GP - 1);
+        for (int wi = 0; wi < 8; wi++) {
+          const int tt = wi >> 1, ww = wi & 1, p0 = 32 * tt + 16 * ww;
+          const uint32_t word = kw[tt * 4 + ww];
+#pragma unroll
+          for (int qq = 0; qq < 8; qq++)
+#pragma unroll
+            for (int e2 = 0; e2 < 2; e2++) {
+              const int pp = p0 + 2 * qq + e2;
+              const float2 ms = window_meta_pos(meta, cv.fmt, pp);
+              const float sc = ms.y * (float)((word >> (16 * e2 + 8 * (qq >> 2) + 2 * (qq & 3))) & 3u);
+              a2[0] = fmaf(sm.qrot[0][r0][pp], sc, fmaf(sm.qrot[1][r0][pp], ms.x, a2[0]));
+              a2[1] = fmaf(sm.qrot[0][r1][pp], sc, fmaf(sm.qrot[1][r1][pp], ms.x, a2[1]));
+            }
+        }
+        const float kn = __half2float(reinterpret_cast<const __half*>(body + B_KNORM)[norm_pos(ti)]);
+        a2[0] *= kn; a2[1] *= kn;
       }
-      sm.tsc[bs][tok][j] = s;
+      s2[0] = a2[0] * P.sm_scale * LOG2E;
+      if (j0 + 1 < G) s2[1] = a2[1] * P.sm_scale * LOG2E;
     }
+    if (tok < sm.TAIL) { sm.tsc[bs][tok][j0] = s2[0]; sm.tsc[bs][tok][j0 + 1] = s2[1]; }
   }
   __syncthreads();
   if (c < GP) {
@@ -596,9 +663,29 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
     sm.Ls[bs][c] = L;
   }
   __syncthreads();
+  // raw-value tokens: softmax numerators in place of the scores, then every value row is read once for all heads
+  for (int idx = c; idx < n_tail * GP; idx += 128) {
+    const int i = idx / GP, j = idx % GP;
+    sm.tsc[bs][i][j] = exp2f(sm.tsc[bs][i][j] - sm.Ms[bs][j]);   // 0 for the heads beyond the group (-inf scores)
+  }
+  __syncthreads();
+  float araw[GP];
+#pragma unroll
+  for (int j = 0; j < GP; j++) araw[j] = 0.f;
+#pragma unroll 4
+  for (int i = 0; i < n_tail; i++) {
+    const float x = __half2float(vt[cv.v_slot(v_pk + i) * D + c]);
+    const float4 w0 = *reinterpret_cast<const float4*>(&sm.tsc[bs][i][0]);
+    const float4 w1 = *reinterpret_cast<const float4*>(&sm.tsc[bs][i][4]);
+    araw[0] = fmaf(w0.x, x, araw[0]); araw[1] = fmaf(w0.y, x, araw[1]);
+    araw[2] = fmaf(w0.z, x, araw[2]); araw[3] = fmaf(w0.w, x, araw[3]);
+    araw[4] = fmaf(w1.x, x, araw[4]); araw[5] = fmaf(w1.y, x, araw[5]);
+    araw[6] = fmaf(w1.z, x, araw[6]); araw[7] = fmaf(w1.w, x, araw[7]);
+  }
 #pragma unroll
   for (int j = 0; j < GP; j++) {
-    float v[3] = {0.f, 0.f, 0.f}, a = 0.f;
+    float v[3] = {0.f, 0.f, 0.f};
+    const float a = araw[j];
     if (j < G) {
       const float M = sm.Ms[bs][j];
       const int r = 4 * (c >> 4) + 2 * ((c >> 3) & 1) + (j & 1), l32 = 4 * (c & 7) + (j >> 1);
@@ -613,7 +700,6 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
           v[m] = fmaf(fmaf(ACC_SCALE, pp.frag[m][r][l32], S_COEF * S), ef, v[m]);
         }
       }
-      for (int i = 0; i < n_tail; i++) a = fmaf(exp2f(sm.tsc[bs][i][j] - M), __half2float(vt[i * D + c]), a);
     }
     sm.vec[0][bs * GP + j][c] = v[0];
     sm.vec[1][bs * GP + j][c] = v[1];
@@ -695,7 +781,9 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
       e = cudaFuncSetAttribute(k_decode_mma<FMT_MXFP4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)sizeof(MmaSmem<FMT_MXFP4>));
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_combine_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem));
+      e = cudaFuncSetAttribute(k_combine_mma<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<false>));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_combine_mma<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<true>));
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
     attr_done(attr_mask, attr_dev);
   }
@@ -703,8 +791,9 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
   if (P.cv.fmt == FMT_MXFP4) k_decode_mma<FMT_MXFP4><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_MXFP4>), s>>>(P);
   else k_decode_mma<FMT_FP16><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_FP16>), s>>>(P);
   if (after) cudaEventRecord(after, s);
-  k_combine_mma<<<dim3(P.cv.n_kv_heads, (P.cv.batch + CB_SEQ - 1) / CB_SEQ, P.layer_count), CB_SEQ * 128,
-                  sizeof(CombineSmem), s>>>(P, n_cta);
+  const dim3 cgrid(P.cv.n_kv_heads, (P.cv.batch + CB_SEQ - 1) / CB_SEQ, P.layer_count);
+  if (P.cv.sched == SCHED_CAPTION) k_combine_mma<true><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<true>), s>>>(P, n_cta);
+  else k_combine_mma<false><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<false>), s>>>(P, n_cta);
   return OKQ_OK;
 }
 

@@ -45,7 +45,7 @@ __device__ inline int block_prefix(const CacheView& cv, int layer0, int n_entrie
     const int chunk = (n_entries + 31) / 32;
     const int e0 = min(n_entries, lane * chunk), e1 = min(n_entries, e0 + chunk);
     int sum = 0;
-    for (int e = e0; e < e1; e++) sum += (cv.seq_len[(size_t)layer0 * cv.batch + e] / W) * cv.n_kv_heads;
+    for (int e = e0; e < e1; e++) sum += (cv.v_packed(cv.seq_len[(size_t)layer0 * cv.batch + e]) / W) * cv.n_kv_heads;
     int incl = sum;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -55,7 +55,7 @@ __device__ inline int block_prefix(const CacheView& cv, int layer0, int n_entrie
     int run = incl - sum;
     for (int e = e0; e < e1; e++) {
       prefix[e] = run;
-      run += (cv.seq_len[(size_t)layer0 * cv.batch + e] / W) * cv.n_kv_heads;
+      run += (cv.v_packed(cv.seq_len[(size_t)layer0 * cv.batch + e]) / W) * cv.n_kv_heads;
     }
     if (lane == 31) prefix[n_entries] = incl;
   }

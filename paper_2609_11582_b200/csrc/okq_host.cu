@@ -26,6 +26,7 @@ okq_status check_cache(const okq_cache* c, bool need_ptrs) {
     return OKQ_ERR_INVALID_ARG;
   if (c->capacity % OKQ_WINDOW != 0) return OKQ_ERR_INVALID_ARG;
   if (c->meta_format != OKQ_META_FP16 && c->meta_format != OKQ_META_MXFP4) return OKQ_ERR_UNSUPPORTED;
+  if (c->schedule != OKQ_SCHEDULE_WINDOW && c->schedule != OKQ_SCHEDULE_CAPTION) return OKQ_ERR_UNSUPPORTED;
   if (c->n_q_heads % c->n_kv_heads != 0 || c->n_q_heads / c->n_kv_heads > OKQ_MAX_GROUP) return OKQ_ERR_UNSUPPORTED;
   if (need_ptrs) {
     if (!c->records || !c->modality || !c->k_tail || !c->v_tail || !c->seq_len || !c->status)
@@ -62,16 +63,15 @@ okq_status okq_cache_sizes(const okq_cache* c, size_t out[6]) {
   if (st != OKQ_OK) return st;
   if (!out) return OKQ_ERR_INVALID_ARG;
   size_t units = (size_t)c->n_layers * c->batch * c->n_kv_heads;
-  {
-    okq::CacheView v{};
-    v.capacity = c->capacity;
-    v.fmt = c->meta_format;
-    out[0] = units * v.unit_bytes();
-  }
+  okq::CacheView v{};
+  v.capacity = c->capacity;
+  v.fmt = c->meta_format;
+  v.sched = c->schedule;
+  out[0] = units * v.unit_bytes();
   out[0] = (out[0] + 15) & ~(size_t)15;
   out[1] = (size_t)c->batch * c->capacity;
-  out[2] = units * OKQ_WINDOW * OKQ_HEAD_DIM * 2;
-  out[3] = out[2];
+  out[2] = units * (size_t)v.k_slots() * OKQ_HEAD_DIM * 2;
+  out[3] = units * (size_t)v.v_slots() * OKQ_HEAD_DIM * 2;
   out[4] = (size_t)c->n_layers * c->batch * sizeof(int32_t);
   out[5] = 16;
   return OKQ_OK;

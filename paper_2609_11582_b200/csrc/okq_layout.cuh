@@ -96,9 +96,14 @@ __host__ __device__ inline size_t mx_body_off(size_t win) {
   return (win >> 1) * MX_PAIR_BYTES + 2 * MX_META_BYTES + (win & 1) * BODY_BYTES;
 }
 
+constexpr int SCHED_WINDOW = 0, SCHED_CAPTION = 1;
+constexpr int CAPTION_K_GROUP = 128;    // keys are packed every 128 tokens
+constexpr int CAPTION_V_LAG = 128;      // values stay raw for 128 tokens
+constexpr int CAPTION_V_SLOTS = CAPTION_V_LAG + W;   // ring of raw values: 128 .. 159 live tokens
+
 struct CacheView {
   int n_layers, batch, n_kv_heads, n_q_heads, capacity;
-  int fmt;
+  int fmt, sched;
   unsigned char* records;
   unsigned char* modality;
   __half* k_tail;
@@ -119,8 +124,23 @@ struct CacheView {
   __host__ __device__ inline unsigned char* body(int layer, int b, int h, size_t win) const {
     return unit(layer, b, h) + (fmt == FMT_MXFP4 ? mx_body_off(win) : win * RECORD_BYTES + META_BYTES_FP16);
   }
-  __host__ __device__ inline size_t tail_off(int layer, int b, int h) const {
-    return (((size_t)layer * batch + b) * n_kv_heads + h) * (size_t)(W * D);
+  // raw-token slots per (layer, sequence, head), number of packed tokens of a sequence of n tokens, and
+  // the slot of raw token t, for keys and for values
+  __host__ __device__ inline int k_slots() const { return sched == SCHED_CAPTION ? CAPTION_K_GROUP : W; }
+  __host__ __device__ inline int v_slots() const { return sched == SCHED_CAPTION ? CAPTION_V_SLOTS : W; }
+  __host__ __device__ inline int k_packed(int n) const {
+    return sched == SCHED_CAPTION ? n - n % CAPTION_K_GROUP : n - n % W;
+  }
+  __host__ __device__ inline int v_packed(int n) const {
+    return sched == SCHED_CAPTION ? (n >= CAPTION_V_LAG ? (n - CAPTION_V_LAG) - (n - CAPTION_V_LAG) % W : 0) : n - n % W;
+  }
+  __host__ __device__ inline int k_slot(int t) const { return t % k_slots(); }
+  __host__ __device__ inline int v_slot(int t) const { return t % v_slots(); }
+  __host__ __device__ inline size_t k_tail_off(int layer, int b, int h) const {
+    return (((size_t)layer * batch + b) * n_kv_heads + h) * (size_t)(k_slots() * D);
+  }
+  __host__ __device__ inline size_t v_tail_off(int layer, int b, int h) const {
+    return (((size_t)layer * batch + b) * n_kv_heads + h) * (size_t)(v_slots() * D);
   }
 };
 

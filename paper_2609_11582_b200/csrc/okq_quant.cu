@@ -328,21 +328,23 @@ __global__ void __launch_bounds__(128) k_quantize_values(CacheView cv, int layer
   quantize_value_window(rows, st, Rset, cv.body(layer, b, h, win), sm);
 }
 
-// raw tail copy + seq_len (+ modality for the value call); grid (n_kv_heads, batch), 128 threads
+// raw tokens behind the packed ones + seq_len (+ modality for the value call); grid (n_kv_heads, batch, slices),
+// 128 threads.  Token t goes to slot t mod (slots of the schedule).
 __global__ void k_bulk_tail(CacheView cv, int layer, const __half* __restrict__ src, long long sb, long long sh,
-                            long long st, int n_tokens, __half* tail, const unsigned char* __restrict__ modality) {
+                            long long st, int n_tokens, int is_value, const unsigned char* __restrict__ modality) {
   const int h = blockIdx.x, b = blockIdx.y;
-  if (blockIdx.z == 0) {
-    const int n_packed = n_tokens & ~(W - 1);
-    const int n_tail = n_tokens - n_packed;
-    __half* dst = tail + cv.tail_off(layer, b, h);
-    for (int idx = threadIdx.x; idx < n_tail * (D / 8); idx += blockDim.x) {
-      int i = idx / (D / 8), c8 = idx % (D / 8);
-      reinterpret_cast<uint4*>(dst + i * D)[c8] =
-          *reinterpret_cast<const uint4*>(src + b * sb + h * sh + (long long)(n_packed + i) * st + c8 * 8);
-    }
-    if (h == 0 && threadIdx.x == 0) cv.seq_len[layer * cv.batch + b] = n_tokens;
+  const int n_packed = is_value ? cv.v_packed(n_tokens) : cv.k_packed(n_tokens);
+  const int n_tail = n_tokens - n_packed;
+  __half* dst = is_value ? cv.v_tail + cv.v_tail_off(layer, b, h) : cv.k_tail + cv.k_tail_off(layer, b, h);
+  const int per = (n_tail + gridDim.z - 1) / gridDim.z;      // tokens per slice
+  const int i0 = blockIdx.z * per, i1 = min(n_tail, i0 + per);
+  for (int idx = i0 * (D / 8) + threadIdx.x; idx < i1 * (D / 8); idx += blockDim.x) {
+    const int t = n_packed + idx / (D / 8), c8 = idx % (D / 8);
+    const int slot = is_value ? cv.v_slot(t) : cv.k_slot(t);
+    reinterpret_cast<uint4*>(dst + slot * D)[c8] =
+        *reinterpret_cast<const uint4*>(src + b * sb + h * sh + (long long)t * st + c8 * 8);
   }
+  if (blockIdx.z == 0 && h == 0 && threadIdx.x == 0) cv.seq_len[layer * cv.batch + b] = n_tokens;
   if (modality) {   // the sequence's modality bytes, spread over the (head, slice) blocks of the sequence
     const int stride = gridDim.x * gridDim.z * blockDim.x;
     for (int i = (h * gridDim.z + blockIdx.z) * blockDim.x + threadIdx.x; i < n_tokens; i += stride) {
@@ -367,29 +369,37 @@ __global__ void __launch_bounds__(128) k_append(CacheView cv, int layer0, const 
     if (threadIdx.x == 0) atomicCAS(cv.status, 0, (int)OKQ_ERR_CAPACITY);
     return;
   }
-  int slot = pos & (W - 1);
   size_t src = (((size_t)li * cv.batch + b) * cv.n_kv_heads + h) * D;
-  __half* kt = cv.k_tail + cv.tail_off(layer, b, h);
-  __half* vt = cv.v_tail + cv.tail_off(layer, b, h);
+  __half* kt = cv.k_tail + cv.k_tail_off(layer, b, h);
+  __half* vt = cv.v_tail + cv.v_tail_off(layer, b, h);
   unsigned char mnew = mod_new[b];
   mnew = mnew > 2 ? 0 : mnew;
-  if (threadIdx.x < 16) reinterpret_cast<uint4*>(kt + slot * D)[threadIdx.x] = reinterpret_cast<const uint4*>(k_new + src)[threadIdx.x];
-  else if (threadIdx.x < 32) reinterpret_cast<uint4*>(vt + slot * D)[threadIdx.x - 16] = reinterpret_cast<const uint4*>(v_new + src)[threadIdx.x - 16];
+  const int kslot = cv.k_slot(pos), vslot = cv.v_slot(pos);
+  if (threadIdx.x < 16) reinterpret_cast<uint4*>(kt + kslot * D)[threadIdx.x] = reinterpret_cast<const uint4*>(k_new + src)[threadIdx.x];
+  else if (threadIdx.x < 32) reinterpret_cast<uint4*>(vt + vslot * D)[threadIdx.x - 16] = reinterpret_cast<const uint4*>(v_new + src)[threadIdx.x - 16];
   if (h == 0 && threadIdx.x == 32) cv.modality[(size_t)b * cv.capacity + pos] = mnew;
-  if (slot != W - 1) return;
-  __syncthreads();  // the 32nd token of the window is now visible to the whole block
-  unsigned char* body = cv.body(layer, b, h, pos / W);
-  quantize_key_window(kt, D, signs + (size_t)li * D, cv.meta(layer, b, h, pos / W), body, cv.fmt, sm);
-  if (threadIdx.x < 32) {
-    unsigned char m = threadIdx.x == W - 1 ? mnew : cv.modality[(size_t)b * cv.capacity + (pos - (W - 1)) + threadIdx.x];
-    sm.mod[threadIdx.x] = m;
-    unsigned char m0 = __shfl_sync(0xffffffffu, m, 0);
-    int uni = __all_sync(0xffffffffu, m == m0);
-    if (threadIdx.x == 0) sm.uniform = uni;
-  }
-  __syncthreads();
+  // windows that the schedule packs now that the sequence holds pos + 1 tokens
+  const int kw0 = cv.k_packed(pos) / W, kw1 = cv.k_packed(pos + 1) / W;
+  const int vw0 = cv.v_packed(pos) / W, vw1 = cv.v_packed(pos + 1) / W;
+  if (kw0 == kw1 && vw0 == vw1) return;
+  __syncthreads();  // the new token is now visible to the whole block
+  for (int win = kw0; win < kw1; win++)   // the window's 32 raw keys sit in consecutive slots
+    quantize_key_window(kt + cv.k_slot(win * W) * D, D, signs + (size_t)li * D, cv.meta(layer, b, h, win),
+                        cv.body(layer, b, h, win), cv.fmt, sm);
   const float* Rset = R + ((size_t)li * n_R + (n_R == 1 ? 0 : h)) * 3 * D * D;
-  quantize_value_window(vt, D, Rset, body, sm);
+  for (int win = vw0; win < vw1; win++) {
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      const int t = win * W + threadIdx.x;   // the newest token's modality may not have reached global memory yet
+      unsigned char m = t == pos ? mnew : cv.modality[(size_t)b * cv.capacity + t];
+      sm.mod[threadIdx.x] = m;
+      unsigned char m0 = __shfl_sync(0xffffffffu, m, 0);
+      int uni = __all_sync(0xffffffffu, m == m0);
+      if (threadIdx.x == 0) sm.uniform = uni;
+    }
+    __syncthreads();
+    quantize_value_window(vt + cv.v_slot(win * W) * D, D, Rset, cv.body(layer, b, h, win), sm);
+  }
 }
 
 __global__ void k_advance(CacheView cv, int layer0, int layer_count) {
@@ -489,7 +499,7 @@ __global__ void k_import(CacheView cv, int layer, const unsigned char* k_codes, 
 }
 
 okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __half* v, const int64_t strides[3],
-                                     const unsigned char* modality, int n_tokens, const float* R, int n_R,
+                                     const unsigned char* modality, int n_tokens, int n_win, const float* R, int n_R,
                                      int n_sm, cudaStream_t s);
 
 constexpr int TAIL_SLICES = 16;   // blocks per (sequence, head) that share the copy of the modality bytes
@@ -520,13 +530,13 @@ okq_status okq_quantize_keys(const okq_cache* cache, int32_t layer, const void* 
   CacheView cv = make_view(cache);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __half* k = static_cast<const __half*>(k_fp16);
-  int n_win = n_tokens / W;
+  int n_win = cv.k_packed(n_tokens) / W;
   if (n_win > 0) {
     dim3 grid(n_win, cv.n_kv_heads, cv.batch);
     k_quantize_keys<<<grid, 128, 0, s>>>(cv, layer, k, strides[0], strides[1], strides[2], signs);
   }
-  k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch), 128, 0, s>>>(cv, layer, k, strides[0], strides[1], strides[2],
-                                                           n_tokens, cv.k_tail, nullptr);
+  k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch, 1), 128, 0, s>>>(cv, layer, k, strides[0], strides[1], strides[2],
+                                                              n_tokens, 0, nullptr);
   return launch_status();
 }
 
@@ -541,14 +551,14 @@ okq_status okq_quantize_values(const okq_cache* cache, int32_t layer, const void
   CacheView cv = make_view(cache);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __half* v = static_cast<const __half*>(v_fp16);
-  int n_win = n_tokens / W;
+  int n_win = cv.v_packed(n_tokens) / W;
   if (n_win > 0) {
     dim3 grid(n_win, cv.n_kv_heads, cv.batch);
     k_quantize_values<<<grid, 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2], modality, n_tokens, R,
                                            n_R);
   }
   k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch, TAIL_SLICES), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
-                                                                        n_tokens, cv.v_tail, n_tokens > 0 ? modality : nullptr);
+                                                                        n_tokens, 1, n_tokens > 0 ? modality : nullptr);
   return launch_status();
 }
 
@@ -563,10 +573,10 @@ okq_status okq_quantize_values_bulk(const okq_cache* cache, int32_t layer, const
   CacheView cv = make_view(cache);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const __half* v = static_cast<const __half*>(v_fp16);
-  st = launch_quantize_values_tc(cv, layer, v, strides, modality, n_tokens, R, n_R, sm_count(), s);
+  st = launch_quantize_values_tc(cv, layer, v, strides, modality, n_tokens, cv.v_packed(n_tokens) / W, R, n_R, sm_count(), s);
   if (st != OKQ_OK) return st;
   k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch, TAIL_SLICES), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
-                                                                        n_tokens, cv.v_tail, n_tokens > 0 ? modality : nullptr);
+                                                                        n_tokens, 1, n_tokens > 0 ? modality : nullptr);
   return launch_status();
 }
 

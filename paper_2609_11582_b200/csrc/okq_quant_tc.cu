@@ -183,12 +183,11 @@ struct Slots {
 // (one accumulator of 128 columns each); jobs alternate between two accumulator sets in tensor memory.
 __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_constant__ CUtensorMap vmap, CacheView cv, int layer,
                                                              const unsigned char* __restrict__ modality, int n_tokens,
-                                                             const float* __restrict__ R, int n_R) {
+                                                             int n_win, const float* __restrict__ R, int n_R) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   TcSmem& sm = *reinterpret_cast<TcSmem*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_win = n_tokens / W;
-  const int tiles_per_unit = (n_win + 3) / 4;
+  const int tiles_per_unit = (n_win + 3) / 4;   // n_win: windows to pack (the schedule may keep recent tokens raw)
   const int n_tiles_all = tiles_per_unit * cv.n_kv_heads * cv.batch;
   // contiguous tile range of this CTA
   const int per_cta = (n_tiles_all + gridDim.x - 1) / gridDim.x;
@@ -508,7 +507,7 @@ EncodeTiledFn encode_tiled() {
 }  // namespace
 
 okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __half* v, const int64_t strides[3],
-                                     const unsigned char* modality, int n_tokens, const float* R, int n_R,
+                                     const unsigned char* modality, int n_tokens, int n_win, const float* R, int n_R,
                                      int n_sm, cudaStream_t s) {
   static thread_local unsigned long long attr_mask = 0;
   int attr_dev = 0;
@@ -518,7 +517,6 @@ okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __hal
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
     attr_done(attr_mask, attr_dev);
   }
-  const int n_win = n_tokens / W;
   const long long n_tiles = (long long)((n_win + 3) / 4) * cv.n_kv_heads * cv.batch;
   if (n_tiles == 0) return OKQ_OK;
   // the values as a 4-d tensor [batch][head][token][channel] for the copy engine; a box is 64 channels x 128 tokens
@@ -537,7 +535,7 @@ okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __hal
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) { set_last_cuda_error((int)cudaErrorInvalidValue); return OKQ_ERR_CUDA; }
   const int grid = (int)(n_tiles < n_sm ? n_tiles : n_sm);
-  k_quantize_values_tc<<<grid, NT_ALL, sizeof(TcSmem) + 1024, s>>>(vmap, cv, layer, modality, n_tokens, R, n_R);
+  k_quantize_values_tc<<<grid, NT_ALL, sizeof(TcSmem) + 1024, s>>>(vmap, cv, layer, modality, n_tokens, n_win, R, n_R);
   return OKQ_OK;
 }
 

@@ -50,7 +50,7 @@ def test_shape_validation(L):
         d = dict(n_layers=1, batch=1, n_kv_heads=1, n_q_heads=7, head_dim=128, window=32, capacity=64)
         d.update(kw)
         c = B.okq_cache(d["n_layers"], d["batch"], d["n_kv_heads"], d["n_q_heads"], d["head_dim"], d["window"],
-                        d["capacity"], 0)
+                        d["capacity"], 0, 0, 0)
         out = (C.c_size_t * 6)()
         return L.okq_cache_sizes(C.byref(c), out)
     assert sizes() == B.OK
@@ -63,11 +63,11 @@ def test_shape_validation(L):
 
 
 def test_pointer_validation_before_any_launch(L):
-    c = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, 0, 0, 0, 0, 0, 0)
+    c = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, 0, 0, 0, 0, 0, 0, 0, 0)
     strides = (C.c_int64 * 3)(64 * 128, 64 * 128, 128)
     assert L.okq_quantize_keys(C.byref(c), 0, 4096, strides, 64, 4096, None) == B.ERR_INVALID_ARG   # null buffers
     fake = 1 << 20
-    c = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, fake, fake, fake, fake, fake, fake)
+    c = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, 0, 0, fake, fake, fake, fake, fake, fake)
     assert L.okq_quantize_keys(C.byref(c), 1, fake, strides, 64, fake, None) == B.ERR_INVALID_ARG   # layer out of range
     assert L.okq_quantize_keys(C.byref(c), 0, fake, strides, 96, fake, None) == B.ERR_CAPACITY
     assert L.okq_quantize_keys(C.byref(c), 0, fake + 2, strides, 64, fake, None) == B.ERR_ALIGNMENT
@@ -78,7 +78,7 @@ def test_pointer_validation_before_any_launch(L):
     assert L.okq_decode_attention(C.byref(c), 0, 1, fake, 0.1, fake, fake, 1, fake, 16, 0, fake, None) == B.ERR_WORKSPACE
     assert L.okq_decode_workspace_bytes(C.byref(c), 1, 3) > 0
     assert L.okq_decode_workspace_bytes(C.byref(c), 0, 3) == 0
-    c8 = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, fake + 8, fake, fake, fake, fake, fake)
+    c8 = B.okq_cache(1, 1, 1, 7, 128, 32, 64, 0, 0, 0, fake + 8, fake, fake, fake, fake, fake)
     assert L.okq_append(C.byref(c8), 0, 1, fake, fake, fake, fake, fake, 1, None) == B.ERR_ALIGNMENT
 
 

@@ -1,0 +1,113 @@
+"""GPU parity of the captioning schedule (keys packed every 128 tokens, values behind a 128-token fp16
+window): cache state after bulk prefill and after token-by-token append, and decode attention against
+the oracle's definition, at lengths around every boundary of the schedule."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import okq_oracle as O
+from paper_2609_11582_b200 import binding as B
+from paper_2609_11582_b200 import workloads as WL
+from tests import harness as Hn
+
+pytestmark = pytest.mark.gpu
+D, W = 128, 32
+CAP = B.SCHEDULE_CAPTION
+
+
+def _inputs(n, batch=2, seed_layer=0):
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=batch)
+    k, v = WL.gen_kv(w, seed_layer, n_tokens=n)
+    mod = WL.modality_layout(w, n)
+    signs = WL.gen_signs(w, seed_layer)
+    R = WL.gen_rotations(w, seed_layer)
+    q = WL.gen_queries(w, seed_layer)
+    return w, k, v, mod, signs, R, q
+
+
+def _decode(cache, w, q, signs, R):
+    ws = torch.empty(max(16, B.decode_workspace_bytes(cache, 1, 0)), dtype=torch.uint8, device="cuda")
+    out = torch.full((1, w.batch, w.n_q_heads, D), float("nan"), dtype=torch.float32, device="cuda")
+    B.decode_attention(cache, 0, 1, q.cuda()[None], signs.cuda()[None], R.cuda()[None, None], ws, out)
+    torch.cuda.synchronize()
+    return out[0].cpu().numpy().astype(np.float64)
+
+
+def _oracle(w, k, v, mod, signs, R, q, n, meta_format):
+    kp, vp = O.packed_counts(n, 1)
+    ref = np.zeros((w.batch, w.n_q_heads, D))
+    G = w.group
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            kb = Hn.u16(k[b, h, :n]); vb = Hn.u16(v[b, h, :n])
+            kq, vq, _ = O.quantize_batch(kb[None], vb[None], mod.numpy()[:n], signs.numpy(), R.numpy(), meta_format=meta_format)
+            kq1 = {a: x[0] for a, x in kq.items()}; vq1 = {a: x[0] for a, x in vq.items()}
+            ref[b, h * G:(h + 1) * G] = O.attention_scheduled(Hn.u16(q[b, h * G:(h + 1) * G]), kq1, vq1, mod.numpy(), kb, vb,
+                                                              signs.numpy(), R.numpy(), kp, vp)
+    return ref
+
+
+def test_buffer_sizes():
+    s = B.cache_sizes(2, 3, 4, 28, 1024, schedule=CAP)
+    units = 2 * 3 * 4
+    assert s[2] == units * 128 * D * 2 and s[3] == units * 160 * D * 2          # raw key / value slots
+    assert s[0] == B.cache_sizes(2, 3, 4, 28, 1024)[0]                            # the records do not change
+
+
+@pytest.mark.parametrize("n", [5, 127, 128, 159, 160, 255, 256, 300, 1024 + 77])
+@pytest.mark.parametrize("meta_format", [B.META_FP16, B.META_MXFP4])
+def test_bulk_prefill_then_decode(n, meta_format):
+    w, k, v, mod, signs, R, q = _inputs(n)
+    cache = B.Cache(1, w.batch, w.n_kv_heads, w.n_q_heads, ((n + 31) // 32 + 2) * 32, meta_format=meta_format, schedule=CAP)
+    modb = mod[None].repeat(w.batch, 1).contiguous().cuda()
+    B.quantize_keys(cache, 0, k.cuda(), signs.cuda())
+    B.quantize_values(cache, 0, v.cuda(), modb, R.cuda()[None], bulk=(n % 2 == 0))   # both value quantisers
+    torch.cuda.synchronize()
+    assert cache.device_status() == 0 and cache.seq_len.cpu().tolist() == [n] * w.batch
+    got = _decode(cache, w, q, signs, R)
+    ref = _oracle(w, k, v, mod, signs, R, q, n, meta_format)
+    print(f"n={n} meta {meta_format}:", Hn.assert_attention_close(got, ref))
+    # the cross-check kernels know the window schedule only
+    ws = torch.empty(max(16, B.decode_workspace_bytes(cache, 1, 0)), dtype=torch.uint8, device="cuda")
+    out = torch.empty(1, w.batch, w.n_q_heads, D, dtype=torch.float32, device="cuda")
+    with pytest.raises(B.OkqError) as ei:
+        B.decode_attention(cache, 0, 1, q.cuda()[None], signs.cuda()[None], R.cuda()[None, None], ws, out, simt=True)
+    assert ei.value.status == B.ERR_UNSUPPORTED
+
+
+def test_append_equals_bulk_and_decode_at_every_step():
+    """Token-by-token append under the captioning schedule: records, raw slots and lengths equal those of a bulk
+    prefill of the same tokens, and the decode output matches the oracle across the schedule's boundaries."""
+    n0, n1 = 100, 420
+    w, k, v, mod, signs, R, q = _inputs(n1)
+    cap = 448
+    part = B.Cache(1, w.batch, w.n_kv_heads, w.n_q_heads, cap, schedule=CAP)
+    modb = mod[None].repeat(w.batch, 1).contiguous().cuda()
+    kd, vd = k.cuda(), v.cuda()
+    B.quantize_keys(part, 0, kd[:, :, :n0].contiguous(), signs.cuda())
+    B.quantize_values(part, 0, vd[:, :, :n0].contiguous(), modb[:, :n0].contiguous(), R.cuda()[None])
+    check_at = {127, 128, 129, 159, 160, 161, 255, 256, 288, 319, 320, 384, n1}
+    for i in range(n0, n1):
+        B.append(part, 0, 1, kd[:, :, i].contiguous()[None], vd[:, :, i].contiguous()[None], modb[:, i].contiguous(),
+                 signs.cuda()[None], R.cuda()[None, None])
+        n = i + 1
+        if n in check_at:
+            torch.cuda.synchronize()
+            assert part.device_status() == 0 and part.seq_len.cpu().tolist() == [n] * w.batch
+            full = B.Cache(1, w.batch, w.n_kv_heads, w.n_q_heads, cap, schedule=CAP)
+            B.quantize_keys(full, 0, kd[:, :, :n].contiguous(), signs.cuda())
+            B.quantize_values(full, 0, vd[:, :, :n].contiguous(), modb[:, :n].contiguous(), R.cuda()[None])
+            kp, vp = O.packed_counts(n, 1)
+            ea, eb = B.cache_export(part, 0), B.cache_export(full, 0)
+            for key, lim in (("k_codes", kp), ("k_norm", kp), ("k_meta", kp // W), ("v_codes", vp), ("v_norm", vp)):
+                assert torch.equal(ea[key][:, :, :lim], eb[key][:, :, :lim]), (n, key)
+            U = w.batch * w.n_kv_heads
+            kt_a, kt_b = part.k_tail.view(U, 128, D), full.k_tail.view(U, 128, D)
+            vt_a, vt_b = part.v_tail.view(U, 160, D), full.v_tail.view(U, 160, D)
+            ks = torch.tensor([t % 128 for t in range(kp, n)], dtype=torch.long, device="cuda")
+            vs = torch.tensor([t % 160 for t in range(vp, n)], dtype=torch.long, device="cuda")
+            assert torch.equal(kt_a[:, ks], kt_b[:, ks]) and torch.equal(vt_a[:, vs], vt_b[:, vs]), n
+            assert torch.equal(kt_a[:, ks].cpu(), k[:, :, kp:n].reshape(U, n - kp, D))
+            got = _decode(part, w, q, signs, R)
+            ref = _oracle(w, k, v, mod, signs, R, q, n, B.META_FP16)
+            Hn.assert_attention_close(got, ref)

@@ -25,7 +25,7 @@ D = 128
 
 def test_noalloc_rejects_oversized_request_without_a_gpu():
     # 48 layers x 16 sequences x 4 heads = 3072 partials + the CTAs: more than the 32 MiB scratch holds
-    c = B.okq_cache(48, 16, 4, 32, 128, 32, 32768, 0, 1 << 20, 1 << 20, 1 << 20, 1 << 20, 1 << 20, 1 << 20)
+    c = B.okq_cache(48, 16, 4, 32, 128, 32, 32768, 0, 0, 0, 1 << 20, 1 << 20, 1 << 20, 1 << 20, 1 << 20, 1 << 20)
     st = B.lib().okq_decode_attention_noalloc(C.byref(c), 0, 48, 1 << 20, 0.1, 1 << 20, 1 << 20, 1, 0, 1 << 20, None)
     assert st == B.ERR_WORKSPACE
     bad = B.okq_cache(1, 1, 1, 7, 64, 32, 64, 0)
