@@ -594,10 +594,18 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
     __syncthreads();
   }
   // tail scores: thread -> (token = c & 31 of a 32-token chunk, heads (c >> 5) * 2 + {0, 1})
+  float* msf = &sm.Rbuf[0][0][0] + bs * 2 * D;   // (m, s) of a packed window as floats (the slice buffer is idle here)
   for (int chunk = 0; chunk * W < n_tail; chunk++) {
     const int tok = chunk * W + (c & 31), t = v_pk + tok;
     float s2[2] = {-INFINITY, -INFINITY};
     const int j0 = (c >> 5) * 2;
+    // a chunk is one 32-token window: its keys are either all packed or all raw
+    const bool packed = CAPTION && v_pk + chunk * W < k_pk;
+    if (packed) {
+      const float2 ms = window_meta_pos(cv.meta(layer, bb, h, (v_pk + chunk * W) / W), cv.fmt, c);
+      msf[c] = ms.x; msf[D + c] = ms.y;
+      asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // the sequence's 128 threads
+    }
     if (tok < n_tail && j0 < G) {
       float a2[2] = {0.f, 0.f};
       if (!CAPTION || t >= k_pk) {   // raw key
@@ -622,7 +630,6 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
         // the 16 codes of word (tt, ww) of a token belong to the consecutive positions 32 tt + 16 ww .. + 15 of
         // the (m, s) planes
         const int win = t / W, ti = t % W;
-        const unsigned char* meta = cv.meta(layer, bb, h, win);
         const unsigned char* body = cv.body(layer, bb, h, win);
         const uint32_t* kw = reinterpret_cast<const uint32_t*>(body + B_KCODE) + (ti >> 4) * 128 + (ti & 7) * 16 + ((ti >> 3) & 1) * 2;
         const int r0 = bs * GP + j0, r1 = bs * GP + min(j0 + 1, GP - 1);
@@ -634,10 +641,10 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
 #pragma unroll
             for (int e2 = 0; e2 < 2; e2++) {
               const int pp = p0 + 2 * qq + e2;
-              const float2 ms = window_meta_pos(meta, cv.fmt, pp);
-              const float sc = ms.y * (float)((word >> (16 * e2 + 8 * (qq >> 2) + 2 * (qq & 3))) & 3u);
-              a2[0] = fmaf(sm.qrot[0][r0][pp], sc, fmaf(sm.qrot[1][r0][pp], ms.x, a2[0]));
-              a2[1] = fmaf(sm.qrot[0][r1][pp], sc, fmaf(sm.qrot[1][r1][pp], ms.x, a2[1]));
+              const float mv = msf[pp];
+              const float sc = msf[D + pp] * (float)((word >> (16 * e2 + 8 * (qq >> 2) + 2 * (qq & 3))) & 3u);
+              a2[0] = fmaf(sm.qrot[0][r0][pp], sc, fmaf(sm.qrot[1][r0][pp], mv, a2[0]));
+              a2[1] = fmaf(sm.qrot[0][r1][pp], sc, fmaf(sm.qrot[1][r1][pp], mv, a2[1]));
             }
         }
         const float kn = __half2float(reinterpret_cast<const __half*>(body + B_KNORM)[norm_pos(ti)]);
@@ -647,6 +654,7 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
       if (j0 + 1 < G) s2[1] = a2[1] * P.sm_scale * LOG2E;
     }
     if (tok < sm.TAIL) { sm.tsc[bs][tok][j0] = s2[0]; sm.tsc[bs][tok][j0 + 1] = s2[1]; }
+    if (packed) asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // before the next window's (m, s)
   }
   __syncthreads();
   if (c < GP) {
@@ -672,7 +680,7 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
   float araw[GP];
 #pragma unroll
   for (int j = 0; j < GP; j++) araw[j] = 0.f;
-#pragma unroll 4
+#pragma unroll 8
   for (int i = 0; i < n_tail; i++) {
     const float x = __half2float(vt[cv.v_slot(v_pk + i) * D + c]);
     const float4 w0 = *reinterpret_cast<const float4*>(&sm.tsc[bs][i][0]);
