@@ -510,14 +510,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
 constexpr int CB_SEQ = 4;                 // sequences per combine CTA (one 128-thread group each)
 constexpr int CB_ROWS = CB_SEQ * GP;      // (sequence, head) rows per combine CTA
 
-constexpr int CB_CHUNK = 32;              // rows of a rotation matrix staged per step
+constexpr int MRG_MAX = 8;                // partials per (sequence, head) whose factors are precomputed
+constexpr int CB_CHUNK = 16;              // rows of a rotation matrix staged per step
+constexpr int CB_NBUF = 4;                // staged slices in flight (three ahead of the one in use)
 
 // CAPTION: the captioning schedule keeps up to 159 raw values (and up to 127 raw keys) per sequence, and
 // the keys of the raw values' tokens may already be packed
 template <bool CAPTION>
 struct CombineSmem {
   static constexpr int TAIL = CAPTION ? CAPTION_V_SLOTS : W;   // most raw-value tokens of a sequence
-  __align__(16) float Rbuf[2][CB_CHUNK][D];   // double-buffered 32-row slices of the rotation matrices
+  __align__(16) float Rbuf[CB_NBUF][CB_CHUNK][D];   // ring of 16-row slices of the rotation matrices
+  __align__(16) float mrg[CB_SEQ][MRG_MAX][GP][4];                // per partial and head: rescale factor, weight sums of the modalities
   __align__(16) float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
   __align__(16) float rawv[CB_ROWS][D];       // raw-tail contribution, [row][channel]
   // q' = H q in the order of the (m, s) planes, for the scores of packed keys: [0] multiplies s * code, [1] the
@@ -671,6 +674,21 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
     sm.Ls[bs][c] = L;
   }
   __syncthreads();
+  // per partial and head: the rescale factor exp2(m - M) and the weight sums S_m (the four lanes of a quad hold
+  // partial sums), so that the merge below only reads accumulator fragments
+  for (int idx = c; idx < min(cta_hi - cta_lo + 1, MRG_MAX) * GP; idx += 128) {
+    const int ci = idx / GP, j = idx % GP;
+    const PartialF& pp = P.partials_f[(size_t)unit + cta_lo + ci];
+    const float pm = pp.m[j];
+    float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (pm != -INFINITY) {
+      f.x = exp2f(pm - sm.Ms[bs][j]);
+      f.y = pp.Sp[0][4 * j] + pp.Sp[0][4 * j + 1] + pp.Sp[0][4 * j + 2] + pp.Sp[0][4 * j + 3];
+      f.z = pp.Sp[1][4 * j] + pp.Sp[1][4 * j + 1] + pp.Sp[1][4 * j + 2] + pp.Sp[1][4 * j + 3];
+      f.w = pp.Sp[2][4 * j] + pp.Sp[2][4 * j + 1] + pp.Sp[2][4 * j + 2] + pp.Sp[2][4 * j + 3];
+    }
+    *reinterpret_cast<float4*>(sm.mrg[bs][ci][j]) = f;
+  }
   // raw-value tokens: softmax numerators in place of the scores, then every value row is read once for all heads
   for (int idx = c; idx < n_tail * GP; idx += 128) {
     const int i = idx / GP, j = idx % GP;
@@ -699,14 +717,19 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
       const int r = 4 * (c >> 4) + 2 * ((c >> 3) & 1) + (j & 1), l32 = 4 * (c & 7) + (j >> 1);
       for (int ct = cta_lo; ct <= cta_hi; ct++) {
         const PartialF& pp = P.partials_f[(size_t)unit + ct];
-        if (pp.m[j] == -INFINITY) continue;
-        const float ef = exp2f(pp.m[j] - M);
+        float ef, S[3];
+        if (ct - cta_lo < MRG_MAX) {
+          const float4 f = *reinterpret_cast<const float4*>(sm.mrg[bs][ct - cta_lo][j]);
+          ef = f.x; S[0] = f.y; S[1] = f.z; S[2] = f.w;
+        } else {   // more partials than the table holds (few heads over many CTAs): compute in place
+          const float pm = pp.m[j];
+          ef = pm == -INFINITY ? 0.f : exp2f(pm - M);
 #pragma unroll
-        for (int m = 0; m < 3; m++) {
-          // weight sum of head j: the four lanes of quad j hold partial sums
-          const float S = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
-          v[m] = fmaf(fmaf(ACC_SCALE, pp.frag[m][r][l32], S_COEF * S), ef, v[m]);
+          for (int m = 0; m < 3; m++) S[m] = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
         }
+        if (ef == 0.f) continue;
+#pragma unroll
+        for (int m = 0; m < 3; m++) v[m] = fmaf(fmaf(ACC_SCALE, pp.frag[m][r][l32], S_COEF * S[m]), ef, v[m]);
       }
     }
     sm.vec[0][bs * GP + j][c] = v[0];
@@ -724,8 +747,9 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
   constexpr int N_CHUNK = 3 * D / CB_CHUNK;
   auto stage = [&](int chunk) {   // rows [32*chunk, 32*chunk+32) of the three stacked matrices
     const float* src = Rset + (size_t)chunk * CB_CHUNK * D;
-    float* dst = &sm.Rbuf[chunk & 1][0][0];
-    for (int i = threadIdx.x - 256; i < CB_CHUNK * D / 4; i += 256) cp_async16(dst + 4 * i, src + 4 * i);
+    float* dst = &sm.Rbuf[chunk % CB_NBUF][0][0];
+    if (chunk < N_CHUNK)
+      for (int i = threadIdx.x - 256; i < CB_CHUNK * D / 4; i += 256) cp_async16(dst + 4 * i, src + 4 * i);
     cp_async_commit();
   };
   float o[4][4];
@@ -733,19 +757,20 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
   for (int i = 0; i < 4; i++)
 #pragma unroll
     for (int k = 0; k < 4; k++) o[i][k] = 0.f;
-  if (!comp) stage(0);
+  if (!comp)
+    for (int pre = 0; pre < CB_NBUF - 1; pre++) stage(pre);
   for (int chunk = 0; chunk < N_CHUNK; chunk++) {
-    if (!comp) cp_async_wait<0>();
+    if (!comp) cp_async_wait<CB_NBUF - 2>();
     __syncthreads();   // slice `chunk` has landed; everyone is done with slice chunk-1 (and, first time, vec is complete)
     if (!comp) {
-      if (chunk + 1 < N_CHUNK) stage(chunk + 1);
+      stage(chunk + CB_NBUF - 1);   // into the buffer of slice chunk-1
     } else {
       const int m = chunk / (D / CB_CHUNK), r0 = (chunk % (D / CB_CHUNK)) * CB_CHUNK;
 #pragma unroll 2
       for (int r = 0; r < CB_CHUNK; r += 4) {
         float4 rr[4], x[4];
 #pragma unroll
-        for (int k = 0; k < 4; k++) rr[k] = *reinterpret_cast<const float4*>(&sm.Rbuf[chunk & 1][r + k][cl]);
+        for (int k = 0; k < 4; k++) rr[k] = *reinterpret_cast<const float4*>(&sm.Rbuf[chunk % CB_NBUF][r + k][cl]);
 #pragma unroll
         for (int i = 0; i < 4; i++) x[i] = *reinterpret_cast<const float4*>(&sm.vec[m][rw + i][r0 + r]);
 #pragma unroll
