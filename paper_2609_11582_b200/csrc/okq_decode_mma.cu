@@ -708,34 +708,51 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
     araw[4] = fmaf(w1.x, x, araw[4]); araw[5] = fmaf(w1.y, x, araw[5]);
     araw[6] = fmaf(w1.z, x, araw[6]); araw[7] = fmaf(w1.w, x, araw[7]);
   }
+  // merge of the split-K partials, four heads at a time: per partial the twelve accumulator fragments of this
+  // thread's channel are fetched together (independent loads), then scaled by the table's factors
 #pragma unroll
-  for (int j = 0; j < GP; j++) {
-    float v[3] = {0.f, 0.f, 0.f};
-    const float a = araw[j];
-    if (j < G) {
-      const float M = sm.Ms[bs][j];
-      const int r = 4 * (c >> 4) + 2 * ((c >> 3) & 1) + (j & 1), l32 = 4 * (c & 7) + (j >> 1);
+  for (int jg = 0; jg < GP; jg += 4) {
+    float vacc[4][3];
+#pragma unroll
+    for (int jj = 0; jj < 4; jj++) vacc[jj][0] = vacc[jj][1] = vacc[jj][2] = 0.f;
+    if (jg < G) {
       for (int ct = cta_lo; ct <= cta_hi; ct++) {
         const PartialF& pp = P.partials_f[(size_t)unit + ct];
-        float ef, S[3];
-        if (ct - cta_lo < MRG_MAX) {
-          const float4 f = *reinterpret_cast<const float4*>(sm.mrg[bs][ct - cta_lo][j]);
-          ef = f.x; S[0] = f.y; S[1] = f.z; S[2] = f.w;
-        } else {   // more partials than the table holds (few heads over many CTAs): compute in place
-          const float pm = pp.m[j];
-          ef = pm == -INFINITY ? 0.f : exp2f(pm - M);
+        float fr[4][3];
 #pragma unroll
-          for (int m = 0; m < 3; m++) S[m] = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
+        for (int jj = 0; jj < 4; jj++) {
+          const int j = jg + jj;
+          const int r = 4 * (c >> 4) + 2 * ((c >> 3) & 1) + (j & 1), l32 = 4 * (c & 7) + (j >> 1);
+#pragma unroll
+          for (int m = 0; m < 3; m++) fr[jj][m] = pp.frag[m][r][l32];
         }
-        if (ef == 0.f) continue;
 #pragma unroll
-        for (int m = 0; m < 3; m++) v[m] = fmaf(fmaf(ACC_SCALE, pp.frag[m][r][l32], S_COEF * S[m]), ef, v[m]);
+        for (int jj = 0; jj < 4; jj++) {
+          const int j = jg + jj;
+          float ef, S[3];
+          if (ct - cta_lo < MRG_MAX) {
+            const float4 f = *reinterpret_cast<const float4*>(sm.mrg[bs][ct - cta_lo][j]);
+            ef = f.x; S[0] = f.y; S[1] = f.z; S[2] = f.w;
+          } else {   // more partials than the table holds (few heads over many CTAs): compute in place
+            const float pm = pp.m[j];
+            ef = pm == -INFINITY ? 0.f : exp2f(pm - sm.Ms[bs][j]);
+#pragma unroll
+            for (int m = 0; m < 3; m++) S[m] = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
+          }
+          if (j < G && ef != 0.f) {
+#pragma unroll
+            for (int m = 0; m < 3; m++) vacc[jj][m] = fmaf(fmaf(ACC_SCALE, fr[jj][m], S_COEF * S[m]), ef, vacc[jj][m]);
+          }
+        }
       }
     }
-    sm.vec[0][bs * GP + j][c] = v[0];
-    sm.vec[1][bs * GP + j][c] = v[1];
-    sm.vec[2][bs * GP + j][c] = v[2];
-    sm.rawv[bs * GP + j][c] = a;
+#pragma unroll
+    for (int jj = 0; jj < 4; jj++) {
+      sm.vec[0][bs * GP + jg + jj][c] = vacc[jj][0];
+      sm.vec[1][bs * GP + jg + jj][c] = vacc[jj][1];
+      sm.vec[2][bs * GP + jg + jj][c] = vacc[jj][2];
+      sm.rawv[bs * GP + jg + jj][c] = araw[jg + jj];
+    }
   }
 
   // out[row][c] = raw[row][c] + sum_m sum_r R_m[r][c] * vec[m][row][r].  Threads 0..255 compute a
