@@ -542,12 +542,14 @@ __device__ __forceinline__ float2 window_meta_pos(const unsigned char* meta, int
   return make_float2(mx_decode(mn, (int)meta[128 + blk] - 127), mx_decode(sn, (int)meta[132 + blk] - 127));
 }
 
-template <bool CAPTION>
+// NS: CTAs that share one (head, sequence group): each computes D / NS output columns (used when the grid
+// would otherwise leave most SMs idle; the merge is repeated by every slice, the matrix streaming is split)
+template <bool CAPTION, int NS>
 __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, int n_cta) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   CombineSmem<CAPTION>& sm = *reinterpret_cast<CombineSmem<CAPTION>*>(smem_raw);
   const CacheView& cv = P.cv;
-  const int h = blockIdx.x, li = blockIdx.z, layer = P.layer0 + li;
+  const int h = blockIdx.x / NS, sl = blockIdx.x % NS, li = blockIdx.z, layer = P.layer0 + li;
   const int bs = threadIdx.x >> 7, c = threadIdx.x & 127;
   const int b = blockIdx.y * CB_SEQ + bs;
   const bool live = b < cv.batch;
@@ -759,21 +761,28 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
   // 4-row x 4-column tile each; threads 256..511 stream the matrices through shared memory in
   // 32-row slices, one slice ahead.
   const bool comp = threadIdx.x < 256;
-  const int rw = (threadIdx.x >> 5) * 4, cl = (threadIdx.x & 31) * 4;   // first row / column of the tile
-  const float* Rset = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D;
+  constexpr int CW = 4 / NS;          // output columns per compute thread
+  constexpr int SW = D / NS;          // output columns of this CTA = floats per staged matrix row
+  static_assert(NS == 1 || NS == 4, "column slices");
+  const int rw = (threadIdx.x >> 5) * 4, cl = (threadIdx.x & 31) * CW;   // first row / column (inside the slice) of the tile
+  const float* Rset = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D + sl * SW;
   constexpr int N_CHUNK = 3 * D / CB_CHUNK;
-  auto stage = [&](int chunk) {   // rows [32*chunk, 32*chunk+32) of the three stacked matrices
+  float* rbuf = &sm.Rbuf[0][0][0];    // ring of CB_NBUF slices of CB_CHUNK x SW floats
+  auto stage = [&](int chunk) {   // rows [16*chunk, 16*chunk+16) of the three stacked matrices, this CTA's columns
     const float* src = Rset + (size_t)chunk * CB_CHUNK * D;
-    float* dst = &sm.Rbuf[chunk % CB_NBUF][0][0];
+    float* dst = rbuf + (chunk % CB_NBUF) * CB_CHUNK * SW;
     if (chunk < N_CHUNK)
-      for (int i = threadIdx.x - 256; i < CB_CHUNK * D / 4; i += 256) cp_async16(dst + 4 * i, src + 4 * i);
+      for (int i = threadIdx.x - 256; i < CB_CHUNK * SW / 4; i += 256) {
+        const int row = i / (SW / 4), c4 = i % (SW / 4);
+        cp_async16(dst + row * SW + 4 * c4, src + (size_t)row * D + 4 * c4);
+      }
     cp_async_commit();
   };
-  float o[4][4];
+  float o[4][CW];
 #pragma unroll
   for (int i = 0; i < 4; i++)
 #pragma unroll
-    for (int k = 0; k < 4; k++) o[i][k] = 0.f;
+    for (int k = 0; k < CW; k++) o[i][k] = 0.f;
   if (!comp)
     for (int pre = 0; pre < CB_NBUF - 1; pre++) stage(pre);
   for (int chunk = 0; chunk < N_CHUNK; chunk++) {
@@ -783,23 +792,32 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
       stage(chunk + CB_NBUF - 1);   // into the buffer of slice chunk-1
     } else {
       const int m = chunk / (D / CB_CHUNK), r0 = (chunk % (D / CB_CHUNK)) * CB_CHUNK;
+      const float* rb = rbuf + (chunk % CB_NBUF) * CB_CHUNK * SW;
 #pragma unroll 2
       for (int r = 0; r < CB_CHUNK; r += 4) {
-        float4 rr[4], x[4];
-#pragma unroll
-        for (int k = 0; k < 4; k++) rr[k] = *reinterpret_cast<const float4*>(&sm.Rbuf[chunk % CB_NBUF][r + k][cl]);
+        float4 x[4];
 #pragma unroll
         for (int i = 0; i < 4; i++) x[i] = *reinterpret_cast<const float4*>(&sm.vec[m][rw + i][r0 + r]);
+        if (NS == 1) {
+          float4 rr[4];
 #pragma unroll
-        for (int i = 0; i < 4; i++) {
-          o[i][0] = fmaf(rr[0].x, x[i].x, o[i][0]); o[i][1] = fmaf(rr[0].y, x[i].x, o[i][1]);
-          o[i][2] = fmaf(rr[0].z, x[i].x, o[i][2]); o[i][3] = fmaf(rr[0].w, x[i].x, o[i][3]);
-          o[i][0] = fmaf(rr[1].x, x[i].y, o[i][0]); o[i][1] = fmaf(rr[1].y, x[i].y, o[i][1]);
-          o[i][2] = fmaf(rr[1].z, x[i].y, o[i][2]); o[i][3] = fmaf(rr[1].w, x[i].y, o[i][3]);
-          o[i][0] = fmaf(rr[2].x, x[i].z, o[i][0]); o[i][1] = fmaf(rr[2].y, x[i].z, o[i][1]);
-          o[i][2] = fmaf(rr[2].z, x[i].z, o[i][2]); o[i][3] = fmaf(rr[2].w, x[i].z, o[i][3]);
-          o[i][0] = fmaf(rr[3].x, x[i].w, o[i][0]); o[i][1] = fmaf(rr[3].y, x[i].w, o[i][1]);
-          o[i][2] = fmaf(rr[3].z, x[i].w, o[i][2]); o[i][3] = fmaf(rr[3].w, x[i].w, o[i][3]);
+          for (int k = 0; k < 4; k++) rr[k] = *reinterpret_cast<const float4*>(&rb[(r + k) * SW + cl]);
+#pragma unroll
+          for (int i = 0; i < 4; i++) {
+            o[i][0] = fmaf(rr[0].x, x[i].x, o[i][0]); o[i][1 % CW] = fmaf(rr[0].y, x[i].x, o[i][1 % CW]);
+            o[i][2 % CW] = fmaf(rr[0].z, x[i].x, o[i][2 % CW]); o[i][3 % CW] = fmaf(rr[0].w, x[i].x, o[i][3 % CW]);
+            o[i][0] = fmaf(rr[1].x, x[i].y, o[i][0]); o[i][1 % CW] = fmaf(rr[1].y, x[i].y, o[i][1 % CW]);
+            o[i][2 % CW] = fmaf(rr[1].z, x[i].y, o[i][2 % CW]); o[i][3 % CW] = fmaf(rr[1].w, x[i].y, o[i][3 % CW]);
+            o[i][0] = fmaf(rr[2].x, x[i].z, o[i][0]); o[i][1 % CW] = fmaf(rr[2].y, x[i].z, o[i][1 % CW]);
+            o[i][2 % CW] = fmaf(rr[2].z, x[i].z, o[i][2 % CW]); o[i][3 % CW] = fmaf(rr[2].w, x[i].z, o[i][3 % CW]);
+            o[i][0] = fmaf(rr[3].x, x[i].w, o[i][0]); o[i][1 % CW] = fmaf(rr[3].y, x[i].w, o[i][1 % CW]);
+            o[i][2 % CW] = fmaf(rr[3].z, x[i].w, o[i][2 % CW]); o[i][3 % CW] = fmaf(rr[3].w, x[i].w, o[i][3 % CW]);
+          }
+        } else {   // one column per thread
+          const float r0v = rb[(r + 0) * SW + cl], r1v = rb[(r + 1) * SW + cl], r2v = rb[(r + 2) * SW + cl], r3v = rb[(r + 3) * SW + cl];
+#pragma unroll
+          for (int i = 0; i < 4; i++)
+            o[i][0] = fmaf(r3v, x[i].w, fmaf(r2v, x[i].z, fmaf(r1v, x[i].y, fmaf(r0v, x[i].x, o[i][0]))));
         }
       }
     }
@@ -810,13 +828,15 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
       const int row = rw + i, ob = blockIdx.y * CB_SEQ + row / GP, j = row % GP;
       if (ob >= cv.batch || j >= G) continue;
       const float L = sm.Ls[row / GP][j];
-      const float4 rv = *reinterpret_cast<const float4*>(&sm.rawv[row][cl]);
-      float4 res = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (L > 0.f) {
-        const float inv = 1.0f / L;
-        res = make_float4((o[i][0] + rv.x) * inv, (o[i][1] + rv.y) * inv, (o[i][2] + rv.z) * inv, (o[i][3] + rv.w) * inv);
+      const float inv = L > 0.f ? 1.0f / L : 0.f;
+      float* dst = &P.out[(((size_t)li * cv.batch + ob) * cv.n_q_heads + h * G + j) * D + sl * SW + cl];
+      if (NS == 1) {
+        const float4 rv = *reinterpret_cast<const float4*>(&sm.rawv[row][cl]);
+        *reinterpret_cast<float4*>(dst) = make_float4((o[i][0] + rv.x) * inv, (o[i][1 % CW] + rv.y) * inv,
+                                                      (o[i][2 % CW] + rv.z) * inv, (o[i][3 % CW] + rv.w) * inv);
+      } else {
+        dst[0] = (o[i][0] + sm.rawv[row][sl * SW + cl]) * inv;
       }
-      *reinterpret_cast<float4*>(&P.out[(((size_t)li * cv.batch + ob) * cv.n_q_heads + h * G + j) * D + cl]) = res;
     }
   }
 }
@@ -831,9 +851,13 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
       e = cudaFuncSetAttribute(k_decode_mma<FMT_MXFP4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)sizeof(MmaSmem<FMT_MXFP4>));
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_combine_mma<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<false>));
+      e = cudaFuncSetAttribute(k_combine_mma<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<false>));
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_combine_mma<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<true>));
+      e = cudaFuncSetAttribute(k_combine_mma<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<false>));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_combine_mma<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<true>));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_combine_mma<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<true>));
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
     attr_done(attr_mask, attr_dev);
   }
@@ -841,9 +865,15 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
   if (P.cv.fmt == FMT_MXFP4) k_decode_mma<FMT_MXFP4><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_MXFP4>), s>>>(P);
   else k_decode_mma<FMT_FP16><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_FP16>), s>>>(P);
   if (after) cudaEventRecord(after, s);
-  const dim3 cgrid(P.cv.n_kv_heads, (P.cv.batch + CB_SEQ - 1) / CB_SEQ, P.layer_count);
-  if (P.cv.sched == SCHED_CAPTION) k_combine_mma<true><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<true>), s>>>(P, n_cta);
-  else k_combine_mma<false><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<false>), s>>>(P, n_cta);
+  // few (head, sequence group, layer) blocks, e.g. a single-layer call: four column slices per block
+  const int n_blocks = P.cv.n_kv_heads * ((P.cv.batch + CB_SEQ - 1) / CB_SEQ) * P.layer_count;
+  const int ns = 4 * n_blocks <= n_cta ? 4 : 1;
+  const dim3 cgrid(P.cv.n_kv_heads * ns, (P.cv.batch + CB_SEQ - 1) / CB_SEQ, P.layer_count);
+  const bool cap = P.cv.sched == SCHED_CAPTION;
+  if (cap && ns == 4) k_combine_mma<true, 4><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<true>), s>>>(P, n_cta);
+  else if (cap) k_combine_mma<true, 1><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<true>), s>>>(P, n_cta);
+  else if (ns == 4) k_combine_mma<false, 4><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<false>), s>>>(P, n_cta);
+  else k_combine_mma<false, 1><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<false>), s>>>(P, n_cta);
   return OKQ_OK;
 }
 
