@@ -57,7 +57,7 @@ extern "C" {
 #define OKQ_META_FP16 0
 #define OKQ_META_MXFP4 1
 #define OKQ_MAX_GROUP 8
-#define OKQ_NOALLOC_SCRATCH_BYTES (32u << 20) /* fixed scratch of okq_decode_attention_noalloc */
+#define OKQ_NOALLOC_SCRATCH_BYTES (64u << 20) /* fixed scratch of okq_decode_attention_noalloc */
 
 typedef enum {
   OKQ_OK = 0,
@@ -204,13 +204,15 @@ okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t l
  * carved up at start-up, under a caching allocator that must not be bypassed, in a plugin
  * that is only handed its inputs and outputs).  The paper has no counterpart; this is the
  * same kernel pair with its split-K partials kept in a fixed OKQ_NOALLOC_SCRATCH_BYTES
- * (32 MiB) array that is part of the library's device image, so every GPU that loads the
- * library carries those 32 MiB until the process exits.  The call allocates nothing: no
+ * (64 MiB) array that is part of the library's device image, so every GPU that loads the
+ * library carries those 64 MiB until the process exits.  The call allocates nothing: no
  * cudaMalloc, no cudaFree, no allocating library routine.
  *
  *   - Arguments are those of okq_decode_attention without workspace / workspace_bytes.
- *   - Limit: (layer_count * batch * n_kv_heads + number of CTAs) * 12736 bytes must fit in the
- *     scratch, i.e. about 2630 (sequence, KV head) pairs per launch with the automatic grid;
+ *   - Limit: okq_decode_workspace_bytes(cache, layer_count, num_splits) of the largest launch, i.e.
+ *     (layer_count * batch * n_kv_heads + number of CTAs) * 12736 bytes of per-CTA partials plus
+ *     (layer_count * batch * n_kv_heads + 8 * number of CTAs) * 12832 bytes of per-warp-pair pieces,
+ *     must fit in the scratch: about 1950 (sequence, KV head) pairs per launch with the automatic grid;
  *     anything larger returns OKQ_ERR_WORKSPACE and launches nothing (use
  *     okq_decode_attention with your own buffer).
  *   - The first call on each device looks up the scratch's device address (with that device

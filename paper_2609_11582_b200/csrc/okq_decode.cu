@@ -407,8 +407,15 @@ static size_t simt_workspace(const okq_cache* c, int layer_count, int num_splits
   return (size_t)layer_count * c->batch * c->n_kv_heads * S * sizeof(Partial);
 }
 
-static size_t mma_workspace(const okq_cache* c, int layer_count, int num_splits) {
+// one PartialF per (CTA, (sequence, head)) overlap, then one PairPartial per (warp pair, (sequence, head))
+// overlap: slot = unit index + CTA (or global pair) index, both non-decreasing along the window axis
+static size_t mma_partials_bytes(const okq_cache* c, int layer_count, int num_splits) {
   return ((size_t)layer_count * c->batch * c->n_kv_heads + mma_ctas(c, layer_count, num_splits)) * sizeof(PartialF);
+}
+static size_t mma_workspace(const okq_cache* c, int layer_count, int num_splits) {
+  return mma_partials_bytes(c, layer_count, num_splits) +
+         ((size_t)layer_count * c->batch * c->n_kv_heads + (size_t)MMA_PAIRS * mma_ctas(c, layer_count, num_splits)) *
+             sizeof(PairPartial);
 }
 
 static okq_status check_decode(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* q,
@@ -432,7 +439,7 @@ static DecodeParams make_params(const okq_cache* cache, int32_t layer, int32_t l
   P.layer0 = layer; P.layer_count = layer_count; P.n_splits = 1;
   P.group = cache->n_q_heads / cache->n_kv_heads;
   P.q = static_cast<const __half*>(q); P.signs = signs; P.R = R; P.n_R = n_R; P.sm_scale = sm_scale;
-  P.partials = nullptr; P.partials_f = nullptr; P.out = out;
+  P.partials = nullptr; P.partials_f = nullptr; P.pair_parts = nullptr; P.out = out;
   return P;
 }
 
@@ -468,6 +475,8 @@ okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t l
     DecodeParams P = make_params(cache, layer + l0, lc, static_cast<const __half*>(q) + l0 * q_stride, sm_scale,
                                  signs + (size_t)l0 * D, R + (size_t)l0 * n_R * 3 * D * D, n_R, out + l0 * q_stride);
     P.partials_f = static_cast<PartialF*>(workspace);
+    P.pair_parts = reinterpret_cast<PairPartial*>(static_cast<unsigned char*>(workspace) +
+                                                  mma_partials_bytes(cache, lc, num_splits));
     const int n_cta = mma_ctas(cache, lc, num_splits);
     st = launch_decode_mma(P, n_cta, s, g_ev_before, g_ev_after);
     if (st != OKQ_OK) return st;
@@ -498,6 +507,8 @@ okq_status okq_decode_attention_noalloc(const okq_cache* cache, int32_t layer, i
     DecodeParams P = make_params(cache, layer + l0, lc, static_cast<const __half*>(q) + l0 * q_stride, sm_scale,
                                  signs + (size_t)l0 * D, R + (size_t)l0 * n_R * 3 * D * D, n_R, out + l0 * q_stride);
     P.partials_f = static_cast<PartialF*>(scratch);
+    P.pair_parts = reinterpret_cast<PairPartial*>(static_cast<unsigned char*>(scratch) +
+                                                  mma_partials_bytes(cache, lc, num_splits));
     st = launch_decode_mma(P, mma_ctas(cache, lc, num_splits), s, nullptr, nullptr);
     if (st != OKQ_OK) return st;
   }

@@ -18,10 +18,13 @@
 // the fp16 numerators to its "value" warp through shared memory; the value warp accumulates
 // the codebook sums of the previous window meanwhile.  One named barrier per pair and
 // iteration keeps the two in step (no spin-waits anywhere).  Values accumulate in the rotated
-// basis of the current modality; the other modalities' accumulators wait in shared memory.
+// basis of the current modality, in registers for at most 32 windows at a time; each modality's
+// running sums live in shared memory.
 // The grid is persistent: CTA i owns an equal slice of the flattened (layer, sequence, head,
-// window) axis and writes one partial per (sequence, head) it touches; the combine kernel
-// merges them, adds the raw fp16 tail tokens, applies R_m^T once per head and normalises.
+// window) axis, each of its pairs an eighth of that slice, which the pair walks without any
+// block-wide step; at the end the block merges its pairs' pieces into one partial per
+// (sequence, head) it touched.  The combine kernel merges the partials, adds the raw fp16 tail
+// tokens, applies R_m^T once per head and normalises.
 #include "okq_common.cuh"
 #include "okq_device.cuh"
 #include "okq_decode_shared.cuh"
@@ -30,7 +33,7 @@ namespace okq {
 
 namespace {
 
-constexpr int NPAIR = 8;                        // warp pairs per CTA
+constexpr int NPAIR = MMA_PAIRS;                // warp pairs per CTA
 constexpr int NTHREADS = NPAIR * 64;
 constexpr int NSTAGE = 4;                       // record ring per pair
 constexpr int PREFETCH = 2;                     // windows in flight ahead of the score warp
@@ -39,7 +42,9 @@ constexpr int PREFETCH = 2;                     // windows in flight ahead of th
 constexpr int STAGE_MOD = RECORD_BYTES, STAGE_MX = RECORD_BYTES + 32;
 template <int FMT> constexpr int stage_bytes() { return FMT == FMT_MXFP4 ? STAGE_MX + 144 : STAGE_MX; }
 constexpr float RESCALE_LOG2 = 3.0f;            // numerators stay below 2^3 * 2^6 * vnorm in fp16
-constexpr int SPILL_REGS = 33;                  // 32 accumulator registers + the running weight sum
+constexpr int FLUSH = 32;                       // windows a value warp accumulates in registers at most
+constexpr int SPILL_STRIDE = 36;                // floats per lane in the deposited sums: 33 used, 144-byte rows
+constexpr int SPILL_REGS = PAIR_REGS;           // 32 accumulator registers + the running weight sum
 
 struct Handoff {
   uint4 pb[32];         // per lane: numerators p * vnorm * 2^6 / 4^nu of its 8 tokens, fp16 pairs (nu = x,y,z,w)
@@ -53,12 +58,9 @@ template <int FMT>
 struct MmaSmem {
   __align__(16) unsigned char stage[NPAIR][NSTAGE][stage_bytes<FMT>()];
   __align__(16) Handoff hand[NPAIR][2];
-  float spill[NPAIR][3][SPILL_REGS][32];
+  __align__(16) float spill[NPAIR][3][32][SPILL_STRIDE];   // [pair][modality][lane]: the lane's 33 sums, 128-bit rows
   float spill_m[NPAIR][3][GP];
-  float qs[GP][D];       // q' * 2^kh, natural channel order
-  uint2 qf[16][32];      // per lane and fragment register r: (hi, lo) fp16 pairs of q' / 4^(r&3)
-  float fscale[GP];      // 2^(24-kh) * sm_scale * log2(e)
-  float wm[NPAIR][GP], wl[NPAIR][GP];
+  float mrg_m[NPAIR][3][GP], mrg_wm[NPAIR][GP], mrg_wl[NPAIR][GP], mrg_M[GP];   // end-of-launch merge: the pieces' maxima
   int prefix[MAX_ENTRIES + 1];
 };
 
@@ -114,19 +116,90 @@ __device__ __forceinline__ void split_product(__half2 qh, __half2 ql, __half2 x,
 struct Segment {
   const unsigned char* rec0;   // first record of the (layer, sequence, head)
   const unsigned char* mod0;   // modality row of the sequence
-  int w0, n_my;                // this pair's contiguous window range: first window, count
+  int w0, n_my;                // this pair's windows of that (layer, sequence, head): first window, count
+  const __half* q;             // query rows of the KV head's group: [group][128]
+  const float* signs;          // Hadamard signs of the layer
+  PairPartial* piece;          // where the pair leaves what it accumulated
 };
+
+// The group's rotated queries q' = H D q / sqrt(128) as mma A-fragment registers, computed by one warp in
+// registers: lane (g, t) holds head g, channels 8 r + 2 t + {0, 1} for r = 0..15, so the transform's
+// butterflies over channel bits 0 and 3..6 stay inside the lane and those over bits 1..2 are two shuffles.
+// Each pair is scaled into the fp16 range (2^kh, per head), pre-divided by 4^(r&3) (the position scale of
+// the matching code field) and split into an fp16 high and low part.  fsc = 2^(24-kh) * sm_scale * log2(e).
+__device__ __forceinline__ void query_fragments(const Segment& sg, int G, float sm_scale, int lane, uint2 (&qreg)[16],
+                                                float& fsc) {
+  const int g = lane >> 2, t = lane & 3;
+  float x[16][2];
+  if (g < G) {
+    const __half* qrow = sg.q + (size_t)g * D + 2 * t;
+    const float* srow = sg.signs + 2 * t;
+#pragma unroll
+    for (int r = 0; r < 16; r++) {
+      const float2 qv = __half22float2(*reinterpret_cast<const __half2*>(qrow + 8 * r));
+      const float2 sv = *reinterpret_cast<const float2*>(srow + 8 * r);
+      x[r][0] = qv.x * sv.x; x[r][1] = qv.y * sv.y;
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < 16; r++) x[r][0] = x[r][1] = 0.f;
+  }
+#pragma unroll
+  for (int r = 0; r < 16; r++) {   // channel bit 0
+    const float a = x[r][0], b = x[r][1];
+    x[r][0] = a + b; x[r][1] = a - b;
+  }
+#pragma unroll
+  for (int d = 1; d < 4; d <<= 1) {   // channel bits 1, 2: lanes t ^ d
+    const bool upper = (lane & d) != 0;
+#pragma unroll
+    for (int r = 0; r < 16; r++)
+#pragma unroll
+      for (int e = 0; e < 2; e++) {
+        const float p = __shfl_xor_sync(0xffffffffu, x[r][e], d);
+        x[r][e] = upper ? p - x[r][e] : x[r][e] + p;
+      }
+  }
+#pragma unroll
+  for (int s = 1; s < 16; s <<= 1)   // channel bits 3..6
+#pragma unroll
+    for (int r = 0; r < 16; r++)
+      if (!(r & s)) {
+#pragma unroll
+        for (int e = 0; e < 2; e++) {
+          const float a = x[r][e], b = x[r + s][e];
+          x[r][e] = a + b; x[r + s][e] = a - b;
+        }
+      }
+  float mx = 0.f;
+#pragma unroll
+  for (int r = 0; r < 16; r++) {
+    x[r][0] *= RSQRT_D; x[r][1] *= RSQRT_D;
+    mx = fmaxf(mx, fmaxf(fabsf(x[r][0]), fabsf(x[r][1])));
+  }
+  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+  int ex = 0;
+  if (mx > 0.f) frexpf(mx, &ex);           // mx < 2^ex
+  const int kh = 14 - ex;                  // |q'| * 2^kh < 2^14
+  const float up = exp2f((float)kh);
+  fsc = exp2f((float)(24 - kh)) * sm_scale * 1.4426950408889634f;
+#pragma unroll
+  for (int r = 0; r < 16; r++) {
+    const float sc = up / (float)(1 << (2 * (r & 3)));
+    const float x0 = x[r][0] * sc, x1 = x[r][1] * sc;
+    const __half2 hi2 = __floats2half2_rn(x0, x1);
+    const float2 hf = __half22float2(hi2);
+    qreg[r] = make_uint2(h2u(hi2), h2u(__floats2half2_rn(x0 - hf.x, x1 - hf.y)));
+  }
+}
 
 // ---------------------------------------------------------------- score warp
 template <int FMT>
-__device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, int pair, int lane, float& run_m_out,
-                                           float& run_l_out) {
+__device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, int G, float sm_scale, int pair,
+                                           int lane) {
   const int g = lane >> 2, t = lane & 3;
-  const float fsc = sm.fscale[g];
   float run_m = -INFINITY, run_l = 0.f;
-  uint2 qreg[16];
-#pragma unroll
-  for (int r = 0; r < 16; r++) qreg[r] = sm.qf[r][lane];
 
   auto issue = [&](int k) {
     if (k < sg.n_my) {
@@ -157,6 +230,9 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
   };
 #pragma unroll
   for (int k = 0; k < PREFETCH; k++) issue(k);
+  uint2 qreg[16];
+  float fsc;
+  query_fragments(sg, G, sm_scale, lane, qreg, fsc);   // while the first windows are on their way
 
   for (int k = 0; k <= sg.n_my; k++) {
     if (k < sg.n_my) {
@@ -250,8 +326,9 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
     pair_barrier(pair);
   }
   cp_async_wait<0>();
-  run_m_out = run_m;
-  run_l_out = run_l;
+  run_l += __shfl_xor_sync(0xffffffffu, run_l, 1);
+  run_l += __shfl_xor_sync(0xffffffffu, run_l, 2);
+  if (t == 0) { sg.piece->wm[g] = run_m; sg.piece->wl[g] = run_l; }
 }
 
 // ---------------------------------------------------------------- value warp
@@ -265,16 +342,45 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
     for (int i = 0; i < 4; i++) acc[mu][i] = 0.f;
   float run_S = 0.f;
   int cur_mod = -1;
-  float cur_m = -INFINITY;   // running maximum of head g the live accumulators refer to
+  int since = 0;             // windows accumulated in registers since the last deposit
+  // nothing deposited yet (the deposited registers themselves are only read where a maximum says so)
+  if (lane < 3 * GP) (&sm.spill_m[pair][0][0])[lane] = -INFINITY;
+  __syncwarp();
 
-  auto park = [&]() {
-    float* dst = &sm.spill[pair][cur_mod][0][lane];
+  // Adds the live accumulators (which refer to the running maxima ho.m) to the current modality's sums in
+  // shared memory and clears them.  Apart from modality changes this happens every FLUSH windows: the
+  // tensor cores' fp32 accumulation does not round to nearest, so a long chain of MMAs into one register
+  // drifts, and the difference against the exactly rounded weight sum run_S is amplified by the codebook's
+  // cancellation (code plane minus b times the weight sum); short chains summed with FFMA do not drift.
+  auto deposit = [&](const Handoff& ho) {
+    float4* dst = reinterpret_cast<float4*>(&sm.spill[pair][cur_mod][lane][0]);
+    float* dm = &sm.spill_m[pair][cur_mod][0];
+    const float s_lo = dm[2 * t], s_hi = dm[2 * t + 1], s_g = dm[g];
+    if (s_g == -INFINITY) {   // first deposit of this modality (the same for every head)
+#pragma unroll
+      for (int mu = 0; mu < 8; mu++) dst[mu] = make_float4(acc[mu][0], acc[mu][1], acc[mu][2], acc[mu][3]);
+      reinterpret_cast<float*>(dst)[32] = run_S;
+    } else {
+      const float f_lo = ex2(s_lo - ho.m[2 * t]), f_hi = ex2(s_hi - ho.m[2 * t + 1]), f_g = ex2(s_g - ho.m[g]);
+#pragma unroll
+      for (int mu = 0; mu < 8; mu++) {
+        float4 v = dst[mu];
+        v.x = fmaf(v.x, f_lo, acc[mu][0]); v.y = fmaf(v.y, f_hi, acc[mu][1]);
+        v.z = fmaf(v.z, f_lo, acc[mu][2]); v.w = fmaf(v.w, f_hi, acc[mu][3]);
+        dst[mu] = v;
+      }
+      float* dS = reinterpret_cast<float*>(dst) + 32;
+      *dS = fmaf(*dS, f_g, run_S);
+    }
+    __syncwarp();
+    if (t == 0) dm[g] = ho.m[g];
+    __syncwarp();
 #pragma unroll
     for (int mu = 0; mu < 8; mu++)
 #pragma unroll
-      for (int i = 0; i < 4; i++) dst[(4 * mu + i) * 32] = acc[mu][i];
-    dst[32 * 32] = run_S;
-    if (t == 0) sm.spill_m[pair][cur_mod][g] = cur_m;
+      for (int i = 0; i < 4; i++) acc[mu][i] = 0.f;
+    run_S = 0.f;
+    since = 0;
   };
 
   for (int k = 0; k <= sg.n_my; k++) {
@@ -289,7 +395,6 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
         }
         run_S *= ho.alpha[g];
       }
-      cur_m = ho.m[g];
       const unsigned char* wmod = st + STAGE_MOD;
       const int mymod = wmod[lane];
       const int first = __shfl_sync(0xffffffffu, mymod, 0);
@@ -310,22 +415,8 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
         int m = (cur_mod >= 0 && (present >> cur_mod) & 1) ? cur_mod : (__ffs(present) - 1);
         present &= ~(1u << m);
         if (m != cur_mod) {
-          if (cur_mod >= 0) park();
-          __syncwarp();
-          const float* src = &sm.spill[pair][m][0][lane];
-          const float sm_lo = sm.spill_m[pair][m][2 * t], sm_hi = sm.spill_m[pair][m][2 * t + 1];
-          const float sm_g = sm.spill_m[pair][m][g];
-          const float f_lo = sm_lo == -INFINITY ? 0.f : ex2(sm_lo - ho.m[2 * t]);
-          const float f_hi = sm_hi == -INFINITY ? 0.f : ex2(sm_hi - ho.m[2 * t + 1]);
-          const float f_g = sm_g == -INFINITY ? 0.f : ex2(sm_g - cur_m);
-#pragma unroll
-          for (int mu = 0; mu < 8; mu++) {
-            acc[mu][0] = src[(4 * mu + 0) * 32] * f_lo; acc[mu][1] = src[(4 * mu + 1) * 32] * f_hi;
-            acc[mu][2] = src[(4 * mu + 2) * 32] * f_lo; acc[mu][3] = src[(4 * mu + 3) * 32] * f_hi;
-          }
-          run_S = src[32 * 32] * f_g;
+          if (cur_mod >= 0) deposit(ho);
           cur_mod = m;
-          __syncwarp();
         }
         uint32_t b0[4], b1[4];
         unsigned halfmask = 3u;  // which 16-token halves hold a token of modality m
@@ -374,15 +465,40 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
           }
         }
       }
+      // before the barrier: the score warp may overwrite this hand-off record right after it
+      if (k == sg.n_my || ++since >= FLUSH) deposit(ho);
     }
     pair_barrier(pair);
   }
-  if (cur_mod >= 0) park();
+  // leave the three modalities' accumulators (each lane its own column) and their maxima in the pair's piece
+#pragma unroll 1
+  for (int m = 0; m < 3; m++) {
+    const float mm = sm.spill_m[pair][m][g];
+    if (t == 0) sg.piece->sm[m][g] = mm;
+    if (mm != -INFINITY) {
+      const float4* src = reinterpret_cast<const float4*>(&sm.spill[pair][m][lane][0]);
+      float* dst = &sg.piece->frag[m][0][lane];
+#pragma unroll
+      for (int mu = 0; mu < 8; mu++) {
+        const float4 v = src[mu];
+        dst[(4 * mu) * 32] = v.x; dst[(4 * mu + 1) * 32] = v.y; dst[(4 * mu + 2) * 32] = v.z; dst[(4 * mu + 3) * 32] = v.w;
+      }
+      dst[32 * 32] = reinterpret_cast<const float*>(src)[32];
+    }
+  }
+  __syncwarp();
 }
 
 }  // namespace
 
 // grid = n_cta (persistent), 512 threads
+//
+// CTA i owns the windows [i * per, (i + 1) * per) of the flattened (layer, sequence, head, window) axis and
+// cuts them into eight contiguous ranges, one per warp pair.  A pair walks its range on its own, with no
+// block-wide step in between: where the range crosses into another (sequence, head) the score warp sets up
+// that head group's query fragments, the value warp leaves what it accumulated in a PairPartial piece and
+// starts afresh.  At the end of the launch the block merges, per (sequence, head) it touched, the pieces of
+// the pairs that worked on it into one PartialF.
 template <int FMT>
 __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -397,110 +513,90 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
   // ---- partition of the flattened window axis
   const int total = block_prefix(cv, P.layer0, n_entries, sm.prefix);
   const int per = (total + gridDim.x - 1) / gridDim.x;
-  int pos = min(total, (int)blockIdx.x * per);
-  const int pos_end = min(total, pos + per);
+  const int pos0 = min(total, (int)blockIdx.x * per), pos1 = min(total, pos0 + per);
+  const int cnt = (pos1 - pos0 + NPAIR - 1) / NPAIR;
 
-  while (pos < pos_end) {
-    // locate (entry, head, first window) of this segment
-    int lo = 0, hi = n_entries;  // largest e with prefix[e] <= pos
+  struct Where { int e, h, w0, nwin; };
+  auto locate = [&](int pos) {   // (entry, head, window) of a flattened position; largest e with prefix[e] <= pos
+    int lo = 0, hi = n_entries;
     while (hi - lo > 1) {
       int mid = (lo + hi) >> 1;
       if (sm.prefix[mid] <= pos) lo = mid; else hi = mid;
     }
-    const int e = lo, li = e / cv.batch, b = e % cv.batch, layer = P.layer0 + li;
-    const int nwin = (sm.prefix[e + 1] - sm.prefix[e]) / Hkv;
-    const int off = pos - sm.prefix[e];
-    const int h = off / nwin, w0 = off % nwin;
-    const int seg = min(pos_end - pos, nwin - w0);
-    const int unit = e * Hkv + h;
+    Where wh;
+    wh.e = lo;
+    wh.nwin = (sm.prefix[lo + 1] - sm.prefix[lo]) / Hkv;
+    const int off = pos - sm.prefix[lo];
+    wh.h = off / wh.nwin;
+    wh.w0 = off % wh.nwin;
+    return wh;
+  };
 
-    // ---- per-segment setup
-    if (is_score) {
-      // q' for head `pair` of the group, scaled into the fp16 range
-      const int hh = pair;
-      float4 qr = make_float4(0, 0, 0, 0);
-      if (hh < G) {
-        const __half* qrow = P.q + (((size_t)li * cv.batch + b) * cv.n_q_heads + h * G + hh) * D;
-        float4 x = load_row4(qrow, lane);
-        const float4 sg = *reinterpret_cast<const float4*>(P.signs + (size_t)li * D + 4 * lane);
-        qr = warp_fwht(make_float4(x.x * sg.x, x.y * sg.y, x.z * sg.z, x.w * sg.w), lane);
-      }
-      float v[4] = {qr.x * RSQRT_D, qr.y * RSQRT_D, qr.z * RSQRT_D, qr.w * RSQRT_D};
-      float mx = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
-#pragma unroll
-      for (int d = 16; d; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
-      int ex = 0;
-      if (mx > 0.f) frexpf(mx, &ex);           // mx < 2^ex
-      const int kh = 14 - ex;                  // |q'| * 2^kh < 2^14
-      const float up = exp2f((float)kh);
-      *reinterpret_cast<float4*>(&sm.qs[hh][4 * lane]) = make_float4(v[0] * up, v[1] * up, v[2] * up, v[3] * up);
-      if (lane == 0) sm.fscale[hh] = exp2f((float)(24 - kh)) * P.sm_scale * 1.4426950408889634f;
-    } else {
-      // clear this pair's parked accumulators
-      float* sp = &sm.spill[pair][0][0][0];
-      for (int i = lane; i < 3 * SPILL_REGS * 32; i += 32) sp[i] = 0.f;
-      if (lane < 3 * GP) (&sm.spill_m[pair][0][0])[lane] = -INFINITY;
+  {
+    int pos = min(pos1, pos0 + pair * cnt);
+    const int pos_end = min(pos1, pos + cnt);
+    while (pos < pos_end) {
+      const Where wh = locate(pos);
+      const int li = wh.e / cv.batch, b = wh.e % cv.batch;
+      Segment sg;
+      sg.rec0 = cv.unit(P.layer0 + li, b, wh.h);
+      sg.mod0 = cv.modality + (size_t)b * cv.capacity;
+      sg.w0 = wh.w0;
+      sg.n_my = min(pos_end - pos, wh.nwin - wh.w0);
+      sg.q = P.q + (((size_t)li * cv.batch + b) * cv.n_q_heads + (size_t)wh.h * G) * D;
+      sg.signs = P.signs + (size_t)li * D;
+      sg.piece = P.pair_parts + (size_t)(wh.e * Hkv + wh.h) + ((size_t)blockIdx.x * NPAIR + pair);
+      if (is_score) score_warp<FMT>(sm, sg, G, P.sm_scale, pair, lane);
+      else value_warp<FMT>(sm, sg, pair, lane);
+      pos += sg.n_my;
     }
-    __syncthreads();
-    {  // fragment registers of the queries: lane (g, t) holds head g, channels {16k + 8p + 2t + e} for
-       // r = 2k + p, pre-divided by 4^(r&3) (the position scale of the matching code field)
-      const int r = tid >> 5, gg = lane >> 2, tt = lane & 3;
-      const int c0 = 16 * (r >> 1) + 8 * (r & 1) + 2 * tt;
-      const float sc = 1.0f / (float)(1 << (2 * (r & 3)));
-      const float x0 = sm.qs[gg][c0] * sc, x1 = sm.qs[gg][c0 + 1] * sc;
-      const __half2 hi2 = __floats2half2_rn(x0, x1);
-      const float2 hf = __half22float2(hi2);
-      sm.qf[r][lane] = make_uint2(h2u(hi2), h2u(__floats2half2_rn(x0 - hf.x, x1 - hf.y)));
-    }
-    __syncthreads();
+  }
+  __syncthreads();   // the pieces were written by this block's own warps: visible to the block from here on
 
-    Segment sg;
-    sg.rec0 = cv.unit(layer, b, h);
-    sg.mod0 = cv.modality + (size_t)b * cv.capacity;
-    const int cnt = (seg + NPAIR - 1) / NPAIR;   // contiguous ranges: few modality changes per pair
-    sg.w0 = w0 + pair * cnt;
-    sg.n_my = max(0, min(cnt, seg - pair * cnt));
-    if (is_score) {
-      float run_m, run_l;
-      score_warp<FMT>(sm, sg, pair, lane, run_m, run_l);
-      run_l += __shfl_xor_sync(0xffffffffu, run_l, 1);
-      run_l += __shfl_xor_sync(0xffffffffu, run_l, 2);
-      if ((lane & 3) == 0) { sm.wm[pair][lane >> 2] = run_m; sm.wl[pair][lane >> 2] = run_l; }
-    } else {
-      value_warp<FMT>(sm, sg, pair, lane);
-    }
-    __syncthreads();
-
-    // ---- merge the eight pairs into one partial
+  // ---- merge the pairs' pieces into one partial per (sequence, head) of the block's range
+  int pos = pos0;
+  while (pos < pos1) {
+    const Where wh = locate(pos);
+    const int seg = min(pos1 - pos, wh.nwin - wh.w0);
+    const int unit = wh.e * Hkv + wh.h;
+    const int pa = (pos - pos0) / cnt, pb = (pos + seg - 1 - pos0) / cnt;   // pairs that worked on it
+    const PairPartial* pieces = P.pair_parts + (size_t)unit + (size_t)blockIdx.x * NPAIR;
     PartialF* out = P.partials_f + (size_t)unit + blockIdx.x;
-    {
-      float M[GP];
+    // maxima of the pieces
+    for (int i = tid; i < (pb - pa + 1) * 5 * GP; i += NTHREADS) {
+      const int p = pa + i / (5 * GP), j = i % (5 * GP);
+      const PairPartial& pp = pieces[p];
+      if (j < 3 * GP) (&sm.mrg_m[p][0][0])[j] = (&pp.sm[0][0])[j];
+      else if (j < 4 * GP) sm.mrg_wm[p][j - 3 * GP] = pp.wm[j - 3 * GP];
+      else sm.mrg_wl[p][j - 4 * GP] = pp.wl[j - 4 * GP];
+    }
+    __syncthreads();
+    if (tid < GP) {
+      float mj = -INFINITY, L = 0.f;
+      for (int p = pa; p <= pb; p++) mj = fmaxf(mj, sm.mrg_wm[p][tid]);
+      for (int p = pa; p <= pb; p++) L += sm.mrg_wl[p][tid] * exp2f(sm.mrg_wm[p][tid] - mj);
+      sm.mrg_M[tid] = mj;
+      out->m[tid] = mj;
+      out->l[tid] = L;
+    }
+    __syncthreads();
+    // four lanes' worth of one (modality, register) row per thread
+    for (int idx = tid; idx < 3 * SPILL_REGS * 8; idx += NTHREADS) {
+      const int l4 = (idx & 7) * 4, r = (idx >> 3) % SPILL_REGS, m = idx / (SPILL_REGS * 8);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int p = pa; p <= pb; p++) {
+        if (sm.mrg_m[p][m][0] == -INFINITY) continue;   // the pair saw no token of this modality
+        const float4 x = *reinterpret_cast<const float4*>(&pieces[p].frag[m][r][l4]);
+        float f[4];
 #pragma unroll
-      for (int j = 0; j < GP; j++) {
-        float mj = -INFINITY;
-#pragma unroll
-        for (int w8 = 0; w8 < NPAIR; w8++) mj = fmaxf(mj, sm.wm[w8][j]);
-        M[j] = mj;
-      }
-      if (tid < GP) {
-        float L = 0.f;
-        for (int w8 = 0; w8 < NPAIR; w8++)
-          L += sm.wm[w8][tid] == -INFINITY ? 0.f : sm.wl[w8][tid] * exp2f(sm.wm[w8][tid] - M[tid]);
-        out->m[tid] = M[tid];
-        out->l[tid] = L;
-      }
-      for (int idx = tid; idx < 3 * SPILL_REGS * 32; idx += NTHREADS) {
-        const int l32 = idx & 31, r = (idx >> 5) % SPILL_REGS, m = idx / (SPILL_REGS * 32);
-        const int head = r < 32 ? 2 * (l32 & 3) + (r & 1) : (l32 >> 2);
-        float v = 0.f;
-#pragma unroll
-        for (int w8 = 0; w8 < NPAIR; w8++) {
-          const float smx = sm.spill_m[w8][m][head];
-          if (smx != -INFINITY) v = fmaf(sm.spill[w8][m][r][l32], exp2f(smx - M[head]), v);
+        for (int i = 0; i < 4; i++) {
+          const int head = r < 32 ? 2 * i + (r & 1) : (l4 >> 2);   // lane l4 + i holds heads 2 (lane & 3) + (r & 1)
+          f[i] = exp2f(sm.mrg_m[p][m][head] - sm.mrg_M[head]);
         }
-        if (r < 32) out->frag[m][r][l32] = v;
-        else out->Sp[m][l32] = v;
+        v.x = fmaf(x.x, f[0], v.x); v.y = fmaf(x.y, f[1], v.y); v.z = fmaf(x.z, f[2], v.z); v.w = fmaf(x.w, f[3], v.w);
       }
+      if (r < 32) *reinterpret_cast<float4*>(&out->frag[m][r][l4]) = v;
+      else *reinterpret_cast<float4*>(&out->Sp[m][l4]) = v;
     }
     __syncthreads();
     pos += seg;

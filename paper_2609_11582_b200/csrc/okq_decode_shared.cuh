@@ -24,6 +24,16 @@ struct PartialF {
   float frag[3][32][32];
 };
 
+// tensor-core kernel: what one warp pair accumulated over its part of one (sequence, head); the CTA
+// merges its pairs' pieces into the PartialF records at the end of the launch
+constexpr int MMA_PAIRS = 8;        // warp pairs per CTA
+constexpr int PAIR_REGS = 33;       // 32 accumulator registers + the running weight sum, per lane
+struct PairPartial {
+  float frag[3][PAIR_REGS][32];   // [modality][register][lane]
+  float sm[3][GP];                // running maximum the modality's accumulators refer to (-inf: none)
+  float wm[GP], wl[GP];           // running maximum and sum of exp2(score - maximum) per head
+};
+
 struct DecodeParams {
   CacheView cv;
   int layer0, layer_count, n_splits, group;
@@ -34,6 +44,7 @@ struct DecodeParams {
   float sm_scale;
   Partial* partials;   // CUDA-core path: [layer_count*batch*n_kv_heads][n_splits]
   PartialF* partials_f;  // tensor-core path: [n_units + n_cta]
+  PairPartial* pair_parts;  // tensor-core path: [n_units + 8 * n_cta]
   float* out;          // [layer_count][batch][n_q_heads][128]
 };
 

@@ -2,7 +2,7 @@
 
 Some callers of this library run where device allocation is not allowed at call time: a serving
 loop whose memory pool was fixed at start-up, a plugin that only receives its inputs and
-outputs.  For them the library carries its own 32 MiB scratch array per GPU.  This test calls
+outputs.  For them the library carries its own 64 MiB scratch array per GPU.  This test calls
 the entry point through the C ABI twice in a row (the array keeps the previous call's contents,
 so the second call shows that nothing stale is picked up) and checks each result against
 okq_decode_attention with a caller-owned workspace, and against the CPU oracle.
@@ -24,7 +24,7 @@ D = 128
 
 
 def test_noalloc_rejects_oversized_request_without_a_gpu():
-    # 48 layers x 16 sequences x 4 heads = 3072 partials + the CTAs: more than the 32 MiB scratch holds
+    # 48 layers x 16 sequences x 4 heads = 3072 partials + the CTAs: more than the 64 MiB scratch holds
     c = B.okq_cache(48, 16, 4, 32, 128, 32, 32768, 0, 0, 0, 1 << 20, 1 << 20, 1 << 20, 1 << 20, 1 << 20, 1 << 20)
     st = B.lib().okq_decode_attention_noalloc(C.byref(c), 0, 48, 1 << 20, 0.1, 1 << 20, 1 << 20, 1, 0, 1 << 20, None)
     assert st == B.ERR_WORKSPACE
