@@ -60,8 +60,14 @@ struct MmaSmem {
   __align__(16) Handoff hand[NPAIR][2];
   __align__(16) float spill[NPAIR][3][32][SPILL_STRIDE];   // [pair][modality][lane]: the lane's 33 sums, 128-bit rows
   float spill_m[NPAIR][3][GP];
-  float mrg_m[NPAIR][3][GP], mrg_wm[NPAIR][GP], mrg_wl[NPAIR][GP], mrg_M[GP];   // end-of-launch merge: the pieces' maxima
   int prefix[MAX_ENTRIES + 1];
+};
+
+constexpr int MB_SEG = 32;                      // (sequence, head) units merged per batch at the end of the launch
+struct MergeSmem {
+  int pa[MB_SEG], pb[MB_SEG];                   // first and last warp pair that worked on the unit (pb < pa: none)
+  float meta[MB_SEG + NPAIR][5 * GP];           // per piece: sm[3][GP], wm[GP], wl[GP]; index = unit + pair - pa[0]
+  float M[MB_SEG][GP];                          // merged running maximum
 };
 
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -553,53 +559,105 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
   }
   __syncthreads();   // the pieces were written by this block's own warps: visible to the block from here on
 
-  // ---- merge the pairs' pieces into one partial per (sequence, head) of the block's range
-  int pos = pos0;
-  while (pos < pos1) {
-    const Where wh = locate(pos);
-    const int seg = min(pos1 - pos, wh.nwin - wh.w0);
-    const int unit = wh.e * Hkv + wh.h;
-    const int pa = (pos - pos0) / cnt, pb = (pos + seg - 1 - pos0) / cnt;   // pairs that worked on it
-    const PairPartial* pieces = P.pair_parts + (size_t)unit + (size_t)blockIdx.x * NPAIR;
-    PartialF* out = P.partials_f + (size_t)unit + blockIdx.x;
-    // maxima of the pieces
-    for (int i = tid; i < (pb - pa + 1) * 5 * GP; i += NTHREADS) {
-      const int p = pa + i / (5 * GP), j = i % (5 * GP);
-      const PairPartial& pp = pieces[p];
-      if (j < 3 * GP) (&sm.mrg_m[p][0][0])[j] = (&pp.sm[0][0])[j];
-      else if (j < 4 * GP) sm.mrg_wm[p][j - 3 * GP] = pp.wm[j - 3 * GP];
-      else sm.mrg_wl[p][j - 4 * GP] = pp.wl[j - 4 * GP];
+  // ---- merge the pairs' pieces into one partial per (sequence, head) of the block's range, MB_SEG
+  // (sequence, head) units at a time so that the loads of many units are in flight together.  The tables
+  // take the place of the record ring, which is idle by now.
+  if (pos0 >= pos1) return;
+  MergeSmem& mg = *reinterpret_cast<MergeSmem*>(smem_raw);
+  const Where wf = locate(pos0), wl = locate(pos1 - 1);
+  const int u_first = wf.e * Hkv + wf.h, u_last = wl.e * Hkv + wl.h;
+  for (int ub = u_first; ub <= u_last; ub += MB_SEG) {
+    const int n_u = min(MB_SEG, u_last - ub + 1);
+    // (a) the units' window ranges inside the block's slice and the pairs that worked on them
+    if (tid < n_u) {
+      const int u = ub + tid, e = u / Hkv, h = u % Hkv;
+      const int nwin = (sm.prefix[e + 1] - sm.prefix[e]) / Hkv;
+      const int a0 = max(pos0, sm.prefix[e] + h * nwin), a1 = min(pos1, sm.prefix[e] + (h + 1) * nwin);
+      mg.pa[tid] = a1 > a0 ? (a0 - pos0) / cnt : 0;
+      mg.pb[tid] = a1 > a0 ? (a1 - 1 - pos0) / cnt : -1;   // empty: a (sequence, head) with no packed window
     }
     __syncthreads();
-    if (tid < GP) {
-      float mj = -INFINITY, L = 0.f;
-      for (int p = pa; p <= pb; p++) mj = fmaxf(mj, sm.mrg_wm[p][tid]);
-      for (int p = pa; p <= pb; p++) L += sm.mrg_wl[p][tid] * exp2f(sm.mrg_wm[p][tid] - mj);
-      sm.mrg_M[tid] = mj;
-      out->m[tid] = mj;
-      out->l[tid] = L;
+    // (b) the pieces' maxima and weight sums: one warp per (unit, pair)
+    for (int j = warp; j < n_u * NPAIR; j += NTHREADS / 32) {
+      const int su = j / NPAIR, p = j % NPAIR;
+      if (p < mg.pa[su] || p > mg.pb[su]) continue;
+      const PairPartial& pp = P.pair_parts[(size_t)(ub + su) + (size_t)blockIdx.x * NPAIR + p];
+      float* dst = mg.meta[su + p - mg.pa[0]];
+      dst[lane] = (&pp.sm[0][0])[lane];                         // sm[3][GP], then wm[GP]
+      if (lane < GP) dst[32 + lane] = pp.wl[lane];
     }
     __syncthreads();
-    // four lanes' worth of one (modality, register) row per thread
-    for (int idx = tid; idx < 3 * SPILL_REGS * 8; idx += NTHREADS) {
-      const int l4 = (idx & 7) * 4, r = (idx >> 3) % SPILL_REGS, m = idx / (SPILL_REGS * 8);
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int p = pa; p <= pb; p++) {
-        if (sm.mrg_m[p][m][0] == -INFINITY) continue;   // the pair saw no token of this modality
-        const float4 x = *reinterpret_cast<const float4*>(&pieces[p].frag[m][r][l4]);
-        float f[4];
-#pragma unroll
-        for (int i = 0; i < 4; i++) {
-          const int head = r < 32 ? 2 * i + (r & 1) : (l4 >> 2);   // lane l4 + i holds heads 2 (lane & 3) + (r & 1)
-          f[i] = exp2f(sm.mrg_m[p][m][head] - sm.mrg_M[head]);
+    // (c) merged maximum and weight sum per (unit, head)
+    if (tid < n_u * GP) {
+      const int su = tid / GP, j = tid % GP;
+      if (mg.pb[su] >= mg.pa[su]) {
+        float mj = -INFINITY, L = 0.f;
+        for (int p = mg.pa[su]; p <= mg.pb[su]; p++) mj = fmaxf(mj, mg.meta[su + p - mg.pa[0]][3 * GP + j]);
+        for (int p = mg.pa[su]; p <= mg.pb[su]; p++) {
+          const float* me = mg.meta[su + p - mg.pa[0]];
+          L += me[4 * GP + j] * exp2f(me[3 * GP + j] - mj);
         }
-        v.x = fmaf(x.x, f[0], v.x); v.y = fmaf(x.y, f[1], v.y); v.z = fmaf(x.z, f[2], v.z); v.w = fmaf(x.w, f[3], v.w);
+        mg.M[su][j] = mj;
+        PartialF* out = P.partials_f + (size_t)(ub + su) + blockIdx.x;
+        out->m[j] = mj;
+        out->l[j] = L;
       }
-      if (r < 32) *reinterpret_cast<float4*>(&out->frag[m][r][l4]) = v;
-      else *reinterpret_cast<float4*>(&out->Sp[m][l4]) = v;
     }
     __syncthreads();
-    pos += seg;
+    // (d) the accumulators: one item = four lanes' worth of one (unit, modality, register) row
+    constexpr int ROW_ITEMS = 3 * SPILL_REGS * 8, MU = 4, MP = 3;
+    for (int base = tid; base < n_u * ROW_ITEMS; base += MU * NTHREADS) {
+      float4 x[MU][MP];
+#pragma unroll
+      for (int u4 = 0; u4 < MU; u4++) {
+        const int it = base + u4 * NTHREADS;
+#pragma unroll
+        for (int q = 0; q < MP; q++) x[u4][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (it < n_u * ROW_ITEMS) {
+          const int su = it / ROW_ITEMS, idx = it % ROW_ITEMS;
+          const int l4 = (idx & 7) * 4, r = (idx >> 3) % SPILL_REGS, m = idx / (SPILL_REGS * 8);
+#pragma unroll
+          for (int q = 0; q < MP; q++) {
+            const int p = mg.pa[su] + q;
+            if (p <= mg.pb[su] && mg.meta[su + p - mg.pa[0]][m * GP] != -INFINITY)   // else: no token of this modality
+              x[u4][q] = *reinterpret_cast<const float4*>(
+                  &P.pair_parts[(size_t)(ub + su) + (size_t)blockIdx.x * NPAIR + p].frag[m][r][l4]);
+          }
+        }
+      }
+#pragma unroll
+      for (int u4 = 0; u4 < MU; u4++) {
+        const int it = base + u4 * NTHREADS;
+        if (it >= n_u * ROW_ITEMS) continue;
+        const int su = it / ROW_ITEMS, idx = it % ROW_ITEMS;
+        if (mg.pb[su] < mg.pa[su]) continue;
+        const int l4 = (idx & 7) * 4, r = (idx >> 3) % SPILL_REGS, m = idx / (SPILL_REGS * 8);
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p = mg.pa[su]; p <= mg.pb[su]; p++) {
+          const float* me = mg.meta[su + p - mg.pa[0]] + m * GP;
+          if (me[0] == -INFINITY) continue;
+          const int q = p - mg.pa[su];
+          float4 xx;
+          if (q < MP) {
+            xx = q == 0 ? x[u4][0] : (q == 1 ? x[u4][1] : x[u4][2]);
+          } else {   // more than MP pairs on one unit: short slices
+            xx = *reinterpret_cast<const float4*>(
+                &P.pair_parts[(size_t)(ub + su) + (size_t)blockIdx.x * NPAIR + p].frag[m][r][l4]);
+          }
+          float f[4];
+#pragma unroll
+          for (int i = 0; i < 4; i++) {
+            const int head = r < 32 ? 2 * i + (r & 1) : (l4 >> 2);   // lane l4 + i holds heads 2 (lane & 3) + (r & 1)
+            f[i] = exp2f(me[head] - mg.M[su][head]);
+          }
+          v.x = fmaf(xx.x, f[0], v.x); v.y = fmaf(xx.y, f[1], v.y); v.z = fmaf(xx.z, f[2], v.z); v.w = fmaf(xx.w, f[3], v.w);
+        }
+        PartialF* out = P.partials_f + (size_t)(ub + su) + blockIdx.x;
+        if (r < 32) *reinterpret_cast<float4*>(&out->frag[m][r][l4]) = v;
+        else *reinterpret_cast<float4*>(&out->Sp[m][l4]) = v;
+      }
+    }
+    __syncthreads();
   }
 }
 
