@@ -31,8 +31,6 @@ class Case:
                              meta_format=meta_format)
         self.mod = WL.modality_layout(w, self.n) if modality is None else modality   # [n]
         self.mod_b = self.mod.unsqueeze(0).repeat(w.batch, 1).contiguous()  # [B, n], as the caller passes it
-        # the oracle takes ids in {0, 1, 2}: ids > 2 count as text
-        self.mod_o = torch.where(self.mod_b > 2, torch.zeros_like(self.mod_b), self.mod_b).numpy()
         self.signs = torch.stack([WL.gen_signs(w, l) for l in range(w.n_layers)])      # [L,128]
         self.R = torch.stack([WL.gen_rotations(w, l) for l in range(w.n_layers)])      # [L,3,128,128]
         self.q = torch.stack([WL.gen_queries(w, l) for l in range(w.n_layers)])        # [L,B,Hq,128]
@@ -49,6 +47,11 @@ class Case:
         torch.cuda.synchronize()
 
     # ---- oracle side
+    @property
+    def mod_o(self):
+        """Modality ids as the oracle takes them ({0, 1, 2}: ids > 2 count as text), from the current mod_b."""
+        return torch.where(self.mod_b > 2, torch.zeros_like(self.mod_b), self.mod_b).numpy()
+
     def oracle_quantize(self, layer):
         w = self.w
         U = w.batch * w.n_kv_heads
