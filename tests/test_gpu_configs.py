@@ -2,6 +2,7 @@
 
   * 30B-A3B shape (GQA group 8, video 400 / audio 100 chunks), reduced layers and context;
   * long-context decode (batch 1, many CTAs per (sequence, head));
+  * long single-modality ranges per warp pair, and thousands of two-window units in one launch;
   * the full 7B decode step (28 layers x batch 8 x 16384 tokens, one append + one decode call
     over all layers, inputs drawn on the GPU exactly as bench.py does), checked on sampled
     (layer, sequence) pairs the oracle can afford, plus properties that hold at any size.
@@ -41,6 +42,33 @@ def test_long_context_batch1():
     print("long context", Hn.assert_attention_close(got, ref))
     got4 = c.gpu_decode(0, num_splits=3)[0]
     Hn.assert_attention_close(got4, ref)
+
+
+def test_one_modality_long_ranges():
+    """One warp pair covers 256 windows of a single modality (one CTA per (sequence, head), no modality change
+    that would move the register sums out): the value sums must not drift with the length of the range.  The
+    tensor cores accumulate without rounding to nearest, so a long chain into one register is biased; the
+    kernel bounds the chain, and this case fails (worst head above the tolerance) if it does not."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], n_tokens=65536 + 3)
+    c = Hn.Case(w, modality=torch.zeros(w.n_tokens, dtype=torch.uint8))
+    ref, _ = c.oracle_attention(0)
+    for splits in (1, 0):
+        got = c.gpu_decode(0, num_splits=splits)[0]
+        errs = Hn.assert_attention_close(got, ref)
+        assert errs[1] < 6e-4, errs      # worst head: well inside the 1e-3 tolerance
+        print("one modality, splits", splits, errs)
+
+
+def test_many_short_units_per_cta():
+    """8192 (sequence, head) units of two windows each in one launch: every warp pair crosses several unit
+    boundaries and every CTA merges ~55 units, more than one batch of its end-of-launch merge."""
+    w = WL.Workload("short", 5, 8, 128, 16, 8, 64 + 5, 16, 20, 12, 0)
+    c = Hn.Case(w)
+    got = c.gpu_decode(0, layer_count=w.n_layers)
+    for l in range(w.n_layers):
+        ref, _ = c.oracle_attention(l)
+        Hn.assert_attention_close(got[l], ref)
+    assert c.cache.device_status() == 0
 
 
 @pytest.mark.parametrize("meta_format", [B.META_FP16, B.META_MXFP4])
