@@ -189,6 +189,12 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
       const float2 r2 = *reinterpret_cast<const float2*>(&sm.b[c0]);
       mch[2 * q] = m2.x; mch[2 * q + 1] = m2.y; rch[2 * q] = r2.x; rch[2 * q + 1] = r2.y;
     }
+    // code = clamp(rint((z - m) / s), 0, 3).  Clamping first gives the same integer (rounding is monotone and
+    // keeps 0 and 3), and adding 1.5 * 2^23 to a value in [0, 3] rounds it to nearest-even into the low
+    // mantissa bits; the sixteen 2-bit fields are then summed with integer multiply-adds and the sixteen
+    // copies of the constant's bit pattern are taken off at the end (all modulo 2^32).
+    constexpr float MAGIC = 12582912.0f;                 // 1.5 * 2^23, bit pattern 0x4B400000
+    constexpr uint32_t MAGIC_SUM = 0x4B400000u * 0x55555555u;   // sum over the sixteen field positions 4^j
 #pragma unroll
     for (int k = 0; k < 2; k++) {
       const int i = tg + 16 * k;
@@ -199,11 +205,12 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
         const float2 z2 = *reinterpret_cast<const float2*>(&sm.z[i * ZS + zpos(c0)]);
 #pragma unroll
         for (int e = 0; e < 2; e++) {
-          const float qv = rintf(__fmul_rn(__fsub_rn(e ? z2.y : z2.x, mch[2 * q + e]), rch[2 * q + e]));
-          const uint32_t code = (uint32_t)fminf(fmaxf(qv, 0.0f), 3.0f);   // clamp to [0, 3]
-          word |= code << (16 * e + 8 * (q >> 2) + 2 * (q & 3));
+          const float u = __fmul_rn(__fsub_rn(e ? z2.y : z2.x, mch[2 * q + e]), rch[2 * q + e]);
+          const float r = __fadd_rn(fminf(fmaxf(u, 0.0f), 3.0f), MAGIC);
+          word += __float_as_uint(r) << (16 * e + 8 * (q >> 2) + 2 * (q & 3));
         }
       }
+      word -= MAGIC_SUM;
       // word index of (token i, t, ww): [i >> 4][lane 4*(i & 7) + t][(i >> 3) & 1][ww]
       words[(i >> 4) * 128 + (4 * (i & 7) + t) * 4 + ((i >> 3) & 1) * 2 + ww] = word;
     }
