@@ -38,16 +38,41 @@ struct WindowSmem {
 // first four levels of the norm's summation tree), then each holds the 2 x 8 channels that differ in
 // the three high index bits (stages h = 16, 32, 64).  The stage order, and with it every rounding,
 // is that of the plain butterfly loop.
+// two fp32 values in one 64-bit register and the packed arithmetic on them (each half rounds like the scalar op)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
 __device__ void quantize_key_window(const __half* rows, long long stride, const float* __restrict__ signs,
                                     unsigned char* rec, unsigned char* body, int fmt, WindowSmem& sm) {
   const int tid = threadIdx.x;
   __half* knorm = reinterpret_cast<__half*>(body + B_KNORM);
   const int a = tid & 7;          // which 16-channel block (first half) / which channel pair (second half)
-  float sg[16];
+  uint64_t sgp[8];   // the signs of the thread's 16 channels, two per register
 #pragma unroll
   for (int q = 0; q < 4; q++) {
     const float4 s4 = *reinterpret_cast<const float4*>(signs + 16 * a + 4 * q);
-    sg[4 * q] = s4.x; sg[4 * q + 1] = s4.y; sg[4 * q + 2] = s4.z; sg[4 * q + 3] = s4.w;
+    sgp[2 * q] = pack2(s4.x, s4.y); sgp[2 * q + 1] = pack2(s4.z, s4.w);
   }
 #pragma unroll 1
   for (int round = 0; round < 2; round++) {
@@ -65,10 +90,15 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
         y[2 * q] = f0.x; y[2 * q + 1] = f0.y; y[8 + 2 * q] = f1.x; y[8 + 2 * q + 1] = f1.y;
       }
     }
+    // Two channels per instruction (add / sub / mul .f32x2: each half is the same IEEE operation as the
+    // scalar one, so the results do not change): P[i] = (y[2i], y[2i+1]).
+    uint64_t P[8];
+#pragma unroll
+    for (int q = 0; q < 8; q++) P[q] = pack2(y[2 * q], y[2 * q + 1]);
     // norm: adjacent-pair tree (4 levels here, 3 across the eight threads)
     float t[16];
 #pragma unroll
-    for (int c = 0; c < 16; c++) t[c] = __fmul_rn(y[c], y[c]);
+    for (int q = 0; q < 8; q++) unpack2(mul2(P[q], P[q]), t[2 * q], t[2 * q + 1]);
 #pragma unroll
     for (int n = 8; n >= 1; n >>= 1)
 #pragma unroll
@@ -83,44 +113,45 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
     const float nf = __half2float(nh);
     if (a == 0) knorm[norm_pos(i)] = nh;
     const float cinv = nf != 0.0f ? __fdiv_rn(RSQRT_D, nf) : 0.0f;
-    // D x, then stages h = 1, 2, 4, 8 inside the 16-channel block
+    // D x, then stages h = 1, 2, 4, 8 inside the 16-channel block: h = 1 pairs the two halves of one P[i]
+    // (scalar), h = 2, 4, 8 pair P[i] with P[i + h/2]
 #pragma unroll
-    for (int c = 0; c < 16; c++) y[c] = __fmul_rn(sg[c], y[c]);
-#pragma unroll
-    for (int hh = 1; hh < 16; hh <<= 1)
-#pragma unroll
-      for (int j = 0; j < 16; j++)
-        if ((j & hh) == 0) {
-          const float p = y[j], q2 = y[j + hh];
-          y[j] = __fadd_rn(p, q2);
-          y[j + hh] = __fsub_rn(p, q2);
-        }
-#pragma unroll
-    for (int q = 0; q < 4; q++)
-      *reinterpret_cast<float4*>(&zrow[zpos(16 * a + 4 * q)]) = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
-    __syncwarp();
-    // second half: channels 16*u + 2*a + e, u = 0..7: stages h = 16, 32, 64 act on u
-    float v0[8], v1[8];
-#pragma unroll
-    for (int u = 0; u < 8; u++) {
-      const float2 p = *reinterpret_cast<const float2*>(&zrow[zpos(16 * u + 2 * a)]);
-      v0[u] = p.x; v1[u] = p.y;
+    for (int q = 0; q < 8; q++) {
+      float lo, hi;
+      unpack2(mul2(sgp[q], P[q]), lo, hi);
+      P[q] = pack2(__fadd_rn(lo, hi), __fsub_rn(lo, hi));
     }
 #pragma unroll
     for (int hh = 1; hh < 8; hh <<= 1)
 #pragma unroll
       for (int j = 0; j < 8; j++)
         if ((j & hh) == 0) {
-          float p = v0[j], q2 = v0[j + hh];
-          v0[j] = __fadd_rn(p, q2); v0[j + hh] = __fsub_rn(p, q2);
-          p = v1[j]; q2 = v1[j + hh];
-          v1[j] = __fadd_rn(p, q2); v1[j + hh] = __fsub_rn(p, q2);
+          const uint64_t p = P[j], q2 = P[j + hh];
+          P[j] = add2(p, q2);
+          P[j + hh] = sub2(p, q2);
+        }
+#pragma unroll
+    for (int q = 0; q < 4; q++)
+      *reinterpret_cast<ulonglong2*>(&zrow[zpos(16 * a + 4 * q)]) = make_ulonglong2(P[2 * q], P[2 * q + 1]);
+    __syncwarp();
+    // second half: channels 16*u + 2*a + e, u = 0..7: stages h = 16, 32, 64 act on u; Q[u] = both e
+    uint64_t Q[8];
+#pragma unroll
+    for (int u = 0; u < 8; u++) Q[u] = *reinterpret_cast<const uint64_t*>(&zrow[zpos(16 * u + 2 * a)]);
+#pragma unroll
+    for (int hh = 1; hh < 8; hh <<= 1)
+#pragma unroll
+      for (int j = 0; j < 8; j++)
+        if ((j & hh) == 0) {
+          const uint64_t p = Q[j], q2 = Q[j + hh];
+          Q[j] = add2(p, q2);
+          Q[j + hh] = sub2(p, q2);
         }
     __syncwarp();   // every thread of the token has read the first-half values before they are overwritten
+    const uint64_t cinv2 = pack2(cinv, cinv);
 #pragma unroll
     for (int u = 0; u < 8; u++)
-      *reinterpret_cast<float2*>(&zrow[zpos(16 * u + 2 * a)]) =
-          nf != 0.0f ? make_float2(__fmul_rn(v0[u], cinv), __fmul_rn(v1[u], cinv)) : make_float2(0.f, 0.f);
+      *reinterpret_cast<uint64_t*>(&zrow[zpos(16 * u + 2 * a)]) = nf != 0.0f ? mul2(Q[u], cinv2) : 0ull;
   }
   __syncthreads();
   {  // per channel: window minimum and step (Eq. 4)
@@ -181,20 +212,20 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
   {
     uint32_t* words = reinterpret_cast<uint32_t*>(body + B_KCODE);
     const int t = tid & 3, ww = (tid >> 2) & 1, tg = tid >> 3;   // tokens tg and tg + 16
-    float mch[16], rch[16];
+    uint64_t mch[8], rch[8];   // (m, 1/s) of the channel pairs 2q, 2q+1 of the word
 #pragma unroll
     for (int q = 0; q < 8; q++) {
       const int c0 = 16 * ((ww * 8 + q) >> 1) + 8 * (q & 1) + 2 * t;
-      const float2 m2 = *reinterpret_cast<const float2*>(&sm.a[c0]);
-      const float2 r2 = *reinterpret_cast<const float2*>(&sm.b[c0]);
-      mch[2 * q] = m2.x; mch[2 * q + 1] = m2.y; rch[2 * q] = r2.x; rch[2 * q + 1] = r2.y;
+      mch[q] = *reinterpret_cast<const uint64_t*>(&sm.a[c0]);
+      rch[q] = *reinterpret_cast<const uint64_t*>(&sm.b[c0]);
     }
     // code = clamp(rint((z - m) / s), 0, 3).  Clamping first gives the same integer (rounding is monotone and
     // keeps 0 and 3), and adding 1.5 * 2^23 to a value in [0, 3] rounds it to nearest-even into the low
-    // mantissa bits; the sixteen 2-bit fields are then summed with integer multiply-adds and the sixteen
+    // mantissa bits; the sixteen 2-bit fields are then summed with integer shift-adds and the sixteen
     // copies of the constant's bit pattern are taken off at the end (all modulo 2^32).
     constexpr float MAGIC = 12582912.0f;                 // 1.5 * 2^23, bit pattern 0x4B400000
     constexpr uint32_t MAGIC_SUM = 0x4B400000u * 0x55555555u;   // sum over the sixteen field positions 4^j
+    const uint64_t magic2 = pack2(MAGIC, MAGIC);
 #pragma unroll
     for (int k = 0; k < 2; k++) {
       const int i = tg + 16 * k;
@@ -202,13 +233,13 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
 #pragma unroll
       for (int q = 0; q < 8; q++) {
         const int c0 = 16 * ((ww * 8 + q) >> 1) + 8 * (q & 1) + 2 * t;
-        const float2 z2 = *reinterpret_cast<const float2*>(&sm.z[i * ZS + zpos(c0)]);
-#pragma unroll
-        for (int e = 0; e < 2; e++) {
-          const float u = __fmul_rn(__fsub_rn(e ? z2.y : z2.x, mch[2 * q + e]), rch[2 * q + e]);
-          const float r = __fadd_rn(fminf(fmaxf(u, 0.0f), 3.0f), MAGIC);
-          word += __float_as_uint(r) << (16 * e + 8 * (q >> 2) + 2 * (q & 3));
-        }
+        const uint64_t z2 = *reinterpret_cast<const uint64_t*>(&sm.z[i * ZS + zpos(c0)]);
+        float u0, u1;
+        unpack2(mul2(sub2(z2, mch[q]), rch[q]), u0, u1);
+        float r0, r1;
+        unpack2(add2(pack2(fminf(fmaxf(u0, 0.0f), 3.0f), fminf(fmaxf(u1, 0.0f), 3.0f)), magic2), r0, r1);
+        word += __float_as_uint(r0) << (8 * (q >> 2) + 2 * (q & 3));
+        word += __float_as_uint(r1) << (16 + 8 * (q >> 2) + 2 * (q & 3));
       }
       word -= MAGIC_SUM;
       // word index of (token i, t, ww): [i >> 4][lane 4*(i & 7) + t][(i >> 3) & 1][ww]
