@@ -59,6 +59,16 @@ def test_one_modality_long_ranges():
         print("one modality, splits", splits, errs)
 
 
+def test_decode_is_deterministic():
+    """No atomics and a fixed partition: two calls on the same cache give bit-identical outputs (both grids)."""
+    w = WL.scaled(WL.WORKLOADS["step7b"], n_layers=2, batch=3, n_tokens=2048 + 17)
+    c = Hn.Case(w)
+    for splits in (0, 2):
+        a = c.gpu_decode(0, layer_count=2, num_splits=splits)
+        b = c.gpu_decode(0, layer_count=2, num_splits=splits)
+        assert np.array_equal(a, b)
+
+
 def test_many_short_units_per_cta():
     """8192 (sequence, head) units of two windows each in one launch: every warp pair crosses several unit
     boundaries and every CTA merges ~55 units, more than one batch of its end-of-launch merge."""
