@@ -661,8 +661,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
   }
 }
 
-constexpr int CB_SEQ = 4;                 // sequences per combine CTA (one 128-thread group each)
-constexpr int CB_ROWS = CB_SEQ * GP;      // (sequence, head) rows per combine CTA
+constexpr int CB_SEQ_MAX = 4;             // most sequences per combine CTA (one 128-thread group each)
 
 constexpr int MRG_MAX = 8;                // partials per (sequence, head) whose factors are precomputed
 constexpr int CB_CHUNK = 16;              // rows of a rotation matrix staged per step
@@ -670,8 +669,11 @@ constexpr int CB_NBUF = 4;                // staged slices in flight (three ahea
 
 // CAPTION: the captioning schedule keeps up to 159 raw values (and up to 127 raw keys) per sequence, and
 // the keys of the raw values' tokens may already be packed
-template <bool CAPTION>
+// SEQ: sequences per CTA (4 for full grids: the matrices are streamed once per four sequences; 1 when the
+// grid would otherwise leave most SMs idle, e.g. a single-layer call)
+template <bool CAPTION, int SEQ>
 struct CombineSmem {
+  static constexpr int CB_SEQ = SEQ, CB_ROWS = SEQ * GP;
   static constexpr int TAIL = CAPTION ? CAPTION_V_SLOTS : W;   // most raw-value tokens of a sequence
   __align__(16) float Rbuf[CB_NBUF][CB_CHUNK][D];   // ring of 16-row slices of the rotation matrices
   __align__(16) float mrg[CB_SEQ][MRG_MAX][GP][4];                // per partial and head: rescale factor, weight sums of the modalities
@@ -698,10 +700,11 @@ __device__ __forceinline__ float2 window_meta_pos(const unsigned char* meta, int
 
 // NS: CTAs that share one (head, sequence group): each computes D / NS output columns (used when the grid
 // would otherwise leave most SMs idle; the merge is repeated by every slice, the matrix streaming is split)
-template <bool CAPTION, int NS>
-__global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, int n_cta) {
+template <bool CAPTION, int NS, int SEQ>
+__global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n_cta) {
+  constexpr int CB_SEQ = SEQ, CB_ROWS = SEQ * GP;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  CombineSmem<CAPTION>& sm = *reinterpret_cast<CombineSmem<CAPTION>*>(smem_raw);
+  CombineSmem<CAPTION, SEQ>& sm = *reinterpret_cast<CombineSmem<CAPTION, SEQ>*>(smem_raw);
   const CacheView& cv = P.cv;
   const int h = blockIdx.x / NS, sl = blockIdx.x % NS, li = blockIdx.z, layer = P.layer0 + li;
   const int bs = threadIdx.x >> 7, c = threadIdx.x & 127;
@@ -911,10 +914,10 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
     }
   }
 
-  // out[row][c] = raw[row][c] + sum_m sum_r R_m[r][c] * vec[m][row][r].  Threads 0..255 compute a
-  // 4-row x 4-column tile each; threads 256..511 stream the matrices through shared memory in
-  // 32-row slices, one slice ahead.
-  const bool comp = threadIdx.x < 256;
+  // out[row][c] = raw[row][c] + sum_m sum_r R_m[r][c] * vec[m][row][r].  The first half of the threads compute
+  // a 4-row x 4-column tile each; the second half stream the matrices through shared memory in 16-row
+  // slices, three slices ahead.
+  const bool comp = threadIdx.x < CB_SEQ * 64;
   constexpr int CW = 4 / NS;          // output columns per compute thread
   constexpr int SW = D / NS;          // output columns of this CTA = floats per staged matrix row
   static_assert(NS == 1 || NS == 4, "column slices");
@@ -926,7 +929,7 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
     const float* src = Rset + (size_t)chunk * CB_CHUNK * D;
     float* dst = rbuf + (chunk % CB_NBUF) * CB_CHUNK * SW;
     if (chunk < N_CHUNK)
-      for (int i = threadIdx.x - 256; i < CB_CHUNK * SW / 4; i += 256) {
+      for (int i = threadIdx.x - CB_SEQ * 64; i < CB_CHUNK * SW / 4; i += CB_SEQ * 64) {
         const int row = i / (SW / 4), c4 = i % (SW / 4);
         cp_async16(dst + row * SW + 4 * c4, src + (size_t)row * D + 4 * c4);
       }
@@ -995,6 +998,29 @@ __global__ void __launch_bounds__(CB_SEQ * 128) k_combine_mma(DecodeParams P, in
   }
 }
 
+template <bool CAPTION, int NS, int SEQ>
+static cudaError_t combine_attr() {
+  return cudaFuncSetAttribute(k_combine_mma<CAPTION, NS, SEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)sizeof(CombineSmem<CAPTION, SEQ>));
+}
+
+template <bool CAPTION, int NS, int SEQ>
+static void combine_launch(const DecodeParams& P, int n_cta, cudaStream_t s) {
+  const dim3 grid(P.cv.n_kv_heads * NS, (P.cv.batch + SEQ - 1) / SEQ, P.layer_count);
+  k_combine_mma<CAPTION, NS, SEQ><<<grid, SEQ * 128, sizeof(CombineSmem<CAPTION, SEQ>), s>>>(P, n_cta);
+}
+
+template <bool CAPTION>
+static void combine_dispatch(const DecodeParams& P, int n_cta, cudaStream_t s) {
+  // full grids: four sequences per block, so that a layer's matrices are streamed once per four sequences;
+  // fewer such blocks than SMs: one sequence per block; a handful (e.g. a single-layer call): one sequence
+  // and a quarter of the output columns per block
+  const int n_blocks = P.cv.n_kv_heads * ((P.cv.batch + CB_SEQ_MAX - 1) / CB_SEQ_MAX) * P.layer_count;
+  if (4 * n_blocks <= n_cta) combine_launch<CAPTION, 4, 1>(P, n_cta, s);
+  else if (n_blocks <= n_cta) combine_launch<CAPTION, 1, 1>(P, n_cta, s);
+  else combine_launch<CAPTION, 1, CB_SEQ_MAX>(P, n_cta, s);
+}
+
 okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, cudaEvent_t before, cudaEvent_t after) {
   static thread_local unsigned long long attr_mask = 0;
   int attr_dev = 0;
@@ -1004,14 +1030,12 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k_decode_mma<FMT_MXFP4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)sizeof(MmaSmem<FMT_MXFP4>));
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_combine_mma<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<false>));
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_combine_mma<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<false>));
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_combine_mma<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<true>));
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_combine_mma<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CombineSmem<true>));
+    if (e == cudaSuccess) e = combine_attr<false, 4, 1>();
+    if (e == cudaSuccess) e = combine_attr<false, 1, 1>();
+    if (e == cudaSuccess) e = combine_attr<false, 1, CB_SEQ_MAX>();
+    if (e == cudaSuccess) e = combine_attr<true, 4, 1>();
+    if (e == cudaSuccess) e = combine_attr<true, 1, 1>();
+    if (e == cudaSuccess) e = combine_attr<true, 1, CB_SEQ_MAX>();
     if (e != cudaSuccess) { set_last_cuda_error((int)e); return OKQ_ERR_CUDA; }
     attr_done(attr_mask, attr_dev);
   }
@@ -1019,15 +1043,8 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
   if (P.cv.fmt == FMT_MXFP4) k_decode_mma<FMT_MXFP4><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_MXFP4>), s>>>(P);
   else k_decode_mma<FMT_FP16><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_FP16>), s>>>(P);
   if (after) cudaEventRecord(after, s);
-  // few (head, sequence group, layer) blocks, e.g. a single-layer call: four column slices per block
-  const int n_blocks = P.cv.n_kv_heads * ((P.cv.batch + CB_SEQ - 1) / CB_SEQ) * P.layer_count;
-  const int ns = 4 * n_blocks <= n_cta ? 4 : 1;
-  const dim3 cgrid(P.cv.n_kv_heads * ns, (P.cv.batch + CB_SEQ - 1) / CB_SEQ, P.layer_count);
-  const bool cap = P.cv.sched == SCHED_CAPTION;
-  if (cap && ns == 4) k_combine_mma<true, 4><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<true>), s>>>(P, n_cta);
-  else if (cap) k_combine_mma<true, 1><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<true>), s>>>(P, n_cta);
-  else if (ns == 4) k_combine_mma<false, 4><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<false>), s>>>(P, n_cta);
-  else k_combine_mma<false, 1><<<cgrid, CB_SEQ * 128, sizeof(CombineSmem<false>), s>>>(P, n_cta);
+  if (P.cv.sched == SCHED_CAPTION) combine_dispatch<true>(P, n_cta, s);
+  else combine_dispatch<false>(P, n_cta, s);
   return OKQ_OK;
 }
 
