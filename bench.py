@@ -435,6 +435,38 @@ def main():
     achieved = packed_bytes / (kernel_ms * 1e-3) / 1e9
     traffic = (NCU_DRAM_BYTES_PER_TOKEN_HEAD_MX if mx else NCU_DRAM_BYTES_PER_TOKEN_HEAD) * L * Bn * H * N
 
+    # The same step as a model issues it: one okq_append + one okq_decode_attention per layer (2 L calls),
+    # captured once in a CUDA graph and replayed, so that the launch gaps between the per-layer kernels count.
+    def per_layer_graph_ms():
+        def one_step():
+            for l in range(L):
+                B.append(cache, l, 1, kn_dev[0][l:l + 1], vn_dev[0][l:l + 1], mn_dev, signs[l:l + 1], R[l:l + 1])
+                B.decode_attention(cache, l, 1, q_dev[l:l + 1], signs[l:l + 1], R[l:l + 1], ws, out[l:l + 1],
+                                   num_splits=args.splits)
+        cache.seq_len.copy_(seq0)
+        one_step()                       # every kernel has run once before the capture
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            one_step()
+        cache.seq_len.copy_(seq0)
+        for _ in range(args.warmup):
+            g.replay()
+        cache.seq_len.copy_(seq0)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        a.record()
+        for _ in range(args.steps):
+            g.replay()
+        b.record()
+        barrier()
+        cache.seq_len.copy_(seq0)
+        return a.elapsed_time(b) / args.steps
+
+    ms_graph = per_layer_graph_ms() if world == 1 else None
+    if cache.device_status() != 0:
+        raise RuntimeError("device status word set during the per-layer graph run")
+
     if rank != 0:
         return
     cpu = None
@@ -461,7 +493,11 @@ def main():
                     "d2h_bytes_per_step": out_host.numel() * 4,
                     "how": "copies on a second stream over two sets of device buffers: the transfers of neighbouring "
                            "steps overlap the kernels; timed from the first copy to the last read-back"},
-            "gpu_launches": 4 * args.steps,
+            "per_layer_graph": None if ms_graph is None else {
+                "us_per_step": ms_graph * 1e3, "value": packed_bytes / (ms_graph * 1e-3) / 1e9, "unit": "GB/s",
+                "calls_per_step": 2 * L,
+                "how": "one okq_append + one okq_decode_attention per layer, captured in one CUDA graph and replayed"},
+            "gpu_launches": 3 * args.steps,
             "roofline": {"bound": "hbm", "kernel": "okq split-K decode kernel (one launch per step)",
                          "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                          "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0,

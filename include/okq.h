@@ -171,7 +171,9 @@ okq_status okq_quantize_values_bulk(const okq_cache* cache, int32_t layer, const
  *   signs          device float [layer_count][128]
  *   R              device float [layer_count][n_R][3][128][128]
  * A sequence already at `capacity` is left unchanged and the device status word becomes
- * OKQ_ERR_CAPACITY.
+ * OKQ_ERR_CAPACITY.  One kernel launch; while it runs, the top byte of the touched seq_len
+ * entries holds a transient count (it is clear again when the kernel ends), which limits
+ * the call to capacity < 2^24 and n_kv_heads <= 127 (OKQ_ERR_UNSUPPORTED otherwise).
  */
 okq_status okq_append(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* k_new,
                       const void* v_new, const uint8_t* modality_new, const float* signs,

@@ -394,6 +394,8 @@ __global__ void k_bulk_tail(CacheView cv, int layer, const __half* __restrict__ 
 
 // ---------------------------------------------------------------- append
 
+constexpr int APPEND_ARRIVAL = 1 << 24;   // one arrived block in the transient count kept in seq_len's top byte
+
 // grid (n_kv_heads, batch, layer_count), 128 threads
 __global__ void __launch_bounds__(128) k_append(CacheView cv, int layer0, const __half* __restrict__ k_new,
                                                const __half* __restrict__ v_new,
@@ -401,8 +403,20 @@ __global__ void __launch_bounds__(128) k_append(CacheView cv, int layer0, const 
                                                const float* __restrict__ signs, const float* __restrict__ R,
                                                int n_R) {
   __shared__ WindowSmem sm;
+  __shared__ int s_pos;
   int h = blockIdx.x, b = blockIdx.y, li = blockIdx.z, layer = layer0 + li;
-  int pos = cv.seq_len[layer * cv.batch + b];
+  // The n_kv_heads blocks of a (layer, sequence) all need the position before any of them may advance it.
+  // Each block counts itself in the top byte of seq_len while reading it; the block that finds the others
+  // already counted stores the new length (which also clears the count): by then every block has its copy.
+  if (threadIdx.x == 0) {
+    int* len = cv.seq_len + layer * cv.batch + b;
+    const int old = atomicAdd(len, APPEND_ARRIVAL);
+    const int p = old & (APPEND_ARRIVAL - 1);
+    if (old / APPEND_ARRIVAL == cv.n_kv_heads - 1) *len = p < cv.capacity ? p + 1 : p;
+    s_pos = p;
+  }
+  __syncthreads();
+  const int pos = s_pos;
   if (pos >= cv.capacity) {
     if (threadIdx.x == 0) atomicCAS(cv.status, 0, (int)OKQ_ERR_CAPACITY);
     return;
@@ -438,13 +452,6 @@ __global__ void __launch_bounds__(128) k_append(CacheView cv, int layer0, const 
     __syncthreads();
     quantize_value_window(vt + cv.v_slot(win * W) * D, D, Rset, cv.body(layer, b, h, win), sm);
   }
-}
-
-__global__ void k_advance(CacheView cv, int layer0, int layer_count) {
-  int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= layer_count * cv.batch) return;
-  int* p = cv.seq_len + (size_t)layer0 * cv.batch + idx;
-  if (*p < cv.capacity) *p += 1;
 }
 
 // ---------------------------------------------------------------- canonical <-> physical
@@ -629,10 +636,10 @@ okq_status okq_append(const okq_cache* cache, int32_t layer, int32_t layer_count
   if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(signs) || !aligned16(R)) return OKQ_ERR_ALIGNMENT;
   CacheView cv = make_view(cache);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // the kernel counts a sequence's blocks in the top byte of its seq_len entry while it runs
+  if (cache->capacity >= APPEND_ARRIVAL || cache->n_kv_heads > 127) return OKQ_ERR_UNSUPPORTED;
   k_append<<<dim3(cv.n_kv_heads, cv.batch, layer_count), 128, 0, s>>>(
       cv, layer, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new), modality_new, signs, R, n_R);
-  int n = layer_count * cv.batch;
-  k_advance<<<(n + 127) / 128, 128, 0, s>>>(cv, layer, layer_count);
   return launch_status();
 }
 
