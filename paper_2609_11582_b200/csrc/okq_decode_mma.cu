@@ -675,7 +675,10 @@ template <bool CAPTION, int SEQ>
 struct CombineSmem {
   static constexpr int CB_SEQ = SEQ, CB_ROWS = SEQ * GP;
   static constexpr int TAIL = CAPTION ? CAPTION_V_SLOTS : W;   // most raw-value tokens of a sequence
-  __align__(16) float Rbuf[CB_NBUF][CB_CHUNK][D];   // ring of 16-row slices of the rotation matrices
+  // ring of 16-row slices of the rotation matrices; with one sequence per block it is large enough for a quarter
+  // of the columns of all three matrices, which the four-slice configuration fetches whole at the start
+  static constexpr int RBUF_FLOATS = SEQ == 1 ? 3 * D * (D / 4) : CB_NBUF * CB_CHUNK * D;
+  __align__(16) float Rbuf[RBUF_FLOATS];
   __align__(16) float mrg[CB_SEQ][MRG_MAX][GP][4];                // per partial and head: rescale factor, weight sums of the modalities
   __align__(16) float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
   __align__(16) float rawv[CB_ROWS][D];       // raw-tail contribution, [row][channel]
@@ -723,6 +726,18 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   constexpr float DELTA_REL = (3.0f * CB_INNER - CB_OUTER) / (2.0f * (CB_OUTER - CB_INNER));
   const float S_COEF = -CB_OUTER + (CB_OUTER - CB_INNER) * (DELTA_REL - __half2float(__float2half_rn(DELTA_REL)));
 
+  // four column slices per (head, sequence): this block's 32 columns of the three matrices (48 KB) start their way
+  // into shared memory now and are used at the very end
+  constexpr bool PRELOAD = NS == 4;
+  static_assert(!PRELOAD || SEQ == 1, "the whole-slice preload needs the one-sequence buffer");
+  if (PRELOAD) {
+    const float* Rsl = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D + sl * (D / NS);
+    for (int i = threadIdx.x; i < 3 * D * (D / NS) / 4; i += SEQ * 128) {
+      const int row = i / (D / NS / 4), c4 = i % (D / NS / 4);
+      cp_async16(&sm.Rbuf[row * (D / NS) + 4 * c4], Rsl + (size_t)row * D + 4 * c4);
+    }
+    cp_async_commit();
+  }
   const int e = li * cv.batch + bb;
   const int seq = live ? cv.seq_len[layer * cv.batch + bb] : 0;
   // tokens [0, v_pk) have packed values (and keys): they are in the split-K partials; tokens [v_pk, seq) have raw
@@ -756,7 +771,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     __syncthreads();
   }
   // tail scores: thread -> (token = c & 31 of a 32-token chunk, heads (c >> 5) * 2 + {0, 1})
-  float* msf = &sm.Rbuf[0][0][0] + bs * 2 * D;   // (m, s) of a packed window as floats (the slice buffer is idle here)
+  float* msf = &sm.vec[0][0][0] + bs * 2 * D;   // (m, s) of a packed window as floats (the rotated sums are written later)
   for (int chunk = 0; chunk * W < n_tail; chunk++) {
     const int tok = chunk * W + (c & 31), t = v_pk + tok;
     float s2[2] = {-INFINITY, -INFINITY};
@@ -924,7 +939,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   const int rw = (threadIdx.x >> 5) * 4, cl = (threadIdx.x & 31) * CW;   // first row / column (inside the slice) of the tile
   const float* Rset = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D + sl * SW;
   constexpr int N_CHUNK = 3 * D / CB_CHUNK;
-  float* rbuf = &sm.Rbuf[0][0][0];    // ring of CB_NBUF slices of CB_CHUNK x SW floats
+  float* rbuf = &sm.Rbuf[0];          // ring of CB_NBUF slices of CB_CHUNK x SW floats (or, preloaded, all rows)
   auto stage = [&](int chunk) {   // rows [16*chunk, 16*chunk+16) of the three stacked matrices, this CTA's columns
     const float* src = Rset + (size_t)chunk * CB_CHUNK * D;
     float* dst = rbuf + (chunk % CB_NBUF) * CB_CHUNK * SW;
@@ -940,16 +955,22 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   for (int i = 0; i < 4; i++)
 #pragma unroll
     for (int k = 0; k < CW; k++) o[i][k] = 0.f;
-  if (!comp)
+  if (PRELOAD) {
+    cp_async_wait<0>();
+    __syncthreads();   // the matrices have landed and vec is complete
+  } else if (!comp) {
     for (int pre = 0; pre < CB_NBUF - 1; pre++) stage(pre);
+  }
   for (int chunk = 0; chunk < N_CHUNK; chunk++) {
-    if (!comp) cp_async_wait<CB_NBUF - 2>();
-    __syncthreads();   // slice `chunk` has landed; everyone is done with slice chunk-1 (and, first time, vec is complete)
+    if (!PRELOAD) {
+      if (!comp) cp_async_wait<CB_NBUF - 2>();
+      __syncthreads();   // slice `chunk` has landed; everyone is done with slice chunk-1 (and, first time, vec is complete)
+    }
     if (!comp) {
-      stage(chunk + CB_NBUF - 1);   // into the buffer of slice chunk-1
+      if (!PRELOAD) stage(chunk + CB_NBUF - 1);   // into the buffer of slice chunk-1
     } else {
       const int m = chunk / (D / CB_CHUNK), r0 = (chunk % (D / CB_CHUNK)) * CB_CHUNK;
-      const float* rb = rbuf + (chunk % CB_NBUF) * CB_CHUNK * SW;
+      const float* rb = rbuf + (PRELOAD ? chunk : chunk % CB_NBUF) * CB_CHUNK * SW;
 #pragma unroll 2
       for (int r = 0; r < CB_CHUNK; r += 4) {
         float4 x[4];
