@@ -726,18 +726,6 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   constexpr float DELTA_REL = (3.0f * CB_INNER - CB_OUTER) / (2.0f * (CB_OUTER - CB_INNER));
   const float S_COEF = -CB_OUTER + (CB_OUTER - CB_INNER) * (DELTA_REL - __half2float(__float2half_rn(DELTA_REL)));
 
-  // four column slices per (head, sequence): this block's 32 columns of the three matrices (48 KB) start their way
-  // into shared memory now and are used at the very end
-  constexpr bool PRELOAD = NS == 4;
-  static_assert(!PRELOAD || SEQ == 1, "the whole-slice preload needs the one-sequence buffer");
-  if (PRELOAD) {
-    const float* Rsl = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D + sl * (D / NS);
-    for (int i = threadIdx.x; i < 3 * D * (D / NS) / 4; i += SEQ * 128) {
-      const int row = i / (D / NS / 4), c4 = i % (D / NS / 4);
-      cp_async16(&sm.Rbuf[row * (D / NS) + 4 * c4], Rsl + (size_t)row * D + 4 * c4);
-    }
-    cp_async_commit();
-  }
   const int e = li * cv.batch + bb;
   const int seq = live ? cv.seq_len[layer * cv.batch + bb] : 0;
   // tokens [0, v_pk) have packed values (and keys): they are in the split-K partials; tokens [v_pk, seq) have raw
@@ -771,7 +759,16 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     __syncthreads();
   }
   // tail scores: thread -> (token = c & 31 of a 32-token chunk, heads (c >> 5) * 2 + {0, 1})
-  float* msf = &sm.vec[0][0][0] + bs * 2 * D;   // (m, s) of a packed window as floats (the rotated sums are written later)
+  // Scratch inside the rotated-sum array (written much later): per sequence the (m, s) of a packed window as
+  // floats, then the chunk's raw key rows (272-byte rows: 16-byte reads of 32 different rows hit different banks)
+  // and the group's query rows, both fetched with cp.async so that all their loads are in flight together.
+  constexpr int KROW = D + 8;                              // halfs per staged key row
+  constexpr int KSM_FLOATS = W * KROW / 2, QSM_FLOATS = GP * D / 2;
+  static_assert(CB_SEQ * (2 * D + KSM_FLOATS + QSM_FLOATS) <= 3 * CB_ROWS * D, "tail scratch must fit the rotated-sum array");
+  float* msf = &sm.vec[0][0][0] + bs * 2 * D;
+  __half* ksm = reinterpret_cast<__half*>(&sm.vec[0][0][0] + CB_SEQ * 2 * D + bs * (KSM_FLOATS + QSM_FLOATS));
+  __half* qsm = ksm + W * KROW;
+  if (n_tail > 0 && c < G * (D / 8)) cp_async16(qsm + 8 * c, qbase + 8 * c);
   for (int chunk = 0; chunk * W < n_tail; chunk++) {
     const int tok = chunk * W + (c & 31), t = v_pk + tok;
     float s2[2] = {-INFINITY, -INFINITY};
@@ -781,19 +778,28 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     if (packed) {
       const float2 ms = window_meta_pos(cv.meta(layer, bb, h, (v_pk + chunk * W) / W), cv.fmt, c);
       msf[c] = ms.x; msf[D + c] = ms.y;
-      asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // the sequence's 128 threads
+    } else {
+      for (int idx = c; idx < W * (D / 8); idx += 128) {
+        const int r = idx / (D / 8), c8 = idx % (D / 8);
+        if (chunk * W + r < n_tail)
+          cp_async16(ksm + r * KROW + 8 * c8, kt + cv.k_slot(v_pk + chunk * W + r) * D + 8 * c8);
+      }
     }
+    cp_async_commit();
+    cp_async_wait<0>();
+    asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // the sequence's 128 threads
     if (tok < n_tail && j0 < G) {
       float a2[2] = {0.f, 0.f};
-      if (!CAPTION || t >= k_pk) {   // raw key
-        const __half* krow = kt + cv.k_slot(t) * D;
+      if (!packed) {   // raw key
+        const __half* krow = ksm + (c & 31) * KROW;
+#pragma unroll 4
         for (int k = 0; k < D; k += 8) {
           const uint4 kv = *reinterpret_cast<const uint4*>(krow + k);
           const __half2* k2 = reinterpret_cast<const __half2*>(&kv);
 #pragma unroll
           for (int hh = 0; hh < 2; hh++) {
             if (j0 + hh >= G) continue;
-            const uint4 qv = *reinterpret_cast<const uint4*>(qbase + (j0 + hh) * D + k);
+            const uint4 qv = *reinterpret_cast<const uint4*>(qsm + (j0 + hh) * D + k);
             const __half2* q2 = reinterpret_cast<const __half2*>(&qv);
 #pragma unroll
             for (int u = 0; u < 4; u++) {
@@ -831,7 +837,21 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
       if (j0 + 1 < G) s2[1] = a2[1] * P.sm_scale * LOG2E;
     }
     if (tok < sm.TAIL) { sm.tsc[bs][tok][j0] = s2[0]; sm.tsc[bs][tok][j0 + 1] = s2[1]; }
-    if (packed) asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // before the next window's (m, s)
+    if ((chunk + 1) * W < n_tail)
+      asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // before the next chunk's rows or (m, s) land
+  }
+  // four column slices per (head, sequence): this block's 32 columns of the three matrices (48 KB) start their way
+  // into shared memory now (behind the tail's own cp.async groups, which had to be waited for) and are used at the
+  // very end, after the merge
+  constexpr bool PRELOAD = NS == 4;
+  static_assert(!PRELOAD || SEQ == 1, "the whole-slice preload needs the one-sequence buffer");
+  if (PRELOAD) {
+    const float* Rsl = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D + sl * (D / NS);
+    for (int i = threadIdx.x; i < 3 * D * (D / NS) / 4; i += SEQ * 128) {
+      const int row = i / (D / NS / 4), c4 = i % (D / NS / 4);
+      cp_async16(&sm.Rbuf[row * (D / NS) + 4 * c4], Rsl + (size_t)row * D + 4 * c4);
+    }
+    cp_async_commit();
   }
   __syncthreads();
   if (c < GP) {
