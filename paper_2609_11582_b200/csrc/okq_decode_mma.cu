@@ -661,6 +661,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
   }
 }
 
+constexpr int PARTIAL_HDR_FLOATS = 2 * GP + 3 * 32;   // m[GP], l[GP], Sp[3][32] at the start of a PartialF
 constexpr int CB_SEQ_MAX = 4;             // most sequences per combine CTA (one 128-thread group each)
 
 constexpr int MRG_MAX = 8;                // partials per (sequence, head) whose factors are precomputed
@@ -687,6 +688,8 @@ struct CombineSmem {
   __align__(16) float qrot[2][CAPTION ? CB_ROWS : 1][D];
   __align__(16) float tsc[CB_SEQ][TAIL][GP];  // tail scores (log2 domain), then softmax numerators
   float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
+  // one-sequence blocks: the headers (m, l, weight sums) of the sequence's first MRG_MAX partials, fetched early
+  __align__(16) float hdr[SEQ == 1 ? MRG_MAX * PARTIAL_HDR_FLOATS : 4];
   int prefix[MAX_ENTRIES + 1];
 };
 
@@ -716,6 +719,35 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   const int bb = live ? b : 0;
   const int G = P.group, Hkv = cv.n_kv_heads;
   const int n_entries = P.layer_count * cv.batch;
+  const int seq = live ? cv.seq_len[layer * cv.batch + bb] : 0;
+  // tokens [0, v_pk) have packed values (and keys): they are in the split-K partials; tokens [v_pk, seq) have raw
+  // values; of those, [v_pk, k_pk) have packed keys (captioning schedule only), the rest raw keys
+  const int v_pk = cv.v_packed(seq), k_pk = cv.k_packed(seq);
+  const int nwin = v_pk / W, n_tail = seq - v_pk;
+  const __half* qbase = P.q + (((size_t)li * cv.batch + bb) * cv.n_q_heads + h * G) * D;
+  const __half* kt = cv.k_tail + cv.k_tail_off(layer, bb, h);
+  const __half* vt = cv.v_tail + cv.v_tail_off(layer, bb, h);
+  // Scratch inside the rotated-sum array (written much later): per sequence the (m, s) of a packed window as
+  // floats, then the chunk's raw key rows (272-byte rows: 16-byte reads of 32 different rows hit different banks)
+  // and the group's query rows, both fetched with cp.async so that all their loads are in flight together.
+  constexpr int KROW = D + 8;                              // halfs per staged key row
+  constexpr int KSM_FLOATS = W * KROW / 2, QSM_FLOATS = GP * D / 2;
+  static_assert(CB_SEQ * (2 * D + KSM_FLOATS + QSM_FLOATS) <= 3 * CB_ROWS * D, "tail scratch must fit the rotated-sum array");
+  float* msf = &sm.vec[0][0][0] + bs * 2 * D;
+  __half* ksm = reinterpret_cast<__half*>(&sm.vec[0][0][0] + CB_SEQ * 2 * D + bs * (KSM_FLOATS + QSM_FLOATS));
+  __half* qsm = ksm + W * KROW;
+  // a chunk of the tail is one 32-token window: its keys are either all packed or all raw
+  auto stage_tail = [&](int chunk) {
+    if (chunk == 0 && c < G * (D / 8)) cp_async16(qsm + 8 * c, qbase + 8 * c);
+    if (!(CAPTION && v_pk + chunk * W < k_pk))
+      for (int idx = c; idx < W * (D / 8); idx += 128) {
+        const int r = idx / (D / 8), c8 = idx % (D / 8);
+        if (chunk * W + r < n_tail)
+          cp_async16(ksm + r * KROW + 8 * c8, kt + cv.k_slot(v_pk + chunk * W + r) * D + 8 * c8);
+      }
+    cp_async_commit();
+  };
+  if (n_tail > 0) stage_tail(0);   // on its way while the prefix is computed
   const int total = block_prefix(cv, P.layer0, n_entries, sm.prefix);
   const int per = total > 0 ? (total + n_cta - 1) / n_cta : 1;
   constexpr float ACC_SCALE = (CB_OUTER - CB_INNER) * 262144.0f;  // (b - a) * 2^18
@@ -727,17 +759,18 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   const float S_COEF = -CB_OUTER + (CB_OUTER - CB_INNER) * (DELTA_REL - __half2float(__float2half_rn(DELTA_REL)));
 
   const int e = li * cv.batch + bb;
-  const int seq = live ? cv.seq_len[layer * cv.batch + bb] : 0;
-  // tokens [0, v_pk) have packed values (and keys): they are in the split-K partials; tokens [v_pk, seq) have raw
-  // values; of those, [v_pk, k_pk) have packed keys (captioning schedule only), the rest raw keys
-  const int v_pk = cv.v_packed(seq), k_pk = cv.k_packed(seq);
-  const int nwin = v_pk / W, n_tail = seq - v_pk;
   const int unit = e * Hkv + h;
   const int start = sm.prefix[e] + h * nwin, end = start + nwin;
   const int cta_lo = nwin > 0 ? start / per : 0, cta_hi = nwin > 0 ? (end - 1) / per : -1;
-  const __half* qbase = P.q + (((size_t)li * cv.batch + bb) * cv.n_q_heads + h * G) * D;
-  const __half* kt = cv.k_tail + cv.k_tail_off(layer, bb, h);
-  const __half* vt = cv.v_tail + cv.v_tail_off(layer, bb, h);
+  const int n_hdr = SEQ == 1 ? max(0, min(cta_hi - cta_lo + 1, MRG_MAX)) : 0;   // partials whose headers are staged
+  if (SEQ == 1) {
+    for (int idx = c; idx < n_hdr * (PARTIAL_HDR_FLOATS / 4); idx += 128) {
+      const int ci = idx / (PARTIAL_HDR_FLOATS / 4), q4 = idx % (PARTIAL_HDR_FLOATS / 4);
+      cp_async16(&sm.hdr[ci * PARTIAL_HDR_FLOATS + 4 * q4],
+                 reinterpret_cast<const float*>(&P.partials_f[(size_t)unit + cta_lo + ci]) + 4 * q4);
+    }
+    cp_async_commit();
+  }
   if (CAPTION) {   // q' = H q for the scores of packed keys: one warp per (sequence, head) row
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int row = warp; row < CB_ROWS; row += CB_SEQ * 4) {
@@ -759,33 +792,16 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     __syncthreads();
   }
   // tail scores: thread -> (token = c & 31 of a 32-token chunk, heads (c >> 5) * 2 + {0, 1})
-  // Scratch inside the rotated-sum array (written much later): per sequence the (m, s) of a packed window as
-  // floats, then the chunk's raw key rows (272-byte rows: 16-byte reads of 32 different rows hit different banks)
-  // and the group's query rows, both fetched with cp.async so that all their loads are in flight together.
-  constexpr int KROW = D + 8;                              // halfs per staged key row
-  constexpr int KSM_FLOATS = W * KROW / 2, QSM_FLOATS = GP * D / 2;
-  static_assert(CB_SEQ * (2 * D + KSM_FLOATS + QSM_FLOATS) <= 3 * CB_ROWS * D, "tail scratch must fit the rotated-sum array");
-  float* msf = &sm.vec[0][0][0] + bs * 2 * D;
-  __half* ksm = reinterpret_cast<__half*>(&sm.vec[0][0][0] + CB_SEQ * 2 * D + bs * (KSM_FLOATS + QSM_FLOATS));
-  __half* qsm = ksm + W * KROW;
-  if (n_tail > 0 && c < G * (D / 8)) cp_async16(qsm + 8 * c, qbase + 8 * c);
   for (int chunk = 0; chunk * W < n_tail; chunk++) {
     const int tok = chunk * W + (c & 31), t = v_pk + tok;
     float s2[2] = {-INFINITY, -INFINITY};
     const int j0 = (c >> 5) * 2;
-    // a chunk is one 32-token window: its keys are either all packed or all raw
     const bool packed = CAPTION && v_pk + chunk * W < k_pk;
     if (packed) {
       const float2 ms = window_meta_pos(cv.meta(layer, bb, h, (v_pk + chunk * W) / W), cv.fmt, c);
       msf[c] = ms.x; msf[D + c] = ms.y;
-    } else {
-      for (int idx = c; idx < W * (D / 8); idx += 128) {
-        const int r = idx / (D / 8), c8 = idx % (D / 8);
-        if (chunk * W + r < n_tail)
-          cp_async16(ksm + r * KROW + 8 * c8, kt + cv.k_slot(v_pk + chunk * W + r) * D + 8 * c8);
-      }
     }
-    cp_async_commit();
+    if (chunk > 0) stage_tail(chunk);
     cp_async_wait<0>();
     asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // the sequence's 128 threads
     if (tok < n_tail && j0 < G) {
@@ -853,13 +869,21 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     }
     cp_async_commit();
   }
+  // the staged headers must have landed (a sequence without tail tokens has not waited yet); the matrix preload,
+  // the newest group, may stay in flight
+  if (SEQ == 1) { if (PRELOAD) cp_async_wait<1>(); else cp_async_wait<0>(); }
   __syncthreads();
   if (c < GP) {
     float M = -INFINITY;
-    for (int ct = cta_lo; ct <= cta_hi; ct++) M = fmaxf(M, P.partials_f[(size_t)unit + ct].m[c]);
+    for (int ci = 0; ci < n_hdr; ci++) M = fmaxf(M, sm.hdr[ci * PARTIAL_HDR_FLOATS + c]);
+    for (int ct = cta_lo + n_hdr; ct <= cta_hi; ct++) M = fmaxf(M, P.partials_f[(size_t)unit + ct].m[c]);
     for (int i = 0; i < n_tail; i++) M = fmaxf(M, sm.tsc[bs][i][c]);
     float L = 0.f;
-    for (int ct = cta_lo; ct <= cta_hi; ct++) {
+    for (int ci = 0; ci < n_hdr; ci++) {
+      const float pm = sm.hdr[ci * PARTIAL_HDR_FLOATS + c];
+      if (pm != -INFINITY) L += sm.hdr[ci * PARTIAL_HDR_FLOATS + GP + c] * exp2f(pm - M);
+    }
+    for (int ct = cta_lo + n_hdr; ct <= cta_hi; ct++) {
       const PartialF& pp = P.partials_f[(size_t)unit + ct];
       if (pp.m[c] != -INFINITY) L += pp.l[c] * exp2f(pp.m[c] - M);
     }
