@@ -976,11 +976,14 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   // out[row][c] = raw[row][c] + sum_m sum_r R_m[r][c] * vec[m][row][r].  The first half of the threads compute
   // a 4-row x 4-column tile each; the second half stream the matrices through shared memory in 16-row
   // slices, three slices ahead.
-  const bool comp = threadIdx.x < CB_SEQ * 64;
+  // (with the matrices preloaded there is nothing to stream: both halves compute, each every other 16-row slice)
+  constexpr bool PRE = NS == 4;
+  const int khalf = PRE ? threadIdx.x / (CB_SEQ * 64) : 0;
+  const bool comp = PRE || threadIdx.x < CB_SEQ * 64;
   constexpr int CW = 4 / NS;          // output columns per compute thread
   constexpr int SW = D / NS;          // output columns of this CTA = floats per staged matrix row
   static_assert(NS == 1 || NS == 4, "column slices");
-  const int rw = (threadIdx.x >> 5) * 4, cl = (threadIdx.x & 31) * CW;   // first row / column (inside the slice) of the tile
+  const int rw = ((threadIdx.x % (CB_SEQ * 64)) >> 5) * 4, cl = (threadIdx.x & 31) * CW;   // first row / column (inside the slice) of the tile
   const float* Rset = P.R + ((size_t)li * P.n_R + (P.n_R == 1 ? 0 : h)) * 3 * D * D + sl * SW;
   constexpr int N_CHUNK = 3 * D / CB_CHUNK;
   float* rbuf = &sm.Rbuf[0];          // ring of CB_NBUF slices of CB_CHUNK x SW floats (or, preloaded, all rows)
@@ -1012,7 +1015,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     }
     if (!comp) {
       if (!PRELOAD) stage(chunk + CB_NBUF - 1);   // into the buffer of slice chunk-1
-    } else {
+    } else if (!PRE || (chunk & 1) == khalf) {
       const int m = chunk / (D / CB_CHUNK), r0 = (chunk % (D / CB_CHUNK)) * CB_CHUNK;
       const float* rb = rbuf + (PRELOAD ? chunk : chunk % CB_NBUF) * CB_CHUNK * SW;
 #pragma unroll 2
@@ -1044,7 +1047,24 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
       }
     }
   }
-  if (comp) {
+  if (PRE) {   // the second half's sums reach the first through the tail-score array, idle by now
+    float* red = &sm.tsc[0][0][0] + (threadIdx.x % (CB_SEQ * 64)) * 4 * CW;
+    static_assert(!PRE || CB_SEQ * 64 * 4 * CW <= CB_SEQ * W * GP, "reduction scratch");
+    if (khalf) {
+#pragma unroll
+      for (int i = 0; i < 4; i++)
+#pragma unroll
+        for (int k = 0; k < CW; k++) red[i * CW + k] = o[i][k];
+    }
+    __syncthreads();
+    if (!khalf) {
+#pragma unroll
+      for (int i = 0; i < 4; i++)
+#pragma unroll
+        for (int k = 0; k < CW; k++) o[i][k] += red[i * CW + k];
+    }
+  }
+  if (comp && !khalf) {
 #pragma unroll
     for (int i = 0; i < 4; i++) {
       const int row = rw + i, ob = blockIdx.y * CB_SEQ + row / GP, j = row % GP;
