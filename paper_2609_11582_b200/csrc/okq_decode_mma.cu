@@ -690,6 +690,7 @@ struct CombineSmem {
   float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
   // one-sequence blocks: the headers (m, l, weight sums) of the sequence's first MRG_MAX partials, fetched early
   __align__(16) float hdr[SEQ == 1 ? MRG_MAX * PARTIAL_HDR_FLOATS : 4];
+  __align__(16) __half vsm[SEQ == 1 ? TAIL * D : 8];   // one-sequence blocks: the raw value rows, fetched early
   int prefix[MAX_ENTRIES + 1];
 };
 
@@ -747,6 +748,11 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
       }
     cp_async_commit();
   };
+  if (SEQ == 1)   // the raw value rows go the same way (used after the softmax numerators are known)
+    for (int idx = c; idx < n_tail * (D / 8); idx += 128) {
+      const int r = idx / (D / 8), c8 = idx % (D / 8);
+      cp_async16(&sm.vsm[r * D + 8 * c8], vt + cv.v_slot(v_pk + r) * D + 8 * c8);
+    }
   if (n_tail > 0) stage_tail(0);   // on its way while the prefix is computed
   const int total = block_prefix(cv, P.layer0, n_entries, sm.prefix);
   const int per = total > 0 ? (total + n_cta - 1) / n_cta : 1;
@@ -918,7 +924,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   for (int j = 0; j < GP; j++) araw[j] = 0.f;
 #pragma unroll 8
   for (int i = 0; i < n_tail; i++) {
-    const float x = __half2float(vt[cv.v_slot(v_pk + i) * D + c]);
+    const float x = __half2float(SEQ == 1 ? sm.vsm[i * D + c] : vt[cv.v_slot(v_pk + i) * D + c]);
     const float4 w0 = *reinterpret_cast<const float4*>(&sm.tsc[bs][i][0]);
     const float4 w1 = *reinterpret_cast<const float4*>(&sm.tsc[bs][i][4]);
     araw[0] = fmaf(w0.x, x, araw[0]); araw[1] = fmaf(w0.y, x, araw[1]);
