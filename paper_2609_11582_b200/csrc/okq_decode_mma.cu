@@ -60,14 +60,17 @@ struct MmaSmem {
   __align__(16) Handoff hand[NPAIR][2];
   __align__(16) float spill[NPAIR][3][32][SPILL_STRIDE];   // [pair][modality][lane]: the lane's 33 sums, 128-bit rows
   float spill_m[NPAIR][3][GP];
+  float fin_w[NPAIR][2][GP];   // running maximum and weight sum a pair's score warp ended its last range with
   int prefix[MAX_ENTRIES + 1];
 };
 
 constexpr int MB_SEG = 32;                      // (sequence, head) units merged per batch at the end of the launch
 struct MergeSmem {
   int pa[MB_SEG], pb[MB_SEG];                   // first and last warp pair that worked on the unit (pb < pa: none)
+  int last_kept[MB_SEG];                        // whether pair pb's piece is in shared memory (all before it are)
   float meta[MB_SEG + NPAIR][5 * GP];           // per piece: sm[3][GP], wm[GP], wl[GP]; index = unit + pair - pa[0]
   float M[MB_SEG][GP];                          // merged running maximum
+  float fac[MB_SEG + NPAIR][3][GP];             // per piece, modality and head: exp2(sm - M), 0 where the piece holds nothing
 };
 
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -125,7 +128,8 @@ struct Segment {
   int w0, n_my;                // this pair's windows of that (layer, sequence, head): first window, count
   const __half* q;             // query rows of the KV head's group: [group][128]
   const float* signs;          // Hadamard signs of the layer
-  PairPartial* piece;          // where the pair leaves what it accumulated
+  PairPartial* piece;          // where the pair leaves what it accumulated ...
+  bool keep;                   // ... unless this is the last unit of the pair's range: then it stays in shared memory
 };
 
 // The group's rotated queries q' = H D q / sqrt(128) as mma A-fragment registers, computed by one warp in
@@ -334,7 +338,10 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
   cp_async_wait<0>();
   run_l += __shfl_xor_sync(0xffffffffu, run_l, 1);
   run_l += __shfl_xor_sync(0xffffffffu, run_l, 2);
-  if (t == 0) { sg.piece->wm[g] = run_m; sg.piece->wl[g] = run_l; }
+  if (t == 0) {
+    if (sg.keep) { sm.fin_w[pair][0][g] = run_m; sm.fin_w[pair][1][g] = run_l; }
+    else { sg.piece->wm[g] = run_m; sg.piece->wl[g] = run_l; }
+  }
 }
 
 // ---------------------------------------------------------------- value warp
@@ -477,6 +484,7 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
     pair_barrier(pair);
   }
   // leave the three modalities' accumulators (each lane its own column) and their maxima in the pair's piece
+  if (sg.keep) return;   // the block's merge reads this pair's sums where they are
 #pragma unroll 1
   for (int m = 0; m < 3; m++) {
     const float mm = sm.spill_m[pair][m][g];
@@ -552,6 +560,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
       sg.q = P.q + (((size_t)li * cv.batch + b) * cv.n_q_heads + (size_t)wh.h * G) * D;
       sg.signs = P.signs + (size_t)li * D;
       sg.piece = P.pair_parts + (size_t)(wh.e * Hkv + wh.h) + ((size_t)blockIdx.x * NPAIR + pair);
+      sg.keep = pos + sg.n_my == pos_end;
       if (is_score) score_warp<FMT>(sm, sg, G, P.sm_scale, pair, lane);
       else value_warp<FMT>(sm, sg, pair, lane);
       pos += sg.n_my;
@@ -574,17 +583,26 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
       const int nwin = (sm.prefix[e + 1] - sm.prefix[e]) / Hkv;
       const int a0 = max(pos0, sm.prefix[e] + h * nwin), a1 = min(pos1, sm.prefix[e] + (h + 1) * nwin);
       mg.pa[tid] = a1 > a0 ? (a0 - pos0) / cnt : 0;
-      mg.pb[tid] = a1 > a0 ? (a1 - 1 - pos0) / cnt : -1;   // empty: a (sequence, head) with no packed window
+      const int pb = a1 > a0 ? (a1 - 1 - pos0) / cnt : -1;   // empty: a (sequence, head) with no packed window
+      mg.pb[tid] = pb;
+      // pairs before the last end their range inside this unit, so their sums are still in shared memory; the
+      // last one's are too unless its range goes on into the next unit
+      mg.last_kept[tid] = pb >= 0 && min(pos1, pos0 + (pb + 1) * cnt) <= a1;
     }
     __syncthreads();
     // (b) the pieces' maxima and weight sums: one warp per (unit, pair)
     for (int j = warp; j < n_u * NPAIR; j += NTHREADS / 32) {
       const int su = j / NPAIR, p = j % NPAIR;
       if (p < mg.pa[su] || p > mg.pb[su]) continue;
-      const PairPartial& pp = P.pair_parts[(size_t)(ub + su) + (size_t)blockIdx.x * NPAIR + p];
       float* dst = mg.meta[su + p - mg.pa[0]];
-      dst[lane] = (&pp.sm[0][0])[lane];                         // sm[3][GP], then wm[GP]
-      if (lane < GP) dst[32 + lane] = pp.wl[lane];
+      if (p < mg.pb[su] || mg.last_kept[su]) {
+        dst[lane] = lane < 3 * GP ? (&sm.spill_m[p][0][0])[lane] : sm.fin_w[p][0][lane - 3 * GP];
+        if (lane < GP) dst[32 + lane] = sm.fin_w[p][1][lane];
+      } else {
+        const PairPartial& pp = P.pair_parts[(size_t)(ub + su) + (size_t)blockIdx.x * NPAIR + p];
+        dst[lane] = (&pp.sm[0][0])[lane];                         // sm[3][GP], then wm[GP]
+        if (lane < GP) dst[32 + lane] = pp.wl[lane];
+      }
     }
     __syncthreads();
     // (c) merged maximum and weight sum per (unit, head)
@@ -605,56 +623,49 @@ __global__ void __launch_bounds__(NTHREADS, 1) k_decode_mma(DecodeParams P) {
     }
     __syncthreads();
     // (d) the accumulators: one item = four lanes' worth of one (unit, modality, register) row
-    constexpr int ROW_ITEMS = 3 * SPILL_REGS * 8, MU = 4, MP = 3;
-    for (int base = tid; base < n_u * ROW_ITEMS; base += MU * NTHREADS) {
-      float4 x[MU][MP];
+    // rescale factors, once per (piece, modality, head)
+    for (int j = tid; j < n_u * NPAIR * 3 * GP; j += NTHREADS) {
+      const int su = j / (NPAIR * 3 * GP), p = (j / (3 * GP)) % NPAIR, k = j % (3 * GP);
+      if (p < mg.pa[su] || p > mg.pb[su]) continue;
+      const float smv = mg.meta[su + p - mg.pa[0]][k];
+      (&mg.fac[su + p - mg.pa[0]][0][0])[k] = smv == -INFINITY ? 0.f : exp2f(smv - mg.M[su][k % GP]);
+    }
+    __syncthreads();
+    // (d) the accumulators: one item = four consecutive registers of one lane of one (unit, modality), or that
+    // lane's weight sum.  A lane's registers are one 128-bit row read where the piece is still in shared memory;
+    // registers r and r + 2 belong to head 2 (lane & 3), r + 1 and r + 3 to the next head.
+    constexpr int RG = 9, UNIT_ITEMS = 3 * RG * 32;
+    for (int it = tid; it < n_u * UNIT_ITEMS; it += NTHREADS) {
+      const int su = it / UNIT_ITEMS, idx = it % UNIT_ITEMS;
+      const int L = idx & 31, rg = (idx >> 5) % RG, m = idx / (RG * 32);
+      const int pa = mg.pa[su], np = mg.pb[su] - pa + 1;
+      if (np <= 0) continue;
+      const int inc0 = su + pa - mg.pa[0];
+      const bool last_kept = mg.last_kept[su] != 0;
+      const int hsel = rg < 8 ? 2 * (L & 3) : (L >> 2);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int u4 = 0; u4 < MU; u4++) {
-        const int it = base + u4 * NTHREADS;
-#pragma unroll
-        for (int q = 0; q < MP; q++) x[u4][q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (it < n_u * ROW_ITEMS) {
-          const int su = it / ROW_ITEMS, idx = it % ROW_ITEMS;
-          const int l4 = (idx & 7) * 4, r = (idx >> 3) % SPILL_REGS, m = idx / (SPILL_REGS * 8);
-#pragma unroll
-          for (int q = 0; q < MP; q++) {
-            const int p = mg.pa[su] + q;
-            if (p <= mg.pb[su] && mg.meta[su + p - mg.pa[0]][m * GP] != -INFINITY)   // else: no token of this modality
-              x[u4][q] = *reinterpret_cast<const float4*>(
-                  &P.pair_parts[(size_t)(ub + su) + (size_t)blockIdx.x * NPAIR + p].frag[m][r][l4]);
-          }
+      for (int q = 0; q < NPAIR; q++) {
+        if (q >= np || mg.meta[inc0 + q][m * GP] == -INFINITY) continue;   // no such pair / no token of this modality
+        const float* fc = mg.fac[inc0 + q][m];
+        const float fe = fc[hsel], fo = rg < 8 ? fc[hsel + 1] : fe;
+        float4 x;
+        if (q < np - 1 || last_kept) {
+          const float* sp = &sm.spill[pa + q][m][L][0];
+          x = rg < 8 ? *reinterpret_cast<const float4*>(sp + 4 * rg) : make_float4(sp[32], 0.f, 0.f, 0.f);
+        } else {
+          const float* gp = &P.pair_parts[(size_t)(ub + su) + (size_t)blockIdx.x * NPAIR + pa + q].frag[m][0][L];
+          x = rg < 8 ? make_float4(gp[(4 * rg) * 32], gp[(4 * rg + 1) * 32], gp[(4 * rg + 2) * 32], gp[(4 * rg + 3) * 32])
+                     : make_float4(gp[32 * 32], 0.f, 0.f, 0.f);
         }
+        v.x = fmaf(x.x, fe, v.x); v.y = fmaf(x.y, fo, v.y); v.z = fmaf(x.z, fe, v.z); v.w = fmaf(x.w, fo, v.w);
       }
-#pragma unroll
-      for (int u4 = 0; u4 < MU; u4++) {
-        const int it = base + u4 * NTHREADS;
-        if (it >= n_u * ROW_ITEMS) continue;
-        const int su = it / ROW_ITEMS, idx = it % ROW_ITEMS;
-        if (mg.pb[su] < mg.pa[su]) continue;
-        const int l4 = (idx & 7) * 4, r = (idx >> 3) % SPILL_REGS, m = idx / (SPILL_REGS * 8);
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int p = mg.pa[su]; p <= mg.pb[su]; p++) {
-          const float* me = mg.meta[su + p - mg.pa[0]] + m * GP;
-          if (me[0] == -INFINITY) continue;
-          const int q = p - mg.pa[su];
-          float4 xx;
-          if (q < MP) {
-            xx = q == 0 ? x[u4][0] : (q == 1 ? x[u4][1] : x[u4][2]);
-          } else {   // more than MP pairs on one unit: short slices
-            xx = *reinterpret_cast<const float4*>(
-                &P.pair_parts[(size_t)(ub + su) + (size_t)blockIdx.x * NPAIR + p].frag[m][r][l4]);
-          }
-          float f[4];
-#pragma unroll
-          for (int i = 0; i < 4; i++) {
-            const int head = r < 32 ? 2 * i + (r & 1) : (l4 >> 2);   // lane l4 + i holds heads 2 (lane & 3) + (r & 1)
-            f[i] = exp2f(me[head] - mg.M[su][head]);
-          }
-          v.x = fmaf(xx.x, f[0], v.x); v.y = fmaf(xx.y, f[1], v.y); v.z = fmaf(xx.z, f[2], v.z); v.w = fmaf(xx.w, f[3], v.w);
-        }
-        PartialF* out = P.partials_f + (size_t)(ub + su) + blockIdx.x;
-        if (r < 32) *reinterpret_cast<float4*>(&out->frag[m][r][l4]) = v;
-        else *reinterpret_cast<float4*>(&out->Sp[m][l4]) = v;
+      PartialF* out = P.partials_f + (size_t)(ub + su) + blockIdx.x;
+      if (rg < 8) {
+        out->frag[m][4 * rg][L] = v.x; out->frag[m][4 * rg + 1][L] = v.y;
+        out->frag[m][4 * rg + 2][L] = v.z; out->frag[m][4 * rg + 3][L] = v.w;
+      } else {
+        out->Sp[m][L] = v.x;
       }
     }
     __syncthreads();
