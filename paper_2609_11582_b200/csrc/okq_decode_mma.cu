@@ -44,7 +44,6 @@ template <int FMT> constexpr int stage_bytes() { return FMT == FMT_MXFP4 ? STAGE
 constexpr float RESCALE_LOG2 = 3.0f;            // numerators stay below 2^3 * 2^6 * vnorm in fp16
 constexpr int FLUSH = 32;                       // windows a value warp accumulates in registers at most
 constexpr int SPILL_STRIDE = 36;                // floats per lane in the deposited sums: 33 used, 144-byte rows
-constexpr int SPILL_REGS = PAIR_REGS;           // 32 accumulator registers + the running weight sum
 
 struct Handoff {
   uint4 pb[32];         // per lane: numerators p * vnorm * 2^6 / 4^nu of its 8 tokens, fp16 pairs (nu = x,y,z,w)
@@ -691,7 +690,10 @@ struct CombineSmem {
   // of the columns of all three matrices, which the four-slice configuration fetches whole at the start
   static constexpr int RBUF_FLOATS = SEQ == 1 ? 3 * D * (D / 4) : CB_NBUF * CB_CHUNK * D;
   __align__(16) float Rbuf[RBUF_FLOATS];
-  __align__(16) float mrg[CB_SEQ][MRG_MAX][GP][4];                // per partial and head: rescale factor, weight sums of the modalities
+  // per partial and head: rescale factor, weight sums of the modalities (one-sequence blocks have room for the
+  // partials of a long single sequence, which is spread over many CTAs of the split-K kernel)
+  static constexpr int MRG_TAB = SEQ == 1 ? 64 : MRG_MAX;
+  __align__(16) float mrg[CB_SEQ][MRG_TAB][GP][4];
   __align__(16) float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
   __align__(16) float rawv[CB_ROWS][D];       // raw-tail contribution, [row][channel]
   // q' = H q in the order of the (m, s) planes, for the scores of packed keys: [0] multiplies s * code, [1] the
@@ -911,16 +913,21 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   __syncthreads();
   // per partial and head: the rescale factor exp2(m - M) and the weight sums S_m (the four lanes of a quad hold
   // partial sums), so that the merge below only reads accumulator fragments
-  for (int idx = c; idx < min(cta_hi - cta_lo + 1, MRG_MAX) * GP; idx += 128) {
+  for (int idx = c; idx < min(cta_hi - cta_lo + 1, sm.MRG_TAB) * GP; idx += 128) {
     const int ci = idx / GP, j = idx % GP;
-    const PartialF& pp = P.partials_f[(size_t)unit + cta_lo + ci];
-    const float pm = pp.m[j];
+    // the partial's header: staged in shared memory (one-sequence blocks, first MRG_MAX partials) or in global memory
+    const float* ph = ci < n_hdr ? &sm.hdr[ci * PARTIAL_HDR_FLOATS]
+                                 : reinterpret_cast<const float*>(&P.partials_f[(size_t)unit + cta_lo + ci]);
+    const float pm = ph[j];
     float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
     if (pm != -INFINITY) {
+      const float4 s0 = *reinterpret_cast<const float4*>(ph + 2 * GP + 4 * j);
+      const float4 s1 = *reinterpret_cast<const float4*>(ph + 2 * GP + 32 + 4 * j);
+      const float4 s2 = *reinterpret_cast<const float4*>(ph + 2 * GP + 64 + 4 * j);
       f.x = exp2f(pm - sm.Ms[bs][j]);
-      f.y = pp.Sp[0][4 * j] + pp.Sp[0][4 * j + 1] + pp.Sp[0][4 * j + 2] + pp.Sp[0][4 * j + 3];
-      f.z = pp.Sp[1][4 * j] + pp.Sp[1][4 * j + 1] + pp.Sp[1][4 * j + 2] + pp.Sp[1][4 * j + 3];
-      f.w = pp.Sp[2][4 * j] + pp.Sp[2][4 * j + 1] + pp.Sp[2][4 * j + 2] + pp.Sp[2][4 * j + 3];
+      f.y = s0.x + s0.y + s0.z + s0.w;
+      f.z = s1.x + s1.y + s1.z + s1.w;
+      f.w = s2.x + s2.y + s2.z + s2.w;
     }
     *reinterpret_cast<float4*>(sm.mrg[bs][ci][j]) = f;
   }
@@ -951,32 +958,44 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
 #pragma unroll
     for (int jj = 0; jj < 4; jj++) vacc[jj][0] = vacc[jj][1] = vacc[jj][2] = 0.f;
     if (jg < G) {
-      for (int ct = cta_lo; ct <= cta_hi; ct++) {
-        const PartialF& pp = P.partials_f[(size_t)unit + ct];
-        float fr[4][3];
+      // one-sequence blocks have registers to spare: the fragments of four partials are fetched together (a long
+      // single sequence has dozens of partials per head)
+      constexpr int MU4 = SEQ == 1 ? 4 : 1;
+      for (int ct0 = cta_lo; ct0 <= cta_hi; ct0 += MU4) {
+        float fr[MU4][4][3];
 #pragma unroll
-        for (int jj = 0; jj < 4; jj++) {
-          const int j = jg + jj;
-          const int r = 4 * (c >> 4) + 2 * ((c >> 3) & 1) + (j & 1), l32 = 4 * (c & 7) + (j >> 1);
+        for (int u = 0; u < MU4; u++) {
+          const PartialF& pp = P.partials_f[(size_t)unit + min(ct0 + u, cta_hi)];
 #pragma unroll
-          for (int m = 0; m < 3; m++) fr[jj][m] = pp.frag[m][r][l32];
+          for (int jj = 0; jj < 4; jj++) {
+            const int j = jg + jj;
+            const int r = 4 * (c >> 4) + 2 * ((c >> 3) & 1) + (j & 1), l32 = 4 * (c & 7) + (j >> 1);
+#pragma unroll
+            for (int m = 0; m < 3; m++) fr[u][jj][m] = pp.frag[m][r][l32];
+          }
         }
 #pragma unroll
-        for (int jj = 0; jj < 4; jj++) {
-          const int j = jg + jj;
-          float ef, S[3];
-          if (ct - cta_lo < MRG_MAX) {
-            const float4 f = *reinterpret_cast<const float4*>(sm.mrg[bs][ct - cta_lo][j]);
-            ef = f.x; S[0] = f.y; S[1] = f.z; S[2] = f.w;
-          } else {   // more partials than the table holds (few heads over many CTAs): compute in place
-            const float pm = pp.m[j];
-            ef = pm == -INFINITY ? 0.f : exp2f(pm - sm.Ms[bs][j]);
+        for (int u = 0; u < MU4; u++) {
+          const int ct = ct0 + u;
+          if (ct > cta_hi) continue;
+          const PartialF& pp = P.partials_f[(size_t)unit + ct];
 #pragma unroll
-            for (int m = 0; m < 3; m++) S[m] = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
-          }
-          if (j < G && ef != 0.f) {
+          for (int jj = 0; jj < 4; jj++) {
+            const int j = jg + jj;
+            float ef, S[3];
+            if (ct - cta_lo < sm.MRG_TAB) {
+              const float4 f = *reinterpret_cast<const float4*>(sm.mrg[bs][ct - cta_lo][j]);
+              ef = f.x; S[0] = f.y; S[1] = f.z; S[2] = f.w;
+            } else {   // more partials than the table holds (few heads over many CTAs): compute in place
+              const float pm = pp.m[j];
+              ef = pm == -INFINITY ? 0.f : exp2f(pm - sm.Ms[bs][j]);
 #pragma unroll
-            for (int m = 0; m < 3; m++) vacc[jj][m] = fmaf(fmaf(ACC_SCALE, fr[jj][m], S_COEF * S[m]), ef, vacc[jj][m]);
+              for (int m = 0; m < 3; m++) S[m] = pp.Sp[m][4 * j] + pp.Sp[m][4 * j + 1] + pp.Sp[m][4 * j + 2] + pp.Sp[m][4 * j + 3];
+            }
+            if (j < G && ef != 0.f) {
+#pragma unroll
+              for (int m = 0; m < 3; m++) vacc[jj][m] = fmaf(fmaf(ACC_SCALE, fr[u][jj][m], S_COEF * S[m]), ef, vacc[jj][m]);
+            }
           }
         }
       }
