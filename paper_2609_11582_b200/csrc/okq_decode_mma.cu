@@ -701,8 +701,8 @@ struct CombineSmem {
   __align__(16) float qrot[2][CAPTION ? CB_ROWS : 1][D];
   __align__(16) float tsc[CB_SEQ][TAIL][GP];  // tail scores (log2 domain), then softmax numerators
   float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
-  // one-sequence blocks: the headers (m, l, weight sums) of the sequence's first MRG_MAX partials, fetched early
-  __align__(16) float hdr[SEQ == 1 ? MRG_MAX * PARTIAL_HDR_FLOATS : 4];
+  // one-sequence blocks: the headers (m, l, weight sums) of the sequence's first MRG_TAB partials, fetched early
+  __align__(16) float hdr[SEQ == 1 ? MRG_TAB * PARTIAL_HDR_FLOATS : 4];
   __align__(16) __half vsm[SEQ == 1 ? TAIL * D : 8];   // one-sequence blocks: the raw value rows, fetched early
   int prefix[MAX_ENTRIES + 1];
 };
@@ -781,7 +781,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   const int unit = e * Hkv + h;
   const int start = sm.prefix[e] + h * nwin, end = start + nwin;
   const int cta_lo = nwin > 0 ? start / per : 0, cta_hi = nwin > 0 ? (end - 1) / per : -1;
-  const int n_hdr = SEQ == 1 ? max(0, min(cta_hi - cta_lo + 1, MRG_MAX)) : 0;   // partials whose headers are staged
+  const int n_hdr = SEQ == 1 ? max(0, min(cta_hi - cta_lo + 1, sm.MRG_TAB)) : 0;   // partials whose headers are staged
   if (SEQ == 1) {
     for (int idx = c; idx < n_hdr * (PARTIAL_HDR_FLOATS / 4); idx += 128) {
       const int ci = idx / (PARTIAL_HDR_FLOATS / 4), q4 = idx % (PARTIAL_HDR_FLOATS / 4);
@@ -915,7 +915,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   // partial sums), so that the merge below only reads accumulator fragments
   for (int idx = c; idx < min(cta_hi - cta_lo + 1, sm.MRG_TAB) * GP; idx += 128) {
     const int ci = idx / GP, j = idx % GP;
-    // the partial's header: staged in shared memory (one-sequence blocks, first MRG_MAX partials) or in global memory
+    // the partial's header: staged in shared memory (one-sequence blocks) or in global memory
     const float* ph = ci < n_hdr ? &sm.hdr[ci * PARTIAL_HDR_FLOATS]
                                  : reinterpret_cast<const float*>(&P.partials_f[(size_t)unit + cta_lo + ci]);
     const float pm = ph[j];
