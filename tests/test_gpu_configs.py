@@ -59,6 +59,16 @@ def test_one_modality_long_ranges():
         print("one modality, splits", splits, errs)
 
 
+def test_one_head_over_every_cta():
+    """A single (sequence, head) unit of 129 windows: every CTA of the split-K kernel holds one window of it, so the
+    combine kernel merges 129 partials for one head group, more than its table of precomputed factors holds."""
+    w = WL.scaled(WL.WORKLOADS["tiny"], n_tokens=4128 + 5, n_chunks=0)
+    c = Hn.Case(w)
+    ref, _ = c.oracle_attention(0)
+    got = c.gpu_decode(0)[0]
+    print("one head over every CTA", Hn.assert_attention_close(got, ref))
+
+
 def test_decode_is_deterministic():
     """No atomics and a fixed partition: two calls on the same cache give bit-identical outputs (both grids)."""
     w = WL.scaled(WL.WORKLOADS["step7b"], n_layers=2, batch=3, n_tokens=2048 + 17)
