@@ -823,6 +823,28 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     if (chunk > 0) stage_tail(chunk);
     cp_async_wait<0>();
     asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // the sequence's 128 threads
+    // A packed window's scores are norm * (sum_c q'_c m_c + sum_c (q'_c s_c) code_c): the bias and the weights
+    // W = q' s are the same for its 32 tokens, so they are formed once (in the key-row scratch, idle for such a
+    // window) and the per-token work is one multiply-add per code and head.
+    float* Wsm = reinterpret_cast<float*>(ksm);       // [GP][D] weights in (m, s)-plane order, then [4][GP] bias parts
+    float* bpart = Wsm + GP * D;
+    if (packed) {
+      float bj[GP];
+#pragma unroll
+      for (int j = 0; j < GP; j++) {
+        Wsm[j * D + c] = sm.qrot[0][bs * GP + j][c] * msf[D + c];
+        bj[j] = sm.qrot[1][bs * GP + j][c] * msf[c];
+      }
+#pragma unroll
+      for (int j = 0; j < GP; j++)
+#pragma unroll
+        for (int d = 16; d; d >>= 1) bj[j] += __shfl_xor_sync(0xffffffffu, bj[j], d);
+      if ((c & 31) == 0) {
+#pragma unroll
+        for (int j = 0; j < GP; j++) bpart[(c >> 5) * GP + j] = bj[j];
+      }
+      asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");
+    }
     if (tok < n_tail && j0 < G) {
       float a2[2] = {0.f, 0.f};
       if (!packed) {   // raw key
@@ -850,7 +872,11 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
         const int win = t / W, ti = t % W;
         const unsigned char* body = cv.body(layer, bb, h, win);
         const uint32_t* kw = reinterpret_cast<const uint32_t*>(body + B_KCODE) + (ti >> 4) * 128 + (ti & 7) * 16 + ((ti >> 3) & 1) * 2;
-        const int r0 = bs * GP + j0, r1 = bs * GP + min(j0 + 1, GP - 1);
+        const float* W0 = Wsm + j0 * D;
+        const float* W1 = Wsm + min(j0 + 1, GP - 1) * D;
+        a2[0] = (bpart[j0] + bpart[GP + j0]) + (bpart[2 * GP + j0] + bpart[3 * GP + j0]);
+        a2[1] = (bpart[min(j0 + 1, GP - 1)] + bpart[GP + min(j0 + 1, GP - 1)]) +
+                (bpart[2 * GP + min(j0 + 1, GP - 1)] + bpart[3 * GP + min(j0 + 1, GP - 1)]);
         for (int wi = 0; wi < 8; wi++) {
           const int tt = wi >> 1, ww = wi & 1, p0 = 32 * tt + 16 * ww;
           const uint32_t word = kw[tt * 4 + ww];
@@ -859,10 +885,9 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
 #pragma unroll
             for (int e2 = 0; e2 < 2; e2++) {
               const int pp = p0 + 2 * qq + e2;
-              const float mv = msf[pp];
-              const float sc = msf[D + pp] * (float)((word >> (16 * e2 + 8 * (qq >> 2) + 2 * (qq & 3))) & 3u);
-              a2[0] = fmaf(sm.qrot[0][r0][pp], sc, fmaf(sm.qrot[1][r0][pp], mv, a2[0]));
-              a2[1] = fmaf(sm.qrot[0][r1][pp], sc, fmaf(sm.qrot[1][r1][pp], mv, a2[1]));
+              const float code = (float)((word >> (16 * e2 + 8 * (qq >> 2) + 2 * (qq & 3))) & 3u);
+              a2[0] = fmaf(W0[pp], code, a2[0]);
+              a2[1] = fmaf(W1[pp], code, a2[1]);
             }
         }
         const float kn = __half2float(reinterpret_cast<const __half*>(body + B_KNORM)[norm_pos(ti)]);
