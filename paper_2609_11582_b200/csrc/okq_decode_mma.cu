@@ -877,9 +877,13 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
         a2[0] = (bpart[j0] + bpart[GP + j0]) + (bpart[2 * GP + j0] + bpart[3 * GP + j0]);
         a2[1] = (bpart[min(j0 + 1, GP - 1)] + bpart[GP + min(j0 + 1, GP - 1)]) +
                 (bpart[2 * GP + min(j0 + 1, GP - 1)] + bpart[3 * GP + min(j0 + 1, GP - 1)]);
+        uint32_t words[8];   // the token's 128 key codes, fetched together
+#pragma unroll
+        for (int wi = 0; wi < 8; wi++) words[wi] = kw[(wi >> 1) * 4 + (wi & 1)];
+#pragma unroll
         for (int wi = 0; wi < 8; wi++) {
           const int tt = wi >> 1, ww = wi & 1, p0 = 32 * tt + 16 * ww;
-          const uint32_t word = kw[tt * 4 + ww];
+          const uint32_t word = words[wi];
 #pragma unroll
           for (int qq = 0; qq < 8; qq++)
 #pragma unroll
