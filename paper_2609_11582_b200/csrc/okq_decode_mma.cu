@@ -203,6 +203,56 @@ __device__ __forceinline__ void query_fragments(const Segment& sg, int G, float 
   }
 }
 
+// Scores of one packed window against the group's queries, by one warp, from a staged image of the window's key
+// part ((m, s) planes, key norms, key codes at their record offsets): the split-K kernel's score step.
+// sc[nu][e] = log2-domain score of head g = lane >> 2 against token 8 nu + 2 (lane & 3) + e.
+__device__ __forceinline__ void window_scores_mma(const unsigned char* st, const uint2 (&qreg)[16], float fsc, int lane,
+                                                  float (&sc)[4][2]) {
+  const int t = lane & 3;
+  const uint4* mp = reinterpret_cast<const uint4*>(st + OFF_KM + 64 * t);
+  const uint4* sp = reinterpret_cast<const uint4*>(st + OFF_KS + 64 * t);
+  float dbA[4] = {0.f, 0.f, 0.f, 0.f}, dbB[4] = {0.f, 0.f, 0.f, 0.f};
+  float d[4][4];
+#pragma unroll
+  for (int nu = 0; nu < 4; nu++)
+#pragma unroll
+    for (int i = 0; i < 4; i++) d[nu][i] = 0.f;
+  const uint4 kc0 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * lane);
+  const uint4 kc1 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 512 + 16 * lane);
+  const uint32_t kw[4][2] = {{kc0.x, kc0.y}, {kc0.z, kc0.w}, {kc1.x, kc1.y}, {kc1.z, kc1.w}};
+#pragma unroll
+  for (int kq = 0; kq < 4; kq++) {
+    const uint4 m4 = mp[kq], s4 = sp[kq];
+#pragma unroll
+    for (int half = 0; half < 2; half++) {
+      const int kappa = 2 * kq + half;
+      const uint2 q0 = qreg[2 * kappa], q1 = qreg[2 * kappa + 1];
+      uint32_t a0, a1, a2, a3;
+      if (half) mma16816(dbB, q0.x, q0.y, q1.x, q1.y, m4.z, m4.w);
+      else mma16816(dbA, q0.x, q0.y, q1.x, q1.y, m4.x, m4.y);
+      split_product(u2h(q0.x), u2h(q0.y), u2h(half ? s4.z : s4.x), a0, a1);
+      split_product(u2h(q1.x), u2h(q1.y), u2h(half ? s4.w : s4.y), a2, a3);
+      const int ww = kappa >> 2, sh = (kappa >> 1) & 1;
+      const uint32_t mk0 = half ? 0x00300030u : 0x00030003u;
+      const uint32_t mk1 = half ? 0x00c000c0u : 0x000c000cu;
+#pragma unroll
+      for (int nu = 0; nu < 4; nu++) {
+        uint32_t src = sh ? (kw[nu][ww] >> 8) : kw[nu][ww];
+        mma16816(d[nu], a0, a1, a2, a3, src & mk0, src & mk1);
+      }
+    }
+  }
+  const uint4 kn4 = *reinterpret_cast<const uint4*>(st + OFF_KNORM + 16 * t);
+  const uint32_t knu[4] = {kn4.x, kn4.y, kn4.z, kn4.w};
+  const float bias0 = ((dbA[0] + dbB[0]) + (dbA[2] + dbB[2])) * 0x1p-24f;   // the code sums carry 2^-24, the bias does not
+#pragma unroll
+  for (int nu = 0; nu < 4; nu++) {
+    const float2 kn = __half22float2(u2h(knu[nu]));
+    sc[nu][0] = ((d[nu][0] + d[nu][2]) + bias0) * (kn.x * fsc);
+    sc[nu][1] = ((d[nu][1] + d[nu][3]) + bias0) * (kn.y * fsc);
+  }
+}
+
 // ---------------------------------------------------------------- score warp
 template <int FMT>
 __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, int G, float sm_scale, int pair,
@@ -696,9 +746,6 @@ struct CombineSmem {
   __align__(16) float mrg[CB_SEQ][MRG_TAB][GP][4];
   __align__(16) float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
   __align__(16) float rawv[CB_ROWS][D];       // raw-tail contribution, [row][channel]
-  // q' = H q in the order of the (m, s) planes, for the scores of packed keys: [0] multiplies s * code, [1] the
-  // stored m (divided by the m plane's position scale when that plane carries it)
-  __align__(16) float qrot[2][CAPTION ? CB_ROWS : 1][D];
   __align__(16) float tsc[CB_SEQ][TAIL][GP];  // tail scores (log2 domain), then softmax numerators
   float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
   // one-sequence blocks: the headers (m, l, weight sums) of the sequence's first MRG_TAB partials, fetched early
@@ -741,19 +788,22 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   const __half* qbase = P.q + (((size_t)li * cv.batch + bb) * cv.n_q_heads + h * G) * D;
   const __half* kt = cv.k_tail + cv.k_tail_off(layer, bb, h);
   const __half* vt = cv.v_tail + cv.v_tail_off(layer, bb, h);
-  // Scratch inside the rotated-sum array (written much later): per sequence the (m, s) of a packed window as
-  // floats, then the chunk's raw key rows (272-byte rows: 16-byte reads of 32 different rows hit different banks)
-  // and the group's query rows, both fetched with cp.async so that all their loads are in flight together.
+  // Scratch inside the rotated-sum array (written much later), per sequence: the raw key rows of a chunk of the
+  // tail (272-byte rows: 16-byte reads of 32 different rows hit different banks) or, under the captioning
+  // schedule, the key parts of the up to four packed windows among the raw-value tokens; then the group's query
+  // rows.  Everything is fetched with cp.async so that all the loads are in flight together.
   constexpr int KROW = D + 8;                              // halfs per staged key row
   constexpr int KSM_FLOATS = W * KROW / 2, QSM_FLOATS = GP * D / 2;
-  static_assert(CB_SEQ * (2 * D + KSM_FLOATS + QSM_FLOATS) <= 3 * CB_ROWS * D, "tail scratch must fit the rotated-sum array");
-  float* msf = &sm.vec[0][0][0] + bs * 2 * D;
-  __half* ksm = reinterpret_cast<__half*>(&sm.vec[0][0][0] + CB_SEQ * 2 * D + bs * (KSM_FLOATS + QSM_FLOATS));
+  constexpr int KIMG = OFF_VCODE + 144;                    // key part of a window record (+ its MXFP4 metadata bytes)
+  static_assert(CB_SEQ * (KSM_FLOATS + QSM_FLOATS) <= 3 * CB_ROWS * D && 4 * KIMG <= KSM_FLOATS * 4, "tail scratch must fit");
+  __half* ksm = reinterpret_cast<__half*>(&sm.vec[0][0][0] + bs * (KSM_FLOATS + QSM_FLOATS));
   __half* qsm = ksm + W * KROW;
+  unsigned char* kimg = reinterpret_cast<unsigned char*>(ksm);
+  const int npc = CAPTION ? (k_pk - v_pk) / W : 0;   // packed windows among the raw-value tokens: the first chunks
   // a chunk of the tail is one 32-token window: its keys are either all packed or all raw
   auto stage_tail = [&](int chunk) {
     if (chunk == 0 && c < G * (D / 8)) cp_async16(qsm + 8 * c, qbase + 8 * c);
-    if (!(CAPTION && v_pk + chunk * W < k_pk))
+    if (chunk >= npc)
       for (int idx = c; idx < W * (D / 8); idx += 128) {
         const int r = idx / (D / 8), c8 = idx % (D / 8);
         if (chunk * W + r < n_tail)
@@ -766,6 +816,20 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
       const int r = idx / (D / 8), c8 = idx % (D / 8);
       cp_async16(&sm.vsm[r * D + 8 * c8], vt + cv.v_slot(v_pk + r) * D + 8 * c8);
     }
+  for (int ch = 0; ch < npc; ch++) {   // key parts of the packed windows whose values are still raw
+    const int win = v_pk / W + ch;
+    unsigned char* img = kimg + ch * KIMG;
+    if (cv.fmt == FMT_FP16) {
+      const unsigned char* rec = cv.meta(layer, bb, h, win);   // the record starts with its (m, s) planes
+      if (c < OFF_VCODE / 16) cp_async16(img + 16 * c, rec + 16 * c);
+    } else {
+      const unsigned char* body = cv.body(layer, bb, h, win);
+      const unsigned char* meta = cv.meta(layer, bb, h, win);
+      if (c < 4) cp_async16(img + OFF_KNORM + 16 * c, body + B_KNORM + 16 * c);
+      else if (c < 4 + 64) cp_async16(img + OFF_KCODE + 16 * (c - 4), body + B_KCODE + 16 * (c - 4));
+      else if (c < 4 + 64 + MX_META_BYTES / 8) cp_async8(img + OFF_VCODE + 8 * (c - 68), meta + 8 * (c - 68));
+    }
+  }
   if (n_tail > 0) stage_tail(0);   // on its way while the prefix is computed
   const int total = block_prefix(cv, P.layer0, n_entries, sm.prefix);
   const int per = total > 0 ? (total + n_cta - 1) / n_cta : 1;
@@ -790,64 +854,47 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     }
     cp_async_commit();
   }
-  if (CAPTION) {   // q' = H q for the scores of packed keys: one warp per (sequence, head) row
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int row = warp; row < CB_ROWS; row += CB_SEQ * 4) {
-      const int rb = blockIdx.y * CB_SEQ + row / GP, j = row % GP;
-      float4 qr = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (rb < cv.batch && j < G) {
-        const float4 x = load_row4(P.q + (((size_t)li * cv.batch + rb) * cv.n_q_heads + h * G + j) * D, lane);
-        const float4 sg = *reinterpret_cast<const float4*>(P.signs + (size_t)li * D + 4 * lane);
-        qr = warp_fwht(make_float4(x.x * sg.x, x.y * sg.y, x.z * sg.z, x.w * sg.w), lane);
-      }
-      const float v4[4] = {qr.x * RSQRT_D, qr.y * RSQRT_D, qr.z * RSQRT_D, qr.w * RSQRT_D};
-#pragma unroll
-      for (int u = 0; u < 4; u++) {
-        const int ch = 4 * lane + u, pp = meta_pos(ch);
-        sm.qrot[0][row][pp] = v4[u];
-        sm.qrot[1][row][pp] = cv.fmt == FMT_FP16 ? v4[u] * (1.0f / (float)(1 << (2 * meta_shift(ch)))) : v4[u];
-      }
-    }
+  if (CAPTION) {   // scores of the packed windows among the raw-value tokens: one warp per window, on the tensor cores
+    cp_async_wait<0>();
     __syncthreads();
+    const int wv = c >> 5, lane = c & 31;
+    if (wv < npc) {
+      Segment sq;
+      sq.q = qbase;
+      sq.signs = P.signs + (size_t)li * D;
+      uint2 qreg[16];
+      float fsc;
+      query_fragments(sq, G, P.sm_scale, lane, qreg, fsc);
+      unsigned char* st = kimg + wv * KIMG;
+      if (cv.fmt == FMT_MXFP4) {   // decode the stored (m, s) into the fp16 planes of the staged image
+        uint2 m4, s4;
+        mx_decode_lane(st + OFF_VCODE, lane, m4, s4);
+        *reinterpret_cast<uint2*>(st + OFF_KM + 8 * lane) = m4;
+        *reinterpret_cast<uint2*>(st + OFF_KS + 8 * lane) = s4;
+        __syncwarp();
+      }
+      float sc[4][2];
+      window_scores_mma(st, qreg, fsc, lane, sc);
+      const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+      for (int nu = 0; nu < 4; nu++)
+#pragma unroll
+        for (int e2 = 0; e2 < 2; e2++)
+          sm.tsc[bs][wv * W + 8 * nu + 2 * t + e2][g] = g < G ? sc[nu][e2] : -INFINITY;
+    }
+    __syncthreads();   // the images are done with: the scratch takes raw key rows next
   }
   // tail scores: thread -> (token = c & 31 of a 32-token chunk, heads (c >> 5) * 2 + {0, 1})
-  for (int chunk = 0; chunk * W < n_tail; chunk++) {
-    const int tok = chunk * W + (c & 31), t = v_pk + tok;
+  for (int chunk = npc; chunk * W < n_tail; chunk++) {   // chunks of raw keys
+    const int tok = chunk * W + (c & 31);
     float s2[2] = {-INFINITY, -INFINITY};
     const int j0 = (c >> 5) * 2;
-    const bool packed = CAPTION && v_pk + chunk * W < k_pk;
-    if (packed) {
-      const float2 ms = window_meta_pos(cv.meta(layer, bb, h, (v_pk + chunk * W) / W), cv.fmt, c);
-      msf[c] = ms.x; msf[D + c] = ms.y;
-    }
     if (chunk > 0) stage_tail(chunk);
     cp_async_wait<0>();
     asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // the sequence's 128 threads
-    // A packed window's scores are norm * (sum_c q'_c m_c + sum_c (q'_c s_c) code_c): the bias and the weights
-    // W = q' s are the same for its 32 tokens, so they are formed once (in the key-row scratch, idle for such a
-    // window) and the per-token work is one multiply-add per code and head.
-    float* Wsm = reinterpret_cast<float*>(ksm);       // [GP][D] weights in (m, s)-plane order, then [4][GP] bias parts
-    float* bpart = Wsm + GP * D;
-    if (packed) {
-      float bj[GP];
-#pragma unroll
-      for (int j = 0; j < GP; j++) {
-        Wsm[j * D + c] = sm.qrot[0][bs * GP + j][c] * msf[D + c];
-        bj[j] = sm.qrot[1][bs * GP + j][c] * msf[c];
-      }
-#pragma unroll
-      for (int j = 0; j < GP; j++)
-#pragma unroll
-        for (int d = 16; d; d >>= 1) bj[j] += __shfl_xor_sync(0xffffffffu, bj[j], d);
-      if ((c & 31) == 0) {
-#pragma unroll
-        for (int j = 0; j < GP; j++) bpart[(c >> 5) * GP + j] = bj[j];
-      }
-      asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");
-    }
     if (tok < n_tail && j0 < G) {
       float a2[2] = {0.f, 0.f};
-      if (!packed) {   // raw key
+      {
         const __half* krow = ksm + (c & 31) * KROW;
 #pragma unroll 4
         for (int k = 0; k < D; k += 8) {
@@ -866,36 +913,6 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
             }
           }
         }
-      } else {   // packed key: q . k_hat = norm * sum_c q'_c (m_c + s_c code_c)
-        // the 16 codes of word (tt, ww) of a token belong to the consecutive positions 32 tt + 16 ww .. + 15 of
-        // the (m, s) planes
-        const int win = t / W, ti = t % W;
-        const unsigned char* body = cv.body(layer, bb, h, win);
-        const uint32_t* kw = reinterpret_cast<const uint32_t*>(body + B_KCODE) + (ti >> 4) * 128 + (ti & 7) * 16 + ((ti >> 3) & 1) * 2;
-        const float* W0 = Wsm + j0 * D;
-        const float* W1 = Wsm + min(j0 + 1, GP - 1) * D;
-        a2[0] = (bpart[j0] + bpart[GP + j0]) + (bpart[2 * GP + j0] + bpart[3 * GP + j0]);
-        a2[1] = (bpart[min(j0 + 1, GP - 1)] + bpart[GP + min(j0 + 1, GP - 1)]) +
-                (bpart[2 * GP + min(j0 + 1, GP - 1)] + bpart[3 * GP + min(j0 + 1, GP - 1)]);
-        uint32_t words[8];   // the token's 128 key codes, fetched together
-#pragma unroll
-        for (int wi = 0; wi < 8; wi++) words[wi] = kw[(wi >> 1) * 4 + (wi & 1)];
-#pragma unroll
-        for (int wi = 0; wi < 8; wi++) {
-          const int tt = wi >> 1, ww = wi & 1, p0 = 32 * tt + 16 * ww;
-          const uint32_t word = words[wi];
-#pragma unroll
-          for (int qq = 0; qq < 8; qq++)
-#pragma unroll
-            for (int e2 = 0; e2 < 2; e2++) {
-              const int pp = p0 + 2 * qq + e2;
-              const float code = (float)((word >> (16 * e2 + 8 * (qq >> 2) + 2 * (qq & 3))) & 3u);
-              a2[0] = fmaf(W0[pp], code, a2[0]);
-              a2[1] = fmaf(W1[pp], code, a2[1]);
-            }
-        }
-        const float kn = __half2float(reinterpret_cast<const __half*>(body + B_KNORM)[norm_pos(ti)]);
-        a2[0] *= kn; a2[1] *= kn;
       }
       s2[0] = a2[0] * P.sm_scale * LOG2E;
       if (j0 + 1 < G) s2[1] = a2[1] * P.sm_scale * LOG2E;
