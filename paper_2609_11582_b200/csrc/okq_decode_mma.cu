@@ -919,7 +919,21 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     }
     if (tok < sm.TAIL) { sm.tsc[bs][tok][j0] = s2[0]; sm.tsc[bs][tok][j0 + 1] = s2[1]; }
     if ((chunk + 1) * W < n_tail)
-      asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // before the next chunk's rows or (m, s) land
+      asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // before the next chunk's rows land
+  }
+  // Blocks of several sequences have no room to hold all raw value rows: they pass through the key-row scratch 32
+  // rows at a time, the first 32 on their way from here on (used once the softmax numerators are known).
+  __half* vrows = ksm;
+  auto stage_values = [&](int r0) {
+    for (int idx = c; idx < min(W, n_tail - r0) * (D / 8); idx += 128) {
+      const int r = idx / (D / 8), c8 = idx % (D / 8);
+      cp_async16(vrows + r * D + 8 * c8, vt + cv.v_slot(v_pk + r0 + r) * D + 8 * c8);
+    }
+    cp_async_commit();
+  };
+  if (SEQ != 1 && n_tail > 0) {
+    asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // the last chunk's key rows have been read
+    stage_values(0);
   }
   // four column slices per (head, sequence): this block's 32 columns of the three matrices (48 KB) start their way
   // into shared memory now (behind the tail's own cp.async groups, which had to be waited for) and are used at the
@@ -986,15 +1000,28 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   float araw[GP];
 #pragma unroll
   for (int j = 0; j < GP; j++) araw[j] = 0.f;
+  constexpr int TAIL_ALL = 1 << 20;   // one-sequence blocks hold all their raw value rows: a single pass
+  for (int r0 = 0; r0 < n_tail; r0 += (SEQ == 1 ? TAIL_ALL : W)) {
+    const __half* rows = SEQ == 1 ? sm.vsm : vrows;
+    if (SEQ != 1) {
+      if (r0 > 0) {
+        asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // everyone is done with the previous rows
+        stage_values(r0);
+      }
+      cp_async_wait<0>();
+      asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");
+    }
+    const int nr = SEQ == 1 ? n_tail : min(W, n_tail - r0);
 #pragma unroll 8
-  for (int i = 0; i < n_tail; i++) {
-    const float x = __half2float(SEQ == 1 ? sm.vsm[i * D + c] : vt[cv.v_slot(v_pk + i) * D + c]);
-    const float4 w0 = *reinterpret_cast<const float4*>(&sm.tsc[bs][i][0]);
-    const float4 w1 = *reinterpret_cast<const float4*>(&sm.tsc[bs][i][4]);
-    araw[0] = fmaf(w0.x, x, araw[0]); araw[1] = fmaf(w0.y, x, araw[1]);
-    araw[2] = fmaf(w0.z, x, araw[2]); araw[3] = fmaf(w0.w, x, araw[3]);
-    araw[4] = fmaf(w1.x, x, araw[4]); araw[5] = fmaf(w1.y, x, araw[5]);
-    araw[6] = fmaf(w1.z, x, araw[6]); araw[7] = fmaf(w1.w, x, araw[7]);
+    for (int i = 0; i < nr; i++) {
+      const float x = __half2float(rows[i * D + c]);
+      const float4 w0 = *reinterpret_cast<const float4*>(&sm.tsc[bs][r0 + i][0]);
+      const float4 w1 = *reinterpret_cast<const float4*>(&sm.tsc[bs][r0 + i][4]);
+      araw[0] = fmaf(w0.x, x, araw[0]); araw[1] = fmaf(w0.y, x, araw[1]);
+      araw[2] = fmaf(w0.z, x, araw[2]); araw[3] = fmaf(w0.w, x, araw[3]);
+      araw[4] = fmaf(w1.x, x, araw[4]); araw[5] = fmaf(w1.y, x, araw[5]);
+      araw[6] = fmaf(w1.z, x, araw[6]); araw[7] = fmaf(w1.w, x, araw[7]);
+    }
   }
   // merge of the split-K partials, four heads at a time: per partial the twelve accumulator fragments of this
   // thread's channel are fetched together (independent loads), then scaled by the table's factors
