@@ -748,6 +748,7 @@ struct CombineSmem {
   __align__(16) float rawv[CB_ROWS][D];       // raw-tail contribution, [row][channel]
   __align__(16) float tsc[CB_SEQ][TAIL][GP];  // tail scores (log2 domain), then softmax numerators
   float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
+  float red[CB_SEQ][4][GP];   // per warp of a sequence: partial maxima / sums of the softmax bookkeeping
   // one-sequence blocks: the headers (m, l, weight sums) of the sequence's first MRG_TAB partials, fetched early
   __align__(16) float hdr[SEQ == 1 ? MRG_TAB * PARTIAL_HDR_FLOATS : 4];
   __align__(16) __half vsm[SEQ == 1 ? TAIL * D : 8];   // one-sequence blocks: the raw value rows, fetched early
@@ -952,23 +953,45 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   // the newest group, may stay in flight
   if (SEQ == 1) { if (PRELOAD) cp_async_wait<1>(); else cp_async_wait<0>(); }
   __syncthreads();
-  if (c < GP) {
+  {
+    // Softmax bookkeeping by all 128 threads of the sequence: thread = (head j, stripe); a stripe takes every 16th
+    // partial and every 16th tail token (the captioning schedule has up to 159 of them); stripes are joined by two
+    // shuffles inside a warp and a four-entry table across the warps.
+    const int j = c & (GP - 1), stripe = c >> 3, wv = c >> 5, lane = c & 31;
+    const int n_part = cta_hi - cta_lo + 1;
+    auto part_m = [&](int ci) {
+      return ci < n_hdr ? sm.hdr[ci * PARTIAL_HDR_FLOATS + j] : P.partials_f[(size_t)unit + cta_lo + ci].m[j];
+    };
+    auto part_l = [&](int ci) {
+      return ci < n_hdr ? sm.hdr[ci * PARTIAL_HDR_FLOATS + GP + j] : P.partials_f[(size_t)unit + cta_lo + ci].l[j];
+    };
     float M = -INFINITY;
-    for (int ci = 0; ci < n_hdr; ci++) M = fmaxf(M, sm.hdr[ci * PARTIAL_HDR_FLOATS + c]);
-    for (int ct = cta_lo + n_hdr; ct <= cta_hi; ct++) M = fmaxf(M, P.partials_f[(size_t)unit + ct].m[c]);
-    for (int i = 0; i < n_tail; i++) M = fmaxf(M, sm.tsc[bs][i][c]);
+    for (int ci = stripe; ci < n_part; ci += 16) M = fmaxf(M, part_m(ci));
+    for (int i = stripe; i < n_tail; i += 16) M = fmaxf(M, sm.tsc[bs][i][j]);
+    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 8));
+    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 16));
+    if (lane < GP) sm.red[bs][wv][j] = M;
+    asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");
+    M = fmaxf(fmaxf(sm.red[bs][0][j], sm.red[bs][1][j]), fmaxf(sm.red[bs][2][j], sm.red[bs][3][j]));
+    asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // the table is reused for the sums
     float L = 0.f;
-    for (int ci = 0; ci < n_hdr; ci++) {
-      const float pm = sm.hdr[ci * PARTIAL_HDR_FLOATS + c];
-      if (pm != -INFINITY) L += sm.hdr[ci * PARTIAL_HDR_FLOATS + GP + c] * exp2f(pm - M);
+    for (int ci = stripe; ci < n_part; ci += 16) {
+      const float pm = part_m(ci);
+      if (pm != -INFINITY) L += part_l(ci) * exp2f(pm - M);
     }
-    for (int ct = cta_lo + n_hdr; ct <= cta_hi; ct++) {
-      const PartialF& pp = P.partials_f[(size_t)unit + ct];
-      if (pp.m[c] != -INFINITY) L += pp.l[c] * exp2f(pp.m[c] - M);
+    for (int i = stripe; i < n_tail; i += 16) {   // softmax numerators in place of the scores
+      const float pnum = exp2f(sm.tsc[bs][i][j] - M);   // 0 for the heads beyond the group (-inf scores)
+      sm.tsc[bs][i][j] = pnum;
+      L += pnum;
     }
-    for (int i = 0; i < n_tail; i++) L += exp2f(sm.tsc[bs][i][c] - M);
-    sm.Ms[bs][c] = M;
-    sm.Ls[bs][c] = L;
+    L += __shfl_xor_sync(0xffffffffu, L, 8);
+    L += __shfl_xor_sync(0xffffffffu, L, 16);
+    if (lane < GP) sm.red[bs][wv][j] = L;
+    asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");
+    if (c < GP) {
+      sm.Ms[bs][c] = M;
+      sm.Ls[bs][c] = (sm.red[bs][0][c] + sm.red[bs][1][c]) + (sm.red[bs][2][c] + sm.red[bs][3][c]);
+    }
   }
   __syncthreads();
   // per partial and head: the rescale factor exp2(m - M) and the weight sums S_m (the four lanes of a quad hold
@@ -991,12 +1014,8 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     }
     *reinterpret_cast<float4*>(sm.mrg[bs][ci][j]) = f;
   }
-  // raw-value tokens: softmax numerators in place of the scores, then every value row is read once for all heads
-  for (int idx = c; idx < n_tail * GP; idx += 128) {
-    const int i = idx / GP, j = idx % GP;
-    sm.tsc[bs][i][j] = exp2f(sm.tsc[bs][i][j] - sm.Ms[bs][j]);   // 0 for the heads beyond the group (-inf scores)
-  }
   __syncthreads();
+  // raw-value tokens: every value row is read once for all heads
   float araw[GP];
 #pragma unroll
   for (int j = 0; j < GP; j++) araw[j] = 0.f;
