@@ -746,7 +746,11 @@ struct CombineSmem {
   __align__(16) float mrg[CB_SEQ][MRG_TAB][GP][4];
   __align__(16) float vec[3][CB_ROWS][D];     // merged rotated-basis sums, [modality][row][rotated channel]
   __align__(16) float rawv[CB_ROWS][D];       // raw-tail contribution, [row][channel]
-  __align__(16) float tsc[CB_SEQ][TAIL][GP];  // tail scores (log2 domain), then softmax numerators
+  // tail scores (log2 domain), then softmax numerators, [sequence][token][head]: blocks of several sequences keep
+  // them in the matrix ring, which is idle until the rotated sums are complete
+  static constexpr bool TSC_IN_RING = SEQ != 1;
+  static_assert(!TSC_IN_RING || CB_SEQ * TAIL * GP <= RBUF_FLOATS, "tail scores must fit the matrix ring");
+  __align__(16) float tsc_own[TSC_IN_RING ? 4 : CB_SEQ * TAIL * GP];
   float Ms[CB_SEQ][GP], Ls[CB_SEQ][GP];
   float red[CB_SEQ][4][GP];   // per warp of a sequence: partial maxima / sums of the softmax bookkeeping
   // one-sequence blocks: the headers (m, l, weight sums) of the sequence's first MRG_TAB partials, fetched early
@@ -769,10 +773,12 @@ __device__ __forceinline__ float2 window_meta_pos(const unsigned char* meta, int
 // NS: CTAs that share one (head, sequence group): each computes D / NS output columns (used when the grid
 // would otherwise leave most SMs idle; the merge is repeated by every slice, the matrix streaming is split)
 template <bool CAPTION, int NS, int SEQ>
-__global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n_cta) {
+__global__ void __launch_bounds__(SEQ * 128, SEQ == CB_SEQ_MAX ? 2 : 1) k_combine_mma(DecodeParams P, int n_cta) {
   constexpr int CB_SEQ = SEQ, CB_ROWS = SEQ * GP;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   CombineSmem<CAPTION, SEQ>& sm = *reinterpret_cast<CombineSmem<CAPTION, SEQ>*>(smem_raw);
+  float* const tsc_base = sm.TSC_IN_RING ? &sm.Rbuf[0] : &sm.tsc_own[0];
+  auto tsc = [&](int b_, int i_) -> float* { return tsc_base + ((size_t)b_ * sm.TAIL + i_) * GP; };   // one token's eight heads
   const CacheView& cv = P.cv;
   const int h = blockIdx.x / NS, sl = blockIdx.x % NS, li = blockIdx.z, layer = P.layer0 + li;
   const int bs = threadIdx.x >> 7, c = threadIdx.x & 127;
@@ -881,7 +887,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
       for (int nu = 0; nu < 4; nu++)
 #pragma unroll
         for (int e2 = 0; e2 < 2; e2++)
-          sm.tsc[bs][wv * W + 8 * nu + 2 * t + e2][g] = g < G ? sc[nu][e2] : -INFINITY;
+          tsc(bs, wv * W + 8 * nu + 2 * t + e2)[g] = g < G ? sc[nu][e2] : -INFINITY;
     }
     __syncthreads();   // the images are done with: the scratch takes raw key rows next
   }
@@ -918,7 +924,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
       s2[0] = a2[0] * P.sm_scale * LOG2E;
       if (j0 + 1 < G) s2[1] = a2[1] * P.sm_scale * LOG2E;
     }
-    if (tok < sm.TAIL) { sm.tsc[bs][tok][j0] = s2[0]; sm.tsc[bs][tok][j0 + 1] = s2[1]; }
+    if (tok < sm.TAIL) { tsc(bs, tok)[j0] = s2[0]; tsc(bs, tok)[j0 + 1] = s2[1]; }
     if ((chunk + 1) * W < n_tail)
       asm volatile("bar.sync %0, 128;\n" ::"r"(bs + 1) : "memory");   // before the next chunk's rows land
   }
@@ -967,7 +973,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     };
     float M = -INFINITY;
     for (int ci = stripe; ci < n_part; ci += 16) M = fmaxf(M, part_m(ci));
-    for (int i = stripe; i < n_tail; i += 16) M = fmaxf(M, sm.tsc[bs][i][j]);
+    for (int i = stripe; i < n_tail; i += 16) M = fmaxf(M, tsc(bs, i)[j]);
     M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 8));
     M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 16));
     if (lane < GP) sm.red[bs][wv][j] = M;
@@ -980,8 +986,8 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
       if (pm != -INFINITY) L += part_l(ci) * exp2f(pm - M);
     }
     for (int i = stripe; i < n_tail; i += 16) {   // softmax numerators in place of the scores
-      const float pnum = exp2f(sm.tsc[bs][i][j] - M);   // 0 for the heads beyond the group (-inf scores)
-      sm.tsc[bs][i][j] = pnum;
+      const float pnum = exp2f(tsc(bs, i)[j] - M);   // 0 for the heads beyond the group (-inf scores)
+      tsc(bs, i)[j] = pnum;
       L += pnum;
     }
     L += __shfl_xor_sync(0xffffffffu, L, 8);
@@ -1034,8 +1040,8 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
 #pragma unroll 8
     for (int i = 0; i < nr; i++) {
       const float x = __half2float(rows[i * D + c]);
-      const float4 w0 = *reinterpret_cast<const float4*>(&sm.tsc[bs][r0 + i][0]);
-      const float4 w1 = *reinterpret_cast<const float4*>(&sm.tsc[bs][r0 + i][4]);
+      const float4 w0 = *reinterpret_cast<const float4*>(tsc(bs, r0 + i));
+      const float4 w1 = *reinterpret_cast<const float4*>(tsc(bs, r0 + i) + 4);
       araw[0] = fmaf(w0.x, x, araw[0]); araw[1] = fmaf(w0.y, x, araw[1]);
       araw[2] = fmaf(w0.z, x, araw[2]); araw[3] = fmaf(w0.w, x, araw[3]);
       araw[4] = fmaf(w1.x, x, araw[4]); araw[5] = fmaf(w1.y, x, araw[5]);
@@ -1133,8 +1139,10 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
   if (PRELOAD) {
     cp_async_wait<0>();
     __syncthreads();   // the matrices have landed and vec is complete
-  } else if (!comp) {
-    for (int pre = 0; pre < CB_NBUF - 1; pre++) stage(pre);
+  } else {
+    if (sm.TSC_IN_RING) __syncthreads();   // everyone has read its softmax numerators: the ring takes matrices now
+    if (!comp)
+      for (int pre = 0; pre < CB_NBUF - 1; pre++) stage(pre);
   }
   for (int chunk = 0; chunk < N_CHUNK; chunk++) {
     if (!PRELOAD) {
@@ -1176,7 +1184,7 @@ __global__ void __launch_bounds__(SEQ * 128) k_combine_mma(DecodeParams P, int n
     }
   }
   if (PRE) {   // the second half's sums reach the first through the tail-score array, idle by now
-    float* red = &sm.tsc[0][0][0] + (threadIdx.x % (CB_SEQ * 64)) * 4 * CW;
+    float* red = &sm.tsc_own[0] + (threadIdx.x % (CB_SEQ * 64)) * 4 * CW;
     static_assert(!PRE || CB_SEQ * 64 * 4 * CW <= CB_SEQ * W * GP, "reduction scratch");
     if (khalf) {
 #pragma unroll
