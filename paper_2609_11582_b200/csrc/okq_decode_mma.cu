@@ -1048,6 +1048,9 @@ __global__ void __launch_bounds__(SEQ * 128, SEQ == CB_SEQ_MAX ? 2 : 1) k_combin
       araw[6] = fmaf(w1.z, x, araw[6]); araw[7] = fmaf(w1.w, x, araw[7]);
     }
   }
+  // (the value rows passed through scratch inside the rotated-sum array, which the merge below fills: a sequence
+  // group must not start writing it while another still reads its rows)
+  if (SEQ != 1) __syncthreads();
   // merge of the split-K partials, four heads at a time: per partial the twelve accumulator fragments of this
   // thread's channel are fetched together (independent loads), then scaled by the table's factors
 #pragma unroll

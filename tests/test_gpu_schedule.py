@@ -111,3 +111,39 @@ def test_append_equals_bulk_and_decode_at_every_step():
             got = _decode(part, w, q, signs, R)
             ref = _oracle(w, k, v, mod, signs, R, q, n, B.META_FP16)
             Hn.assert_attention_close(got, ref)
+
+
+@pytest.mark.parametrize("schedule", [B.SCHEDULE_WINDOW, CAP])
+def test_full_size_batched_call_equals_per_layer_calls(schedule):
+    """The 28-layer call runs the combine kernel in its four-sequences-per-block configuration, a single-layer call
+    in the one-sequence configuration (which the small cases above reach and check against the oracle).  Both must
+    give the same attention output up to the rounding of a different split of the windows; repeated a few steps so
+    that a timing-dependent fault between the sequence groups of a block would show (non-finite or far-off values)."""
+    w = WL.WORKLOADS["step7b"]
+    dev = torch.device("cuda")
+    L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
+    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev, schedule=schedule)
+    mod = WL.modality_layout(w).unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
+    signs = torch.stack([WL.gen_signs(w, l) for l in range(L)]).to(dev)
+    R = torch.stack([WL.gen_rotations(w, l) for l in range(L)]).unsqueeze(1).contiguous().to(dev)
+    for l in range(L):
+        k, v = WL.gen_kv(w, l, device=dev)
+        B.quantize_keys(cache, l, k, signs[l])
+        B.quantize_values(cache, l, v, mod, R[l], bulk=True)
+        del k, v
+    q = torch.stack([WL.gen_queries(w, l) for l in range(L)]).to(dev)
+    ws = torch.empty(B.decode_workspace_bytes(cache, L, 0), dtype=torch.uint8, device=dev)
+    for s in range(6):
+        kn, vn, mn = WL.gen_new_token(w, 0, s, device=dev)
+        kn = kn.unsqueeze(0).expand(L, -1, -1, -1).contiguous()
+        vn = vn.unsqueeze(0).expand(L, -1, -1, -1).contiguous()
+        B.append(cache, 0, L, kn, vn, mn, signs, R)
+        a = torch.full((L, Bn, Hq, D), float("nan"), dtype=torch.float32, device=dev)
+        b = torch.full_like(a, float("nan"))
+        B.decode_attention(cache, 0, L, q, signs, R, ws, a)
+        for l in range(L):
+            B.decode_attention(cache, l, 1, q[l:l + 1], signs[l:l + 1], R[l:l + 1], ws, b[l:l + 1])
+        torch.cuda.synchronize()
+        assert torch.isfinite(a).all() and torch.isfinite(b).all(), s
+        assert (a - b).abs().max().item() < 2e-3, (s, (a - b).abs().max().item())
+    assert cache.device_status() == 0
