@@ -59,6 +59,18 @@ def test_one_modality_long_ranges():
         print("one modality, splits", splits, errs)
 
 
+@pytest.mark.parametrize("meta_format", [B.META_FP16, B.META_MXFP4])
+def test_middle_sized_grid(meta_format):
+    """64 (head, four-sequence group, layer) blocks: fewer than SMs but too many for four column slices each, the
+    case in which the combine kernel runs one sequence per block over all columns."""
+    w = WL.scaled(WL.WORKLOADS["step7b"], n_layers=8, n_tokens=1024 + 7)
+    c = Hn.Case(w, meta_format=meta_format)
+    got = c.gpu_decode(0, layer_count=w.n_layers)
+    for l in (0, 3, 7):
+        ref, _ = c.oracle_attention(l)
+        Hn.assert_attention_close(got[l], ref)
+
+
 def test_one_head_over_every_cta():
     """A single (sequence, head) unit of 129 windows: every CTA of the split-K kernel holds one window of it, so the
     combine kernel merges 129 partials for one head group, more than its table of precomputed factors holds."""
