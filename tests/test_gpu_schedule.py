@@ -147,3 +147,110 @@ def test_full_size_batched_call_equals_per_layer_calls(schedule):
         assert torch.isfinite(a).all() and torch.isfinite(b).all(), s
         assert (a - b).abs().max().item() < 2e-3, (s, (a - b).abs().max().item())
     assert cache.device_status() == 0
+
+
+def _check_sampled(cache, w, samples, kept, q, signs, R, mod_row, n, out, meta_format):
+    """Sampled (layer, sequence) pairs of a caption-schedule cache of `n` tokens per sequence against the oracle:
+    packed records bit for bit up to the schedule's packed counts, attention output within the tolerance."""
+    H, G = w.n_kv_heads, w.group
+    kp, vp = O.packed_counts(n, 1)
+    for (sl, sb) in samples:
+        kc, vc = kept[(sl, sb)]                                  # [H, n, 128] fp16, host
+        kb, vb = Hn.u16(kc), Hn.u16(vc)
+        kq, vq, _ = O.quantize_batch(kb, vb, mod_row, signs[sl].numpy(), R[sl].numpy(), meta_format=meta_format)
+        e = B.cache_export(cache, sl)
+        torch.cuda.synchronize()
+        assert (e["k_codes"][sb].cpu().numpy()[:, :kp] == kq["codes"][:, :kp]).all()
+        assert (Hn.u16(e["k_norm"][sb])[:, :kp] == kq["norm"][:, :kp]).all()
+        assert (Hn.u16(e["k_meta"][sb])[:, :kp // W] == kq["meta"][:, :kp // W]).all()
+        assert (e["v_codes"][sb].cpu().numpy()[:, :vp] == vq["codes"][:, :vp]).all()
+        assert (Hn.u16(e["v_norm"][sb])[:, :vp] == vq["norm"][:, :vp]).all()
+        del e
+        ref = np.zeros((w.n_q_heads, D))
+        for h in range(H):
+            kq1 = {a: x[h] for a, x in kq.items()}; vq1 = {a: x[h] for a, x in vq.items()}
+            ref[h * G:(h + 1) * G] = O.attention_scheduled(Hn.u16(q[sl, sb, h * G:(h + 1) * G]), kq1, vq1, mod_row, kb[h], vb[h],
+                                                           signs[sl].numpy(), R[sl].numpy(), kp, vp)
+        errs = Hn.assert_attention_close(out[sl, sb], ref)
+        print(f"caption n={n} meta {meta_format} layer {sl} seq {sb}: rel-L2 {errs[0]:.2e} worst head {errs[1]:.2e} max-abs {errs[2]:.2e}")
+
+
+@pytest.mark.parametrize("meta_format", [B.META_FP16, B.META_MXFP4])
+def test_middle_sized_grid_caption(meta_format):
+    """Captioning schedule with 64 (head, four-sequence group, layer) combine blocks: fewer than SMs but too many for
+    four column slices each, so the combine kernel runs one sequence per block over all output columns; every
+    sequence holds packed keys whose values are still raw, raw keys and raw values.  Against the oracle."""
+    w = WL.scaled(WL.WORKLOADS["step7b"], n_layers=8, n_tokens=1024 + 77)
+    n, L, dev = w.n_tokens, w.n_layers, torch.device("cuda")
+    cache = B.Cache(L, w.batch, w.n_kv_heads, w.n_q_heads, ((n + 31) // 32 + 2) * 32, device=dev, meta_format=meta_format, schedule=CAP)
+    mod_cpu = WL.modality_layout(w)
+    mod = mod_cpu.unsqueeze(0).repeat(w.batch, 1).contiguous().to(dev)
+    signs = torch.stack([WL.gen_signs(w, l) for l in range(L)])
+    R = torch.stack([WL.gen_rotations(w, l) for l in range(L)])
+    q = torch.stack([WL.gen_queries(w, l) for l in range(L)])
+    d_signs, d_R = signs.to(dev), R.unsqueeze(1).contiguous().to(dev)
+    samples = [(0, 0), (3, 5), (7, 2), (7, 7)]
+    kept = {}
+    for l in range(L):
+        k, v = WL.gen_kv(w, l)
+        B.quantize_keys(cache, l, k.to(dev), d_signs[l])
+        B.quantize_values(cache, l, v.to(dev), mod, d_R[l], bulk=(l % 2 == 0))
+        for (sl, sb) in samples:
+            if sl == l:
+                kept[(sl, sb)] = (k[sb], v[sb])
+    ws = torch.empty(B.decode_workspace_bytes(cache, L, 0), dtype=torch.uint8, device=dev)
+    out = torch.full((L, w.batch, w.n_q_heads, D), float("nan"), dtype=torch.float32, device=dev)
+    B.decode_attention(cache, 0, L, q.to(dev), d_signs, d_R, ws, out)
+    torch.cuda.synchronize()
+    assert cache.device_status() == 0
+    o = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(o).all()
+    _check_sampled(cache, w, samples, kept, q, signs, R, mod_cpu.numpy(), n, o, meta_format)
+
+
+@pytest.mark.parametrize("meta_format", [B.META_FP16, B.META_MXFP4])
+def test_full_7b_step_caption_sampled(meta_format):
+    """The full 7B decode step under the captioning schedule (28 layers x batch 8, one append call and one decode call
+    over all layers: the combine kernel's four-sequences-per-block configuration), after 45 appended tokens that cross
+    a 32-token boundary (a value window leaves the fp16 window) and a 128-token boundary (four key windows are
+    packed); sampled (layer, sequence) pairs against the oracle."""
+    w0 = WL.WORKLOADS["step7b"]
+    n0, n_app = w0.n_tokens - 40, 45
+    n = n0 + n_app
+    w = WL.scaled(w0, n_tokens=n0)
+    dev = torch.device("cuda")
+    L, Bn, H, Hq = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads
+    cache = B.Cache(L, Bn, H, Hq, w0.n_tokens + 64, device=dev, meta_format=meta_format, schedule=CAP)
+    mod_cpu = WL.modality_layout(w)
+    mod = mod_cpu.unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
+    signs = torch.stack([WL.gen_signs(w, l) for l in range(L)])
+    R = torch.stack([WL.gen_rotations(w, l) for l in range(L)])
+    q = torch.stack([WL.gen_queries(w, l) for l in range(L)])
+    d_signs, d_R = signs.to(dev), R.unsqueeze(1).contiguous().to(dev)
+    samples = [(0, 0), (13, 5), (27, 7)]
+    kept = {}
+    for l in range(L):
+        k, v = WL.gen_kv(w, l, device=dev)
+        B.quantize_keys(cache, l, k, d_signs[l])
+        B.quantize_values(cache, l, v, mod, d_R[l])
+        for (sl, sb) in samples:
+            if sl == l:
+                kept[(sl, sb)] = (k[sb].cpu(), v[sb].cpu())
+        del k, v
+    new_k, new_v = [], []
+    for s in range(n_app):
+        kn, vn, mn = WL.gen_new_token(w, 0, s, device=dev)
+        new_k.append(kn.cpu()); new_v.append(vn.cpu())
+        B.append(cache, 0, L, kn.unsqueeze(0).expand(L, -1, -1, -1).contiguous(), vn.unsqueeze(0).expand(L, -1, -1, -1).contiguous(),
+                 mn, d_signs, d_R)
+    ws = torch.empty(B.decode_workspace_bytes(cache, L, 0), dtype=torch.uint8, device=dev)
+    out = torch.full((L, Bn, Hq, D), float("nan"), dtype=torch.float32, device=dev)
+    B.decode_attention(cache, 0, L, q.to(dev), d_signs, d_R, ws, out)
+    torch.cuda.synchronize()
+    assert cache.device_status() == 0 and (cache.seq_len == n).all()
+    o = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(o).all()
+    tail_k, tail_v = torch.stack(new_k, dim=2), torch.stack(new_v, dim=2)         # [B, H, n_app, 128]
+    full = {key: (torch.cat([kc, tail_k[key[1]]], dim=1), torch.cat([vc, tail_v[key[1]]], dim=1)) for key, (kc, vc) in kept.items()}
+    mod_row = np.concatenate([mod_cpu.numpy(), np.zeros(n_app, np.uint8)])
+    _check_sampled(cache, w, samples, full, q, signs, R, mod_row, n, o, meta_format)
