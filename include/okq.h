@@ -252,6 +252,15 @@ okq_status okq_decode_attention_simt(const okq_cache* cache, int32_t layer, int3
 void okq_profile_events(void* before, void* after);
 
 /*
+ * Choice of the split-K kernel behind okq_decode_attention (the paper has no counterpart; for cross-checks and
+ * timing comparisons).  0 (default): the tcgen05 kernel with the unpacked codes in tensor memory; 1: the
+ * mma.sync warp-pair kernel.  Both fill the same partial records for the same combine kernel.  Process-wide;
+ * not to be changed while a decode call is being issued on another thread.  Returns the previous value;
+ * a value other than 0 or 1 changes nothing.
+ */
+int32_t okq_decode_select(int32_t impl);
+
+/*
  * Canonical view of one layer (checkpointing and parity checks; the paper has no
  * counterpart, the arrays are simply Eq. 2-4 and Eq. 6 outputs in natural order).
  * All windows up to capacity are converted, whatever seq_len says.

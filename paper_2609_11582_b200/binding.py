@@ -76,6 +76,8 @@ def lib():
         L.okq_decode_attention_noalloc.restype = C.c_int
         L.okq_decode_attention_noalloc.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32, C.c_void_p, C.c_float,
                                                    C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.okq_decode_select.restype = C.c_int32
+        L.okq_decode_select.argtypes = [C.c_int32]
         L.okq_profile_events.restype = None
         L.okq_profile_events.argtypes = [C.c_void_p, C.c_void_p]
         L.okq_cache_export.restype = C.c_int
@@ -102,7 +104,7 @@ def lib():
 def exported_symbols():
     return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
-            "okq_cache_import", "okq_profile_events", "okq_decode_attention_simt",
+            "okq_cache_import", "okq_profile_events", "okq_decode_select", "okq_decode_attention_simt",
             "okq_decode_attention_noalloc", "okq_quantize_values_bulk", "okq_cache_export_mx",
             "okq_calib_workspace_bytes", "okq_calib_attention_weights", "okq_calib_moments", "okq_calib_rotation"]
 
@@ -213,6 +215,11 @@ def decode_attention_noalloc(cache: Cache, layer: int, layer_count: int, q, sign
     _check(lib().okq_decode_attention_noalloc(C.byref(cache.c), layer, layer_count, _ptr(q), scale, _ptr(signs),
                                               _ptr(R), n_R, num_splits, _ptr(out), _stream(stream)),
            "okq_decode_attention_noalloc")
+
+
+def decode_select(impl: int) -> int:
+    """Choose the split-K kernel of later decode calls (0: tcgen05, 1: mma.sync warp pairs); returns the previous choice."""
+    return lib().okq_decode_select(impl)
 
 
 def profile_events(before=None, after=None):

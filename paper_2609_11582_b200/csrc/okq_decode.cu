@@ -454,6 +454,12 @@ void okq_profile_events(void* before, void* after) {
   g_ev_after = static_cast<cudaEvent_t>(after);
 }
 
+int32_t okq_decode_select(int32_t impl) {
+  const int32_t prev = g_decode_impl;
+  if (impl == 0 || impl == 1) g_decode_impl = impl;
+  return prev;
+}
+
 size_t okq_decode_workspace_bytes(const okq_cache* cache, int32_t layer_count, int32_t num_splits) {
   if (check_cache(cache, false) != OKQ_OK || layer_count <= 0 || num_splits < 0) return 0;
   size_t a = simt_workspace(cache, layer_count, num_splits), b = mma_workspace(cache, layer_count, num_splits);

@@ -1125,6 +1125,8 @@ static void combine_dispatch(const DecodeParams& P, int n_cta, cudaStream_t s) {
   else combine_launch<CAPTION, 1, CB_SEQ_MAX>(P, n_cta, s);
 }
 
+int g_decode_impl = 0;
+
 okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, cudaEvent_t before, cudaEvent_t after) {
   static thread_local unsigned long long attr_mask = 0;
   int attr_dev = 0;
@@ -1144,7 +1146,10 @@ okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, c
     attr_done(attr_mask, attr_dev);
   }
   if (before) cudaEventRecord(before, s);
-  if (P.cv.fmt == FMT_MXFP4) k_decode_mma<FMT_MXFP4><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_MXFP4>), s>>>(P);
+  if (P.cv.fmt == FMT_FP16 && g_decode_impl == 0) {
+    const okq_status st = launch_decode_tc(P, n_cta, s);
+    if (st != OKQ_OK) return st;
+  } else if (P.cv.fmt == FMT_MXFP4) k_decode_mma<FMT_MXFP4><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_MXFP4>), s>>>(P);
   else k_decode_mma<FMT_FP16><<<n_cta, NTHREADS, sizeof(MmaSmem<FMT_FP16>), s>>>(P);
   if (after) cudaEventRecord(after, s);
   if (P.cv.sched == SCHED_CAPTION) combine_dispatch<true>(P, n_cta, s);
