@@ -253,10 +253,10 @@ void okq_profile_events(void* before, void* after);
 
 /*
  * Choice of the split-K kernel behind okq_decode_attention (the paper has no counterpart; for cross-checks and
- * timing comparisons).  0 (default): the tcgen05 kernel with the unpacked codes in tensor memory; 1: the
- * mma.sync warp-pair kernel.  Both fill the same partial records for the same combine kernel.  Process-wide;
- * not to be changed while a decode call is being issued on another thread.  Returns the previous value;
- * a value other than 0 or 1 changes nothing.
+ * timing comparisons).  1 (default): the mma.sync warp-pair kernel; 0: the tcgen05 kernel with the unpacked codes
+ * in tensor memory (fp16 metadata only; a cache with MXFP4 metadata always takes the warp-pair kernel).  Both fill
+ * the same partial records for the same combine kernel.  Process-wide; not to be changed while a decode call is
+ * being issued on another thread.  Returns the previous value; a value other than 0 or 1 changes nothing.
  */
 int32_t okq_decode_select(int32_t impl);
 

@@ -218,7 +218,7 @@ def decode_attention_noalloc(cache: Cache, layer: int, layer_count: int, q, sign
 
 
 def decode_select(impl: int) -> int:
-    """Choose the split-K kernel of later decode calls (0: tcgen05, 1: mma.sync warp pairs); returns the previous choice."""
+    """Choose the split-K kernel of later decode calls (0: tcgen05, 1: mma.sync warp pairs, the default); returns the previous choice."""
     return lib().okq_decode_select(impl)
 
 

@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(128) k_decode_simt(DecodeParams P) {
       const uint32_t* kw = reinterpret_cast<const uint32_t*>(ws.rec + OFF_KCODE);
       int nu = lane >> 3, g = lane & 7;
       for (int t = 0; t < 4; t++) {
-        uint2 wd = *reinterpret_cast<const uint2*>(&kw[(nu >> 1) * 128 + (4 * g + t) * 4 + (nu & 1) * 2]);
+        uint2 wd = *reinterpret_cast<const uint2*>(&kw[kword_index((nu >> 1) * 128 + (4 * g + t) * 4 + (nu & 1) * 2)]);
 #pragma unroll
         for (int ww = 0; ww < 2; ww++) {
           uint32_t word = ww ? wd.y : wd.x;
@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(128) k_decode_simt(DecodeParams P) {
 #pragma unroll
       for (int musel = 0; musel < 2; musel++) {
         for (int t = 0; t < 4; t++) {
-          uint32_t word = vw[musel * 128 + (4 * gq + t) * 4 + aq];
+          uint32_t word = vw[vword_index(musel * 128 + (4 * gq + t) * 4 + aq)];
 #pragma unroll
           for (int qd = 0; qd < 8; qd++) {
             int sh = qd >> 2, jj = qd & 3;

@@ -97,8 +97,8 @@ __device__ __forceinline__ void window_scores_mma(const unsigned char* st, const
   for (int nu = 0; nu < 4; nu++)
 #pragma unroll
     for (int i = 0; i < 4; i++) d[nu][i] = 0.f;
-  const uint4 kc0 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * lane);
-  const uint4 kc1 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 512 + 16 * lane);
+  const uint4 kc0 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * kpiece_slot(lane));
+  const uint4 kc1 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * kpiece_slot(32 + lane));
   const uint32_t kw[4][2] = {{kc0.x, kc0.y}, {kc0.z, kc0.w}, {kc1.x, kc1.y}, {kc1.z, kc1.w}};
 #pragma unroll
   for (int kq = 0; kq < 4; kq++) {
@@ -196,8 +196,8 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
       for (int nu = 0; nu < 4; nu++)
 #pragma unroll
         for (int i = 0; i < 4; i++) d[nu][i] = 0.f;
-      const uint4 kc0 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * lane);
-      const uint4 kc1 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 512 + 16 * lane);
+      const uint4 kc0 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * kpiece_slot(lane));
+      const uint4 kc1 = *reinterpret_cast<const uint4*>(st + OFF_KCODE + 16 * kpiece_slot(32 + lane));
       const uint32_t kw[4][2] = {{kc0.x, kc0.y}, {kc0.z, kc0.w}, {kc1.x, kc1.y}, {kc1.z, kc1.w}};
 #pragma unroll
       for (int kq = 0; kq < 4; kq++) {
@@ -345,8 +345,8 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
                                  : ((__any_sync(0xffffffffu, mymod == 0) ? 1u : 0u) |
                                     (__any_sync(0xffffffffu, mymod == 1) ? 2u : 0u) |
                                     (__any_sync(0xffffffffu, mymod == 2) ? 4u : 0u));
-      const uint4 vc0 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 16 * lane);
-      const uint4 vc1 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 512 + 16 * lane);
+      const uint4 vc0 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 16 * vpiece_slot(lane));
+      const uint4 vc1 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 16 * vpiece_slot(32 + lane));
       const uint32_t vw[8] = {vc0.x, vc0.y, vc0.z, vc0.w, vc1.x, vc1.y, vc1.z, vc1.w};
       const uint4 pb4 = ho.pb[lane];
       const uint32_t pb[4] = {pb4.x, pb4.y, pb4.z, pb4.w};
@@ -1125,7 +1125,7 @@ static void combine_dispatch(const DecodeParams& P, int n_cta, cudaStream_t s) {
   else combine_launch<CAPTION, 1, CB_SEQ_MAX>(P, n_cta, s);
 }
 
-int g_decode_impl = 0;
+int g_decode_impl = 1;
 
 okq_status launch_decode_mma(const DecodeParams& P, int n_cta, cudaStream_t s, cudaEvent_t before, cudaEvent_t after) {
   static thread_local unsigned long long attr_mask = 0;

@@ -76,7 +76,7 @@ __device__ inline int block_prefix(const CacheView& cv, int layer0, int n_entrie
 
 // tcgen05 split-K kernel (fp16 metadata): fills partials_f exactly where launch_decode_mma's own split kernel would
 okq_status launch_decode_tc(const DecodeParams& P, int n_cta, cudaStream_t s);
-// which split-K kernel launch_decode_mma uses: 0 = default (tcgen05 where it applies), 1 = the mma.sync warp-pair kernel
+// which split-K kernel launch_decode_mma uses: 0 = the tcgen05 kernel (fp16 metadata), 1 = the mma.sync warp-pair kernel
 extern int g_decode_impl;
 
 // launches the tensor-core split kernel (bracketed by the optional events) and its combine kernel

@@ -55,6 +55,18 @@ __host__ __device__ inline int norm_pos(int i) {
   return 8 * t + 2 * nu + e;
 }
 
+// The 64 16-byte pieces of a code block are stored in an order that lets the tcgen05 decode kernel, whose threads
+// own one token (key codes) or one channel (value codes), read them from a staged copy without bank conflicts.
+// With the "fragment" piece index p = 32 a + 4 g + t (the order the mma.sync fragments above describe: piece p holds
+// the words 4 p .. 4 p + 3):
+//   key codes:   piece p sits at position 16 t + 2 g + a   (the 16 pieces of one t are contiguous)
+//   value codes: piece p sits at position 32 a + 8 t + g   (the 8 pieces of one (a, t) are contiguous)
+__host__ __device__ inline int kpiece_slot(int p) { return 16 * (p & 3) + 2 * ((p >> 2) & 7) + (p >> 5); }
+__host__ __device__ inline int vpiece_slot(int p) { return 32 * (p >> 5) + 8 * (p & 3) + ((p >> 2) & 7); }
+// stored position of fragment-order word w of the key / value code block
+__host__ __device__ inline int kword_index(int w) { return 4 * kpiece_slot(w >> 2) + (w & 3); }
+__host__ __device__ inline int vword_index(int w) { return 4 * vpiece_slot(w >> 2) + (w & 3); }
+
 // key code of (token i in window, channel c): 32-bit word index in the key-code block and bit offset
 __host__ __device__ inline void kcode_pos(int i, int c, int& word, int& bit) {
   int nu = i >> 3, g = i & 7;
@@ -62,7 +74,7 @@ __host__ __device__ inline void kcode_pos(int i, int c, int& word, int& bit) {
   int pair = slot >> 3, t = (slot & 7) >> 1, e = slot & 1;
   int r = 2 * kappa + pair;
   int ww = r >> 3, sh = (r >> 2) & 1, j = r & 3;
-  word = (nu >> 1) * 128 + (4 * g + t) * 4 + (nu & 1) * 2 + ww;
+  word = kword_index((nu >> 1) * 128 + (4 * g + t) * 4 + (nu & 1) * 2 + ww);
   bit = 16 * e + 8 * sh + 2 * j;
 }
 
@@ -71,7 +83,7 @@ __host__ __device__ inline void vcode_pos(int i, int c, int& word, int& bit) {
   int mu = c >> 4, sh = (c >> 3) & 1, g = c & 7;
   int kv = i >> 4, pv = (i >> 3) & 1, t = (i & 7) >> 1, e = i & 1;
   int j = 2 * kv + pv;
-  word = (mu >> 2) * 128 + (4 * g + t) * 4 + (mu & 3);
+  word = vword_index((mu >> 2) * 128 + (4 * g + t) * 4 + (mu & 3));
   bit = 16 * e + 8 * sh + 2 * j;
 }
 

@@ -243,7 +243,7 @@ __device__ void quantize_key_window(const __half* rows, long long stride, const 
       }
       word -= MAGIC_SUM;
       // word index of (token i, t, ww): [i >> 4][lane 4*(i & 7) + t][(i >> 3) & 1][ww]
-      words[(i >> 4) * 128 + (4 * (i & 7) + t) * 4 + ((i >> 3) & 1) * 2 + ww] = word;
+      words[kword_index((i >> 4) * 128 + (4 * (i & 7) + t) * 4 + ((i >> 3) & 1) * 2 + ww)] = word;
     }
   }
   __syncthreads();
@@ -326,7 +326,7 @@ __device__ void quantize_value_window(const __half* rows, long long stride, cons
         word |= (uint32_t)sm.code[i * D + c] << (16 * e + 8 * sh + 2 * j);
       }
     }
-    words[wi] = word;
+    words[vword_index(wi)] = word;
   }
   __syncthreads();
 }

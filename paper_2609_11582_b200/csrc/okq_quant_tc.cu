@@ -474,7 +474,7 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
         for (int t = 0; t < 4; t++) {
           const uint32_t own = wacc[t] << (8 * sh);
           const uint32_t full = own | __shfl_xor_sync(0xffffffffu, own, 8);
-          if ((t >> 1) == sh) words[(mu >> 2) * 128 + (4 * g + t) * 4 + (mu & 3)] = full;
+          if ((t >> 1) == sh) words[vword_index((mu >> 2) * 128 + (4 * g + t) * 4 + (mu & 3))] = full;
         }
       }
       __syncwarp();   // sm.c3[warp] is rewritten for the next tile
