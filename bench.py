@@ -251,6 +251,8 @@ def main():
     ap.add_argument("--impl", default="okq", choices=["okq", "reference"])
     ap.add_argument("--workload", default=None, choices=sorted(WL.WORKLOADS))
     ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--decode-kernel", default="default", choices=["default", "tcgen05", "mma"],
+                    help="split-K kernel behind okq_decode_attention (default: the library's choice)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling on a small case)")
     ap.add_argument("--meta", default="fp16", choices=["fp16", "mxfp4"],
@@ -274,6 +276,8 @@ def main():
         return run_reference(args, w)
 
     from paper_2609_11582_b200 import binding as B
+    if args.decode_kernel != "default":
+        B.decode_select(0 if args.decode_kernel == "tcgen05" else 1)
     rank, world, local = dist_env()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)

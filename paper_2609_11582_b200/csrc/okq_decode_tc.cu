@@ -118,13 +118,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t mbar, uint32_t parity) {
 // Up to 64 tries in a loop of two instructions (a try suspends the thread until the phase completes or a short,
 // system-chosen time has passed): a waiting warp must not take issue slots and ALU cycles from the working ones.
 __device__ __forceinline__ bool mbar_try64(uint32_t mbar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p, q;\n\t.reg .u32 cnt;\n\tmov.u32 cnt, 0;\n"
-               "WAIT_LOOP:\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t@p bra WAIT_DONE;\n\t"
-               "add.u32 cnt, cnt, 1;\n\tsetp.lt.u32 q, cnt, 64;\n\t@q bra WAIT_LOOP;\n"
-               "WAIT_DONE:\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-               : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
-  return ok != 0;
+  bool ok = false;
+#pragma unroll 1
+  for (int i = 0; i < 64 && !ok; i++) {
+    ok = mbar_try(mbar, parity);
+#ifdef OKQ_TC_SLEEP
+    if (!ok) __nanosleep(OKQ_TC_SLEEP);
+#endif
+  }
+  return ok;
 }
 // Bounded wait of a whole warp for one phase of an mbarrier; gives up after about two seconds or soon after another
 // role has given up, and raises the abort flag.  The clock and the flag are looked at every 64th try only.
@@ -290,7 +292,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
     const int q = warp - WARP_K;
     const int tp = lane >> 3, nu = (lane >> 1) & 3, ep = lane & 1;
     const int g = 2 * tp + ep;
-    const uint32_t koff = OFF_KCODE + 16 * (2 * g + (nu >> 1)) + 8 * (nu & 1);
+    uint32_t koff[4];   // the lane's 8-byte half of its piece (a = nu >> 1, g, t), t = 0..3
+#pragma unroll
+    for (int t = 0; t < 4; t++) koff[t] = OFF_KCODE + 16 * kpiece_slot(32 * (nu >> 1) + 4 * g + t) + 8 * (nu & 1);
     SegWalk walk = walker();
     Seg sg;
     int n = 0;
@@ -304,9 +308,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
         if (q == 0) TL(1, n, 0);
         uint2 w[4];
         if (q < n_w) {
-          const unsigned char* base = sm.stage[st] + q * STG_WIN + koff;
+          const unsigned char* base = sm.stage[st] + q * STG_WIN;
 #pragma unroll
-          for (int t = 0; t < 4; t++) w[t] = *reinterpret_cast<const uint2*>(base + 256 * t);
+          for (int t = 0; t < 4; t++) w[t] = *reinterpret_cast<const uint2*>(base + koff[t]);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.stage_free[st]);   // the code words are in registers
@@ -386,7 +390,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
           if (t == 0) sm.bias[nb][wq][g] = ((dbA[0] + dbB[0]) + (dbA[2] + dbB[2])) * 0x1p-24f;
           if (wq == 0 && t == 0) sm.fsc[nb][g] = fsc;
         }
+        if (wq == 0) TL(2, n, 2);
         fence_async_smem();
+        if (wq == 0) TL(2, n, 3);
         __syncwarp();
         if (lane == 0) { mbar_arrive(&sm.bw_full[buf]); mbar_arrive(&sm.stage_free[st]); }
         if (wq == 0) TL(2, n, 1);
@@ -543,7 +549,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
         if (valid) {
           const int xw = x0 + wq, slot = xw % NAV, use = xw / NAV;
           if (wq == 0 && hh == 0) TL(4, n, 4);
+#ifndef OKQ_TC_ABLATE_VALUES
           if (use >= 1 && !mbar_wait(sm, &sm.v_done[slot], (uint32_t)(use - 1) & 1u)) { alive = false; break; }
+#endif
           if (wq == 0 && hh == 0) TL(4, n, 5);
           const float vn = __half2float(reinterpret_cast<const __half*>(swin + OFF_VNORM)[lane]);
           int mod = sm.stage[st][STG_MOD + W * wq + tok];
@@ -595,6 +603,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
           }
           touched |= (int)present;
           if (hh == 0 && lane == 0) { sm.bp_present[slot] = (int)present; sm.bp_flush[slot] = (wq == 0 && flag) ? 1 : 0; }
+          if (wq == 0 && hh == 0) TL(4, n, 7);
           fence_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive(&sm.bp_full[slot]);
@@ -651,7 +660,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
     // 32; its words are word (mu & 3) of the pieces (A = mu >> 2, g, t)
     const int vq = (warp - WARP_V) & 3, vpar = (warp - WARP_V) >> 2;
     const int sh = (lane >> 3) & 1, g = lane & 7;
-    const uint32_t voff = OFF_VCODE + 16 * (32 * (vq >> 1) + g) + 4 * (2 * (vq & 1) + (lane >> 4));
+    uint32_t voff[4];   // word (mu & 3) of the lane's piece (A = vq >> 1, g, t), t = 0..3
+#pragma unroll
+    for (int t = 0; t < 4; t++) voff[t] = OFF_VCODE + 16 * vpiece_slot(32 * (vq >> 1) + 4 * g + t) + 4 * (2 * (vq & 1) + (lane >> 4));
     SegWalk walk = walker();
     Seg sg;
     int n = 0, xw = 0;
@@ -665,12 +676,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
         if (!mbar_wait(sm, &sm.stage_full[st], (uint32_t)(n / NST) & 1u)) { alive = false; break; }
         if (vq == 0 && vpar == 0) TL(5, n, 0);
         for (int j = 0; j < n_w; j++, xw++) {
+#ifdef OKQ_TC_ABLATE_VALUES
+          continue;
+#endif
           if ((xw & 1) != vpar) continue;
           const int slot = xw % NAV, use = xw / NAV;
-          const unsigned char* base = sm.stage[st] + j * STG_WIN + voff;
+          const unsigned char* base = sm.stage[st] + j * STG_WIN;
           uint32_t wd[4];
 #pragma unroll
-          for (int t = 0; t < 4; t++) wd[t] = *reinterpret_cast<const uint32_t*>(base + 128 * t) >> (8 * sh);
+          for (int t = 0; t < 4; t++) wd[t] = *reinterpret_cast<const uint32_t*>(base + voff[t]) >> (8 * sh);
           // word t, field jj: tokens with K index 8 t + 2 jj + {0, 1}; columns 4 t + jj (code plane), 16 + 4 t + jj (bit 1)
           uint32_t r[32];
 #pragma unroll
@@ -713,6 +727,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
     int xw = 0, f = 0;
     unsigned acc_valid = 0;
     bool alive = true;
+#ifdef OKQ_TC_ABLATE_VALUES
+    alive = false;
+#endif
     while (alive && walk.next(sg)) {
       for (int j = 0; j < sg.n_my; j++, xw++) {
         const int slot = xw % NAV;
@@ -788,6 +805,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) k_decode_tc(DecodeParams P) {
       while (walk.next(sg)) n_seg++;
     }
     int k = 0, seg_done = 0;
+#ifdef OKQ_TC_ABLATE_VALUES
+    n_seg = 0;
+#endif
     while (seg_done < n_seg) {
       if (!mbar_wait(sm, &sm.req_full[k % NREQ], (uint32_t)(k / NREQ) & 1u) || !mbar_wait(sm, &sm.flush_ready, (uint32_t)k & 1u)) break;
       fence_after();

@@ -55,14 +55,24 @@ __host__ __device__ inline int norm_pos(int i) {
   return 8 * t + 2 * nu + e;
 }
 
-// The 64 16-byte pieces of a code block are stored in an order that lets the tcgen05 decode kernel, whose threads
-// own one token (key codes) or one channel (value codes), read them from a staged copy without bank conflicts.
-// With the "fragment" piece index p = 32 a + 4 g + t (the order the mma.sync fragments above describe: piece p holds
-// the words 4 p .. 4 p + 3):
-//   key codes:   piece p sits at position 16 t + 2 g + a   (the 16 pieces of one t are contiguous)
-//   value codes: piece p sits at position 32 a + 8 t + g   (the 8 pieces of one (a, t) are contiguous)
-__host__ __device__ inline int kpiece_slot(int p) { return 16 * (p & 3) + 2 * ((p >> 2) & 7) + (p >> 5); }
-__host__ __device__ inline int vpiece_slot(int p) { return 32 * (p >> 5) + 8 * (p & 3) + ((p >> 2) & 7); }
+// The 64 16-byte pieces of a code block are stored in an order that lets both decode kernels read a staged copy
+// without bank conflicts: the mma.sync kernel, whose lane l reads the "fragment" pieces l and 32 + l, and the tcgen05
+// kernel, whose threads own one token (key codes) or one channel (value codes).  With the fragment piece index
+// p = 32 a + 4 g + t (the order the mma.sync fragments above describe: piece p holds the words 4 p .. 4 p + 3) and
+// g = 4 g2 + 2 g1 + g0, a piece sits at position 8 * row + column with
+//   key codes:   row = 2 t + g2,  column = (t + 4 g0 + 2 g1 + a)  mod 8
+//   value codes: row = 4 a + t,   column = (t + 4 g0 + 2 g1 + g2) mod 8
+// Eight pieces read together always fall into the eight different 16-byte columns of the 128-byte bank line:
+// the pieces (g0, t) of one quarter-warp of the mma.sync kernel; the pieces (a, g0, g1) that the 16 token-threads of
+// a half-warp read for one t; the pieces g = 0..7 that a warp of channel-threads reads for one (a, t).
+__host__ __device__ inline int kpiece_slot(int p) {
+  const int t = p & 3, g = (p >> 2) & 7, a = p >> 5;
+  return 8 * (2 * t + (g >> 2)) + ((t + 4 * (g & 1) + 2 * ((g >> 1) & 1) + a) & 7);
+}
+__host__ __device__ inline int vpiece_slot(int p) {
+  const int t = p & 3, g = (p >> 2) & 7, a = p >> 5;
+  return 8 * (4 * a + t) + ((t + 4 * (g & 1) + 2 * ((g >> 1) & 1) + (g >> 2)) & 7);
+}
 // stored position of fragment-order word w of the key / value code block
 __host__ __device__ inline int kword_index(int w) { return 4 * kpiece_slot(w >> 2) + (w & 3); }
 __host__ __device__ inline int vword_index(int w) { return 4 * vpiece_slot(w >> 2) + (w & 3); }
