@@ -32,10 +32,11 @@ sys.path.insert(0, ROOT)
 from paper_2609_11582_b200 import workloads as WL  # noqa: E402
 
 METRIC = "2-bit KV decode-attention effective HBM GB/s (packed-KV bytes per decode step / step time)"
+W_TOKENS = 32                      # tokens per window: one step in 32 packs a window ("flush")
 BYTES_PER_TOKEN_HEAD = 84          # 32 B key codes + 2 B key norm + 16 B (m, s) + 32 B value codes + 2 B value norm
 # dram__bytes_read.sum + dram__bytes_write.sum of one split-K decode launch, measured with ncu on a
 # 4-layer slice of the workload (176 MB of records, larger than L2) and divided by its token-heads;
-# traffic grows in proportion to the token-heads (profiles/decode_mma_layers4_ncu_full.md).
+# traffic grows in proportion to the token-heads.  To be re-measured whenever the split-K kernel changes.
 NCU_DRAM_BYTES_PER_TOKEN_HEAD = 86.80
 NCU_DRAM_BYTES_PER_TOKEN_HEAD_MX = 75.11   # same capture with --meta mxfp4
 
@@ -159,9 +160,9 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def run_prefill(args, w, B, dev, rank):
+def run_prefill(args, w, B, dev, rank, emit=True):
     """Secondary measurement: bulk okq_quantize_keys + okq_quantize_values_bulk over a fresh fp16 K/V cache of
-    every layer (the prefill half of the long-context configuration).  One JSON line."""
+    every layer (the prefill half of the long-context configuration).  One JSON line (or, emit=False, the dict)."""
     L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
     cache = B.Cache(L, Bn, H, Hq, N, device=dev)
     mod = WL.modality_layout(w).unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
@@ -198,8 +199,61 @@ def run_prefill(args, w, B, dev, rank):
             "roofline": {"bound": "hbm", "kernel": "key + value quantisers", "achieved": (in_bytes + out_bytes) / (ms * 1e-3) / 1e9,
                          "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                          "frac": (in_bytes + out_bytes) / (ms * 1e-3) / 1e9 / peak, "traffic": None}}
+    del kv, cache
+    if not emit:
+        return line
     if rank == 0:
         print(json.dumps(line), flush=True)
+
+
+def quick_decode(B, dev, w, mx=False, caption=False, steps=8, warmup=3):
+    """Short secondary measurement of the decode step (append + decode over all layers, inputs resident) on another
+    workload / metadata format / schedule: step time, GB/s of packed bytes, split-K kernel time and fraction."""
+    L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
+    bytes_th = 72.25 if mx else BYTES_PER_TOKEN_HEAD
+    cache = B.Cache(L, Bn, H, Hq, N + 64, device=dev, meta_format=B.META_MXFP4 if mx else B.META_FP16,
+                    schedule=B.SCHEDULE_CAPTION if caption else B.SCHEDULE_WINDOW)
+    mod = WL.modality_layout(w).unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
+    signs = torch.stack([WL.gen_signs(w, l) for l in range(L)]).to(dev)
+    R = torch.stack([WL.gen_rotations(w, l) for l in range(L)]).unsqueeze(1).contiguous().to(dev)
+    for l in range(L):
+        k, v = WL.gen_kv(w, l, device=dev)
+        B.quantize_keys(cache, l, k, signs[l])
+        B.quantize_values(cache, l, v, mod, R[l], bulk=True)
+        del k, v
+    torch.cuda.synchronize()
+    seq0 = cache.seq_len.clone()
+    q = torch.stack([WL.gen_queries(w, l) for l in range(L)]).to(dev)
+    kn, vn, mn = WL.gen_new_token(w, 0, 0, device=dev)
+    kn = kn.unsqueeze(0).expand(L, -1, -1, -1).contiguous(); vn = vn.unsqueeze(0).expand(L, -1, -1, -1).contiguous()
+    out = torch.empty(L, Bn, Hq, 128, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(16, B.decode_workspace_bytes(cache, L, 0)), dtype=torch.uint8, device=dev)
+
+    def step():
+        B.append(cache, 0, L, kn, vn, mn, signs, R)
+        B.decode_attention(cache, 0, L, q, signs, R, ws, out)
+    for _ in range(warmup):
+        step()
+    cache.seq_len.copy_(seq0)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in kev:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    for i in range(steps):
+        B.profile_events(*kev[i])
+        ev[i][0].record(); step(); ev[i][1].record()
+    torch.cuda.synchronize()
+    B.profile_events(None, None)
+    if cache.device_status() != 0 or not torch.isfinite(out).all():
+        raise RuntimeError("secondary decode measurement: bad device status or non-finite output")
+    ms = sum(a.elapsed_time(b) for a, b in ev) / steps
+    kms = sum(a.elapsed_time(b) for a, b in kev) / steps
+    packed = L * Bn * H * N * bytes_th
+    peak, _ = measured_peaks()
+    return {"workload": w.name, "meta_format": "mxfp4" if mx else "fp16", "schedule": "caption" if caption else "window",
+            "steps": steps, "us_per_step": ms * 1e3, "value": packed / (ms * 1e-3) / 1e9, "unit": "GB/s",
+            "kernel_us": kms * 1e3, "kernel_gbs": packed / (kms * 1e-3) / 1e9, "kernel_frac": packed / (kms * 1e-3) / 1e9 / peak}
 
 
 def run_calib(args, B, dev, rank):
@@ -254,6 +308,7 @@ def main():
     ap.add_argument("--decode-kernel", default="default", choices=["default", "tcgen05", "mma"],
                     help="split-K kernel behind okq_decode_attention (default: the library's choice)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the short secondary measurements of the default run")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling on a small case)")
     ap.add_argument("--meta", default="fp16", choices=["fp16", "mxfp4"],
                     help="(m, s) metadata format of the cache: fp16 = 84 B per token and KV head (the headline "
@@ -374,7 +429,7 @@ def main():
     def timed_e2e():
         cache.seq_len.copy_(seq0)
         run_e2e(0, args.warmup)
-        cache.seq_len.copy_(seq0)
+        prime()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         a.record()
@@ -398,11 +453,20 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # The timed steps end on a 32-token boundary, so that whatever --steps is they contain a step that packs a
+    # window (one per 32 steps): `pre` untimed appends put the raw tokens of the earlier steps of the cycle in place.
+    pre = (-args.steps) % W_TOKENS
+
+    def prime():
+        cache.seq_len.copy_(seq0)
+        for _ in range(pre):
+            B.append(cache, 0, L, kn_dev[0], vn_dev[0], mn_dev, signs, R)
+
     def timed(step_fn, with_kernel_events):
         cache.seq_len.copy_(seq0)
         for s in range(args.warmup):
             step_fn(s)
-        cache.seq_len.copy_(seq0)       # the timed steps start from the same context length
+        prime()                          # the timed steps always start from the same context length
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
         kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
         for a, b in kev:      # torch creates the CUDA event on first record; the library re-records it later
@@ -419,8 +483,13 @@ def main():
         barrier()
         B.profile_events(None, None)
         clocks = sampler.stop()
-        ms = sum(a.elapsed_time(b) for a, b in ev)
+        per_step = [a.elapsed_time(b) for a, b in ev]
+        ms = sum(per_step)
         kms = sum(a.elapsed_time(b) for a, b in kev) / args.steps if with_kernel_events else None
+        flush = [t for i, t in enumerate(per_step) if (pre + i + 1) % W_TOKENS == 0]
+        tail = [t for i, t in enumerate(per_step) if (pre + i + 1) % W_TOKENS != 0]
+        step_kinds.update(flush_steps=len(flush), us_per_flush_step=1e3 * sum(flush) / max(1, len(flush)),
+                          tail_steps=len(tail), us_per_tail_step=1e3 * sum(tail) / max(1, len(tail)) if tail else None)
         if world > 1:
             import torch.distributed as dist
             t = torch.tensor([ms], device=dev)
@@ -428,6 +497,7 @@ def main():
             ms = float(t.item())
         return ms, kms, clocks
 
+    step_kinds = {}
     ms_total, kernel_ms, clocks = timed(step_resident, True)
     if cache.device_status() != 0:
         raise RuntimeError("device status word set during the benchmark")
@@ -456,7 +526,7 @@ def main():
         cache.seq_len.copy_(seq0)
         for _ in range(args.warmup):
             g.replay()
-        cache.seq_len.copy_(seq0)
+        prime()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         a.record()
@@ -473,6 +543,27 @@ def main():
 
     if rank != 0:
         return
+    # Secondary measurements (short runs; the headline numbers above are not affected): the paper's default MXFP4
+    # metadata, its captioning schedule, the prefill quantisers, and the split-K kernel on the other decode shapes.
+    secondary = None
+    if world == 1 and not args.no_secondary and not mx and not caption and args.workload == "step7b" and args.layers == 0:
+        del cache, ws, out, in_buf, out_buf
+        torch.cuda.empty_cache()
+        secondary = {}
+        for name, fn in (("mxfp4", lambda: quick_decode(B, dev, w, mx=True)),
+                         ("caption", lambda: quick_decode(B, dev, w, caption=True)),
+                         ("long7b", lambda: quick_decode(B, dev, WL.WORKLOADS["long7b"])),
+                         ("step30b", lambda: quick_decode(B, dev, WL.WORKLOADS["step30b"], steps=4, warmup=2)),
+                         ("prefill", lambda: run_prefill(argparse.Namespace(steps=3, warmup=1), WL.WORKLOADS["prefill7b"], B, dev, 0, emit=False))):
+            try:
+                r = fn()
+                if name == "prefill":
+                    r = {k: r[k] for k in ("value", "unit", "ms_per_step", "keys_ms", "values_bulk_ms", "keys_gbs", "values_bulk_gbs",
+                                           "values_bulk_tflops")} | {"frac": r["roofline"]["frac"], "workload": "prefill7b"}
+                secondary[name] = r
+            except Exception as e:          # a secondary number must never cost the headline line
+                secondary[name] = {"error": repr(e)[:200]}
+            torch.cuda.empty_cache()
     cpu = None
     if world == 1 and not args.no_cpu_baseline and not mx and not caption:
         n_l, n_s = min(4, L), min(8, Bn)
@@ -485,13 +576,16 @@ def main():
                "seconds_per_sample_pass": t}
     line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16-mma/f32-acc (decode), f32 (append quantisers)", "data": "synthetic",
             "config": {"workload": w.name, "n_layers": L, "batch": Bn, "n_q_heads": Hq, "n_kv_heads": H, "context": N,
                        "meta_format": args.meta, "bytes_per_token_head": bytes_th, "schedule": args.schedule,
                        "step": "okq_append(1 text token/seq, all layers) + okq_decode_attention(all layers), one call each",
+                       "timed_window": f"{args.steps} consecutive steps ending on a 32-token boundary: "
+                                       f"{step_kinds.get('flush_steps')} of them pack a window",
+                       "decode_kernel": args.decode_kernel,
                        "packed_kv_bytes_per_step": packed_bytes, "l2": f"inputs ({packed_bytes / 1e9:.2f} GB of records per step) exceed L2",
                        "parallelism": "replicas only" if world > 1 else "1 gpu"},
-            "clocks": clocks,
+            "clocks": clocks, "step_kinds": step_kinds,
             "e2e": {"value": e2e_value, "unit": "GB/s", "ms_per_step": ms_e2e / args.steps,
                     "h2d_bytes_per_step": q_host.numel() * 2 + kn_host[0].numel() * 2 + vn_host[0].numel() * 2 + Bn,
                     "d2h_bytes_per_step": out_host.numel() * 4,
@@ -506,7 +600,7 @@ def main():
                          "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                          "frac": achieved / peak, "frac_of_8TBs_nominal": achieved / 8000.0,
                          "kernel_ms": kernel_ms, "traffic": traffic},
-            "cpu_baseline": cpu}
+            "cpu_baseline": cpu, "secondary": secondary}
     print(json.dumps(line), flush=True)
 
 

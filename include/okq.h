@@ -1,9 +1,11 @@
 /*
  * okq — 2-bit KV-cache quantisation and fused decode attention (OmniKVQuant hot path)
  * for NVIDIA B200 (sm_100a).  Plain C ABI: device pointers, sizes, a CUDA stream passed
- * as void*.  The library allocates no device memory, keeps no global state (other than
- * the per-thread record of the last CUDA error), launches asynchronously on the given
- * stream and never aborts the process.
+ * as void*.  The library allocates no device memory, launches asynchronously on the given
+ * stream and never aborts the process.  Its only state: the per-thread record of the last
+ * CUDA error and of the profiling events (okq_profile_events), the process-wide choice of
+ * the split-K kernel (okq_decode_select), and the fixed device array behind
+ * okq_decode_attention_noalloc with the per-device cache of its address.
  *
  * Conventions
  *   - Every pointer inside okq_cache and every tensor argument is a DEVICE pointer owned
@@ -67,7 +69,8 @@ typedef enum {
   OKQ_ERR_CAPACITY = 4,    /* a sequence would exceed `capacity` (also the device status value) */
   OKQ_ERR_WORKSPACE = 5,   /* decode workspace smaller than okq_decode_workspace_bytes() */
   OKQ_ERR_CUDA = 6,        /* a CUDA runtime call failed; see okq_last_cuda_error() */
-  OKQ_ERR_TIMEOUT = 7      /* reserved: a bounded device-side wait gave up */
+  OKQ_ERR_TIMEOUT = 7      /* device status value: a bounded device-side wait (an mbarrier of the tensor-core
+                              pipelines) gave up; the kernel returned by itself, its results are invalid */
 } okq_status;
 
 /* Static, NUL-terminated description of a status value. */
@@ -211,7 +214,8 @@ okq_status okq_decode_attention(const okq_cache* cache, int32_t layer, int32_t l
  * cudaMalloc, no cudaFree, no allocating library routine.
  *
  *   - Arguments are those of okq_decode_attention without workspace / workspace_bytes.
- *   - Limit: okq_decode_workspace_bytes(cache, layer_count, num_splits) of the largest launch, i.e.
+ *   - Limit: the tensor-core path's scratch of the largest launch (this is not okq_decode_workspace_bytes(),
+ *     which also covers okq_decode_attention_simt and can be larger when num_splits is given), i.e.
  *     (layer_count * batch * n_kv_heads + number of CTAs) * 12736 bytes of per-CTA partials plus
  *     (layer_count * batch * n_kv_heads + 8 * number of CTAs) * 12832 bytes of per-warp-pair pieces,
  *     must fit in the scratch: about 1950 (sequence, KV head) pairs per launch with the automatic grid;

@@ -210,7 +210,7 @@ def decode_attention(cache: Cache, layer: int, layer_count: int, q, signs, R, wo
 def decode_attention_noalloc(cache: Cache, layer: int, layer_count: int, q, signs, R, out, n_R=1, sm_scale=None,
                              num_splits=0, stream=None):
     """okq_decode_attention_noalloc: same result as decode_attention, scratch held inside the library
-    (32 MiB per GPU, shared by all calls on that GPU; overlapping calls race).  Allocates nothing."""
+    (64 MiB per GPU, shared by all calls on that GPU; overlapping calls race).  Allocates nothing."""
     scale = HEAD_DIM ** -0.5 if sm_scale is None else sm_scale
     _check(lib().okq_decode_attention_noalloc(C.byref(cache.c), layer, layer_count, _ptr(q), scale, _ptr(signs),
                                               _ptr(R), n_R, num_splits, _ptr(out), _stream(stream)),

@@ -55,3 +55,23 @@ def test_noalloc_matches_decode_attention_twice_in_a_row():
         refs = [case.oracle_attention(l)[0] for l in range(2)]
         want = case.gpu_decode(0, layer_count=2)
     assert cache.device_status() == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("meta_format,num_splits", [(B.META_MXFP4, 0), (B.META_FP16, 3), (B.META_MXFP4, 5)])
+def test_noalloc_other_formats_and_grids(meta_format, num_splits):
+    """The same comparison with MXFP4 metadata and with a caller-chosen number of CTAs per (sequence, head): both reuse
+    the library's scratch with a different partition of it.  Twice in a row, against the caller-owned-workspace call."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=3, n_layers=2)
+    case = Hn.Case(w, n_tokens=512 + 9, meta_format=meta_format)
+    cache, dev = case.cache, case.cache.device
+    for call in range(2):
+        want = case.gpu_decode(0, layer_count=2, num_splits=num_splits)
+        out = torch.full((2, w.batch, w.n_q_heads, D), float("nan"), dtype=torch.float32, device=dev)
+        B.decode_attention_noalloc(cache, 0, 2, case.d_q, case.d_signs, case.d_R, out, num_splits=num_splits)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy().astype(np.float64)
+        rel, worst, mx = Hn.attention_errors(got, want)
+        assert rel < Hn.REL_L2_TOL and worst < Hn.REL_L2_TOL and mx < Hn.MAX_ABS_TOL, (call, rel, worst, mx)
+        case.d_q = torch.flip(case.d_q, dims=[2]).contiguous()
+    assert cache.device_status() == 0
