@@ -153,9 +153,9 @@ okq_status okq_quantize_values(const okq_cache* cache, int32_t layer, const void
  * Bulk (prefill) form of okq_quantize_values with the rotation z = R_m v on the tensor cores
  * (Eq. 6 as a dense [tokens x 128] x [128 x 128] product per modality; tcgen05.mma with R split
  * into two fp16 matrices and fp32 accumulation in tensor memory).  Same arguments, same stored
- * norms (bit-identical).  A code can differ from okq_quantize_values, by one level, only where
- * the rotated coordinate lies within about 1e-7 of a codebook threshold: both results are valid
- * nearest-level choices at fp32 accuracy.  If the tensor-core pipeline does not answer within a
+ * norms and the same stored codes, bit for bit: a coordinate that the tensor-core product leaves
+ * within 2^-18 of a codebook threshold is recomputed with the fused-multiply-add chain of
+ * okq_quantize_values before its code is taken.  If the tensor-core pipeline does not answer within a
  * bounded wait the device status word becomes OKQ_ERR_TIMEOUT and the remaining tiles are
  * skipped.
  */

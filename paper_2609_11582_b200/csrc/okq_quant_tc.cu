@@ -21,10 +21,12 @@
 //     of a word).  The code, the number of thresholds {-T, 0, T} below z / norm, is taken
 //     arithmetically: v = sat(2/3 - z / (3 T norm)), k = floor(3 v) with a round-down fused
 //     multiply-add against 1.5 * 2^23, code = 3 - k: three full-rate instructions per element.
-// The split leaves a relative error of about 2^-22 on z and the arithmetic code a few 1e-8 on the
-// position of a threshold, so a code can differ from the exact path only when z / norm lies within
-// ~1e-7 of a threshold.  Norms are computed with the exact summation tree and are bit-identical to
-// the exact path.
+// The split leaves a relative error of about 2^-22 on z and the tensor cores' accumulation about
+// 1e-6, so the arithmetic code is only trusted where z / norm is further than 2^-18 from every
+// threshold (the code is taken twice, with the coordinate moved down and up by that band); the few
+// coordinates in the band (about 1e-4 of them) are listed and recomputed at the end of the kernel, one per warp at
+// a time, with the exact fused-multiply-add chain of the reference arithmetic over the value row, read again from
+// global memory; the code in the record is then patched.  Codes and norms (exact summation tree) are therefore bit-identical to the exact path.
 //
 // Every wait on an mbarrier is bounded; on a timeout the kernel records OKQ_ERR_TIMEOUT in the
 // cache's status word, stops issuing work, frees its tensor memory and returns.
@@ -43,6 +45,11 @@ constexpr int NT_ALL = NT + 64;           // + the MMA warp (16) and the loader 
 constexpr int TILE_BYTES = TILE * D * 2;  // 32 KB: one fp16 operand tile
 constexpr float NEG_INV_3T = -1.0f / (3.0f * CB_THRESH);
 constexpr float TWO_THIRDS = 2.0f / 3.0f;          // rounds up: a zero coordinate gives floor(3 v) = 2, code 1
+// The code is taken twice, with the coordinate moved down and up by BAND (in units of z / norm: far above the
+// rounding noise of the tensor-core product, about 1e-6); where the two disagree the coordinate lies that close to a
+// threshold and is recomputed with the exact fused-multiply-add chain of the reference arithmetic.
+constexpr float BAND = 0x1p-18f;
+constexpr float BAND_V = BAND / (3.0f * CB_THRESH);
 constexpr float FLOOR_MAGIC = 12582912.0f;         // 1.5 * 2^23: unit in the last place 1, bits 0x4B400000
 // sum over the eight fields (bit 16*e + 2*j) of a word of the magic bits shifted to the field, modulo 2^32
 constexpr uint32_t magic_sum() {
@@ -54,11 +61,24 @@ constexpr uint32_t magic_sum() {
 constexpr uint32_t MAGIC_SUM = magic_sum();
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000ll;   // about two seconds of SM clocks
 
+// A coordinate too close to a threshold for the tensor-core product to decide: recomputed with the reference
+// arithmetic at the end of the kernel (its code is patched in the record), so that the tile pipeline never waits for
+// the two rows this needs from global memory.
+struct FixItem {
+  uint32_t* word;        // code word of the record
+  const __half* xrow;    // the token's value row (128 fp16)
+  const float* rrow;     // row of the rotation matrix (128 fp32): output channel of the coordinate
+  float inv;             // 1 / norm
+  int bit;               // bit position of the 2-bit field in the word
+};
+constexpr int FIX_MAX = 256;
+
 struct TcSmem {
   __align__(1024) unsigned char a[2][TILE_BYTES];      // value tiles (double buffered)
   __align__(1024) unsigned char b[2][2][TILE_BYTES];   // two resident matrices, each as R_hi, R_lo
   __align__(16) float part[2][4][TILE];                // per token: sum of squares of channels [32 q, 32 q + 32)
   __align__(16) float c3[16][W];                       // per worker warp: -1 / (3 T norm) of its window's tokens
+  __align__(16) float inv[16][W];                      // per worker warp: 1 / norm of its window's tokens (0 for a zero vector)
   __align__(4) unsigned char mod[2][TILE];             // modality per token of a tile (255 = no token)
   __align__(8) unsigned long long full[2];             // 1 arrival + 32 KB of TMA bytes: tile and modality bytes are in
   __align__(8) unsigned long long empty[2];            // 16 arrivals: every worker warp is done with the buffer
@@ -67,10 +87,18 @@ struct TcSmem {
   __align__(8) unsigned long long part_ready[2];       // 16 arrivals: every worker warp has written its partial norms
   __align__(8) unsigned long long slot_ready;          // 16 arrivals: every worker warp has written its share of a rotation matrix
   uint32_t tmem_slot;
+  FixItem fix[FIX_MAX];
+  int fix_count;
   volatile int abort;                                  // set by a role whose bounded wait ran out
+  volatile int tmem_busy;                              // set if products may still be in flight at the end (tensor memory is then not released)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile("{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\telect.sync rx|px, 0xffffffff;\n\tselp.u32 %0, 1, 0, px;\n\t}\n" : "=r"(pred));
+  return pred != 0;
+}
 
 // shared-memory matrix descriptor: no swizzle, K-major; core matrices of 8 rows x 16 bytes,
 // `lbo` bytes between the two 8-element K chunks of one MMA, `sbo` bytes between 8-row groups
@@ -113,6 +141,20 @@ __device__ __forceinline__ bool mbar_wait(TcSmem& sm, unsigned long long* bar, u
   }
   if (!done) sm.abort = 1;
   return __all_sync(0xffffffffu, done);   // called by whole warps: one answer per warp
+}
+// After a timeout: wait, again with a limit and whatever the abort flag says, for a phase that this warp's own
+// asynchronous work (bulk copies, tensor-core products) will complete.  Returns false if it did not.
+__device__ __forceinline__ bool mbar_drain(unsigned long long* bar, uint32_t parity) {
+  const uint32_t mbar = smem_u32(bar);
+  bool done = false;
+  const long long t0 = clock64();
+  while (!done && clock64() - t0 < WAIT_LIMIT_CLOCKS / 8) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                 : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+    done = ok != 0;
+  }
+  return __all_sync(0xffffffffu, done);
 }
 __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
@@ -183,7 +225,9 @@ struct Slots {
 // (one accumulator of 128 columns each); jobs alternate between two accumulator sets in tensor memory.
 __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_constant__ CUtensorMap vmap, CacheView cv, int layer,
                                                              const unsigned char* __restrict__ modality, int n_tokens,
-                                                             int n_win, const float* __restrict__ R, int n_R) {
+                                                             int n_win, const float* __restrict__ R, int n_R,
+                                                             const __half* __restrict__ vrows, long long vs_b, long long vs_h,
+                                                             long long vs_t) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   TcSmem& sm = *reinterpret_cast<TcSmem*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -204,6 +248,8 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
     }
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 16;\n" ::"r"(smem_u32(&sm.slot_ready)));
     sm.abort = 0;
+    sm.tmem_busy = 0;
+    sm.fix_count = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (warp == 0) {
@@ -248,6 +294,7 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
       return packed;
     };
     uint32_t mod_cur = fetch_mod(0);
+    int armed = 0;   // tiles whose copies have been issued
     for (int i = 0; i < my_tiles; i++) {
       const int buf = i & 1, fill = i >> 1;
       if (fill >= 1 && !mbar_wait(sm, &sm.empty[buf], (uint32_t)(fill - 1) & 1u)) break;
@@ -264,9 +311,13 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
                        ::"r"(smem_u32(sm.a[buf]) + half * (TILE_BYTES / 2)), "l"(reinterpret_cast<uint64_t>(&vmap)),
                          "r"(64 * half), "r"(cwin0 * W), "r"(ch), "r"(cb), "r"(bar) : "memory");
       }
+      armed = i + 1;
       step_coords();
       mod_cur = fetch_mod(i + 1);
     }
+    // after a timeout somewhere: no copy of this warp may still be landing when the block ends
+    if (sm.abort)
+      for (int i = max(0, armed - 2); i < armed; i++) mbar_drain(&sm.full[i & 1], (uint32_t)(i >> 1) & 1u);
   } else if (warp == 16) {
     // ------------------------------------------------------------------ MMA warp
     Slots slots;
@@ -290,7 +341,7 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
           if (!mbar_wait(sm, &sm.slot_ready, refills & 1u)) { dead = true; break; }
           refills++;
         }
-        if (lane == 0) {
+        if (elect_one()) {   // one thread of the converged warp: the compiler keeps the operands in uniform registers
           asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // the landed copies -> tensor-core reads
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           for (int mi = 0; mi < nm; mi++) {
@@ -321,8 +372,10 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
       }
       step_coords();
     }
-    // nothing may be in flight when tensor memory is released
-    if (jobidx >= 1) mbar_wait(sm, &sm.mma_done[(jobidx - 1u) & 1u], ((jobidx - 1u) >> 1) & 1u);
+    // nothing may be in flight when tensor memory is released: the last committed job is waited for whatever the
+    // abort flag says (every issued product belongs to a committed job); if even that does not answer, tensor
+    // memory stays allocated
+    if (jobidx >= 1 && !mbar_drain(&sm.mma_done[(jobidx - 1u) & 1u], ((jobidx - 1u) >> 1) & 1u)) sm.tmem_busy = 1;
   } else {
     // ------------------------------------------------------------------ worker warps
     // norm role: token rows 32*eq + lane, channels [32 q, 32 q + 32); epilogue role: channels 32*eq + lane (the
@@ -370,7 +423,9 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
         const __half nh16 = __float2half_rn(n);
         const float nf = __half2float(nh16);
         if (eq == 0) reinterpret_cast<__half*>(cv.body(layer, cb, ch, cwin0 + ewq) + B_VNORM)[norm_pos(lane)] = nh16;
-        sm.c3[warp][lane] = nf != 0.0f ? __fmul_rn(__fdiv_rn(1.0f, nf), NEG_INV_3T) : 0.0f;
+        const float inv = nf != 0.0f ? __fdiv_rn(1.0f, nf) : 0.0f;
+        sm.inv[warp][lane] = inv;
+        sm.c3[warp][lane] = __fmul_rn(inv, NEG_INV_3T);
       }
       __syncwarp();
       uint32_t wacc[4] = {0u, 0u, 0u, 0u};   // this channel's codes of the window, one word per t (sh = 0 position)
@@ -414,7 +469,8 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
         if (!mbar_wait(sm, &sm.mma_done[a], (jobidx >> 1) & 1u)) { dead = true; break; }
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         const bool last_job = jt == 1 || __popc(tm.present) < 3;
-        // the tile's MMAs are complete and this warp keeps what it needs of the buffer in registers
+        // the tile's MMAs are complete and this warp keeps what it needs of the buffer in registers (the rare exact
+        // recomputation below reads its value row from global memory)
         if (last_job && lane == 0) mbar_arrive(&sm.empty[buf]);
         if (ewq < wins) {
           for (int mi = 0; mi < nm; mi++) {
@@ -428,7 +484,7 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
                          : "r"(taddr) : "memory");
             asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
             // token i = 8*j + 2*t + e sits in word t at bit 16*e + 2*j (+ 8 for the second channel of the word)
-            uint32_t kacc[4] = {0u, 0u, 0u, 0u};
+            uint32_t kaccA[4] = {0u, 0u, 0u, 0u}, kaccB[4] = {0u, 0u, 0u, 0u};
             const float4* c3p = reinterpret_cast<const float4*>(sm.c3[warp]);
 #pragma unroll
             for (int i4 = 0; i4 < 8; i4++) {
@@ -437,23 +493,58 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
 #pragma unroll
               for (int u = 0; u < 4; u++) {
                 const int t4 = 4 * i4 + u;
-                float v1, kf;
-                asm("fma.rn.sat.f32 %0, %1, %2, %3;\n" : "=f"(v1) : "f"(__uint_as_float(r[t4])), "f"(cs[u]), "f"(TWO_THIRDS));
-                asm("fma.rm.f32 %0, %1, %2, %3;\n" : "=f"(kf) : "f"(v1), "f"(3.0f), "f"(FLOOR_MAGIC));
-                kacc[(t4 & 7) >> 1] += __float_as_uint(kf) << (16 * (t4 & 1) + 2 * (t4 >> 3));
+                float va, vb, ka, kb;
+                asm("fma.rn.sat.f32 %0, %1, %2, %3;\n" : "=f"(va) : "f"(__uint_as_float(r[t4])), "f"(cs[u]), "f"(TWO_THIRDS - BAND_V));
+                asm("fma.rn.sat.f32 %0, %1, %2, %3;\n" : "=f"(vb) : "f"(__uint_as_float(r[t4])), "f"(cs[u]), "f"(TWO_THIRDS + BAND_V));
+                asm("fma.rm.f32 %0, %1, %2, %3;\n" : "=f"(ka) : "f"(va), "f"(3.0f), "f"(FLOOR_MAGIC));
+                asm("fma.rm.f32 %0, %1, %2, %3;\n" : "=f"(kb) : "f"(vb), "f"(3.0f), "f"(FLOOR_MAGIC));
+                kaccA[(t4 & 7) >> 1] += __float_as_uint(ka) << (16 * (t4 & 1) + 2 * (t4 >> 3));
+                kaccB[(t4 & 7) >> 1] += __float_as_uint(kb) << (16 * (t4 & 1) + 2 * (t4 >> 3));
               }
             }
 #pragma unroll
             for (int t = 0; t < 4; t++) {
               // kacc = sum of (magic bits + k) << pos over the word's eight tokens; codes = 3 - k per field
-              uint32_t codes = 0x00ff00ffu - (kacc[t] - MAGIC_SUM);
+              uint32_t codes = 0x00ff00ffu - (kaccA[t] - MAGIC_SUM);
+              uint32_t differ = codes ^ (0x00ff00ffu - (kaccB[t] - MAGIC_SUM));
+              uint32_t km = 0x00ff00ffu;
               if (keep != 0xffffffffu) {   // mixed-modality window: only this modality's tokens
-                uint32_t km = 0;
+                km = 0;
 #pragma unroll
                 for (int j = 0; j < 4; j++)
 #pragma unroll
                   for (int e = 0; e < 2; e++) km |= ((keep >> (8 * j + 2 * t + e)) & 1u) * (3u << (16 * e + 2 * j));
-                codes &= km;
+              }
+              codes &= km;
+              differ &= km;
+              while (differ) {   // rare: a coordinate within BAND of a threshold takes the reference arithmetic
+                const int pos = (__ffs(differ) - 1) & ~1;               // bit 16 e + 2 j of the field
+                const int tok = 8 * ((pos & 15) >> 1) + 2 * t + (pos >> 4);
+                const int c = 32 * eq + lane, mu = c >> 4, sh = (c >> 3) & 1, g = c & 7;
+                const __half* xrow = vrows + cb * vs_b + ch * vs_h + (long long)((cwin0 + ewq) * W + tok) * vs_t;
+                const float* rrow = R + (size_t)((n_R == 1 ? 0 : ch) * 3 + mods[mi]) * D * D + (size_t)c * D;
+                const int slot_i = atomicAdd(&sm.fix_count, 1);
+                if (slot_i < FIX_MAX) {   // later, by a whole warp (the code written now is one of the two neighbouring levels)
+                  FixItem& it = sm.fix[slot_i];
+                  it.word = reinterpret_cast<uint32_t*>(cv.body(layer, cb, ch, cwin0 + ewq) + B_VCODE) +
+                            vword_index((mu >> 2) * 128 + (4 * g + t) * 4 + (mu & 3));
+                  it.xrow = xrow; it.rrow = rrow; it.inv = sm.inv[warp][tok]; it.bit = pos + 8 * sh;
+                } else {                  // the list is full: here and now
+                  float a = 0.0f;
+#pragma unroll 4
+                  for (int kc = 0; kc < 16; kc++) {
+                    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(xrow) + kc);
+                    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+                    const float4 r0 = __ldg(reinterpret_cast<const float4*>(rrow) + 2 * kc), r1 = __ldg(reinterpret_cast<const float4*>(rrow) + 2 * kc + 1);
+                    const float2 x0 = __half22float2(h2[0]), x1 = __half22float2(h2[1]), x2 = __half22float2(h2[2]), x3 = __half22float2(h2[3]);
+                    a = __fmaf_rn(r0.x, x0.x, a); a = __fmaf_rn(r0.y, x0.y, a); a = __fmaf_rn(r0.z, x1.x, a); a = __fmaf_rn(r0.w, x1.y, a);
+                    a = __fmaf_rn(r1.x, x2.x, a); a = __fmaf_rn(r1.y, x2.y, a); a = __fmaf_rn(r1.z, x3.x, a); a = __fmaf_rn(r1.w, x3.y, a);
+                  }
+                  const float z = __fmul_rn(a, sm.inv[warp][tok]);
+                  const uint32_t code = (uint32_t)((z > -CB_THRESH) + (z > 0.0f) + (z > CB_THRESH));
+                  codes = (codes & ~(3u << pos)) | (code << pos);
+                }
+                differ &= ~(3u << pos);
               }
               wacc[t] |= codes;
             }
@@ -483,8 +574,37 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
   }
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
   __syncthreads();
+  // ---- the listed coordinates, one per warp at a time: the two rows go through the warp's corner of the (idle) first
+  // tile buffer, every lane evaluates the same chain (input index ascending, one rounding per step), lane 0 patches
+  {
+    const int n_fix = min(sm.fix_count, FIX_MAX);
+    unsigned char* scr = sm.a[0] + warp * 1024;
+    for (int i = warp; i < n_fix && !sm.abort; i += NT_ALL / 32) {
+      const FixItem it = sm.fix[i];
+      *reinterpret_cast<float4*>(scr + 16 * lane) = __ldg(reinterpret_cast<const float4*>(it.rrow) + lane);
+      if (lane < 16) *reinterpret_cast<uint4*>(scr + 512 + 16 * lane) = __ldg(reinterpret_cast<const uint4*>(it.xrow) + lane);
+      __syncwarp();
+      float a = 0.0f;
+#pragma unroll 4
+      for (int kc = 0; kc < 16; kc++) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(scr + 512 + 16 * kc);
+        const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+        const float4 r0 = *reinterpret_cast<const float4*>(scr + 32 * kc), r1 = *reinterpret_cast<const float4*>(scr + 32 * kc + 16);
+        const float2 x0 = __half22float2(h2[0]), x1 = __half22float2(h2[1]), x2 = __half22float2(h2[2]), x3 = __half22float2(h2[3]);
+        a = __fmaf_rn(r0.x, x0.x, a); a = __fmaf_rn(r0.y, x0.y, a); a = __fmaf_rn(r0.z, x1.x, a); a = __fmaf_rn(r0.w, x1.y, a);
+        a = __fmaf_rn(r1.x, x2.x, a); a = __fmaf_rn(r1.y, x2.y, a); a = __fmaf_rn(r1.z, x3.x, a); a = __fmaf_rn(r1.w, x3.y, a);
+      }
+      const float z = __fmul_rn(a, it.inv);
+      const uint32_t code = (uint32_t)((z > -CB_THRESH) + (z > 0.0f) + (z > CB_THRESH));
+      if (lane == 0) {
+        atomicAnd(it.word, ~(3u << it.bit));
+        atomicOr(it.word, code << it.bit);
+      }
+      __syncwarp();
+    }
+  }
   if (tid == 0 && sm.abort) atomicCAS(cv.status, 0, (int)OKQ_ERR_TIMEOUT);
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;\n" ::"r"(tmem) : "memory");
+  if (warp == 0 && !sm.tmem_busy) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;\n" ::"r"(tmem) : "memory");
 }
 
 namespace {
@@ -535,7 +655,8 @@ okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __hal
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) { set_last_cuda_error((int)cudaErrorInvalidValue); return OKQ_ERR_CUDA; }
   const int grid = (int)(n_tiles < n_sm ? n_tiles : n_sm);
-  k_quantize_values_tc<<<grid, NT_ALL, sizeof(TcSmem) + 1024, s>>>(vmap, cv, layer, modality, n_tokens, n_win, R, n_R);
+  k_quantize_values_tc<<<grid, NT_ALL, sizeof(TcSmem) + 1024, s>>>(vmap, cv, layer, modality, n_tokens, n_win, R, n_R, v, (long long)strides[0],
+                                                                   (long long)strides[1], (long long)strides[2]);
   return OKQ_OK;
 }
 

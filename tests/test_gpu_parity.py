@@ -179,8 +179,8 @@ def test_per_head_rotations():
 
 
 def _check_bulk_codes(c, layer, R_host):
-    """Codes of the tensor-core value quantiser against the oracle: identical except, at most, where the
-    oracle's rotated coordinate lies within 2^-20 of a codebook threshold (then they differ by one level)."""
+    """Codes of the tensor-core value quantiser against the oracle: returns the number that differ (none may: the
+    kernel recomputes every coordinate near a threshold with the reference arithmetic) after saying where."""
     kq, vq, _, vb = c.oracle_quantize(layer)
     e = {k: v.cpu() for k, v in c.gpu_export(layer).items()}
     U = c.w.batch * c.w.n_kv_heads
@@ -195,8 +195,8 @@ def _check_bulk_codes(c, layer, R_host):
     for (u, i, ch) in bad:
         m = c.mod_b.numpy()[unit_seq[u], i]
         _, z = O.value_rotate(vb[u, i], R_host[m])
-        assert abs(int(got[u, i, ch]) - int(ref[u, i, ch])) == 1
-        assert np.abs(float(z[ch]) - thr).min() <= 2.0 ** -20, (u, i, ch, z[ch])
+        print("value code differs:", (u, i, ch), int(got[u, i, ch]), int(ref[u, i, ch]), "distance to threshold",
+              np.abs(float(z[ch]) - thr).min())
     return len(bad), ref.size
 
 
@@ -209,10 +209,9 @@ def test_bulk_value_quantiser_on_tensor_cores():
     torch.cuda.synchronize()
     assert c.cache.device_status() == 0
     n_bad, n_all = _check_bulk_codes(c, 0, c.R[0].numpy())
-    print(f"tensor-core value codes: {n_bad} of {n_all} differ from the exact chain (all within 2^-20 of a threshold)")
-    assert n_bad <= n_all * 2e-4
-    # decode over the bulk-built cache matches the oracle over the value codes the cache holds
-    ref, _ = c.oracle_attention(0, v_codes=c.gpu_export(0)["v_codes"])
+    assert n_bad == 0, f"{n_bad} of {n_all} tensor-core value codes differ from the exact chain"
+    # decode over the bulk-built cache matches the oracle
+    ref, _ = c.oracle_attention(0)
     Hn.assert_attention_close(c.gpu_decode(0)[0], ref)
     # raw tail and modality as in the exact path
     U = w.batch * w.n_kv_heads
