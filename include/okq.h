@@ -165,6 +165,17 @@ okq_status okq_quantize_values_bulk(const okq_cache* cache, int32_t layer, const
                                     void* stream);
 
 /*
+ * Testing aid for the bounded waits of okq_quantize_values_bulk (the paper has no counterpart): the same launch with
+ * the first 128-token tile never delivered to the tensor-core pipeline and every wait limited to `limit_clocks` SM
+ * clocks (a few milliseconds' worth is enough).  Every role's wait for that tile runs out, the kernel returns by
+ * itself, the device status word becomes OKQ_ERR_TIMEOUT and the layer's value records are left incomplete: quantise
+ * the layer again before using it.  Nothing faults and the context stays usable.
+ */
+okq_status okq_debug_bulk_timeout(const okq_cache* cache, int32_t layer, const void* v_fp16,
+                                  const int64_t strides[3], int32_t n_tokens, const uint8_t* modality,
+                                  const float* R, int32_t n_R, int64_t limit_clocks, void* stream);
+
+/*
  * Streaming append (the paper's protocol keeps recent tokens in fp16 before they are
  * quantised): add one token per sequence to layers [layer, layer+layer_count).  The token
  * goes raw into the tail; when the tail reaches 32 tokens they are quantised as one window

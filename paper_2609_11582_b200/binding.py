@@ -64,6 +64,8 @@ def lib():
                                           C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.okq_quantize_values_bulk.restype = C.c_int
         L.okq_quantize_values_bulk.argtypes = L.okq_quantize_values.argtypes
+        L.okq_debug_bulk_timeout.restype = C.c_int
+        L.okq_debug_bulk_timeout.argtypes = list(L.okq_quantize_values.argtypes[:-1]) + [C.c_int64, C.c_void_p]
         L.okq_append.restype = C.c_int
         L.okq_append.argtypes = [C.POINTER(okq_cache), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
@@ -105,7 +107,7 @@ def exported_symbols():
     return ["okq_status_string", "okq_last_cuda_error", "okq_cache_sizes", "okq_decode_workspace_bytes",
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
             "okq_cache_import", "okq_profile_events", "okq_decode_select", "okq_decode_attention_simt",
-            "okq_decode_attention_noalloc", "okq_quantize_values_bulk", "okq_cache_export_mx",
+            "okq_decode_attention_noalloc", "okq_quantize_values_bulk", "okq_debug_bulk_timeout", "okq_cache_export_mx",
             "okq_calib_workspace_bytes", "okq_calib_attention_weights", "okq_calib_moments", "okq_calib_rotation"]
 
 
@@ -185,6 +187,16 @@ def quantize_values(cache: Cache, layer: int, v: torch.Tensor, modality: torch.T
     fn = lib().okq_quantize_values_bulk if bulk else lib().okq_quantize_values
     _check(fn(C.byref(cache.c), layer, _ptr(v), strides, n, _ptr(modality), _ptr(R), n_R, _stream(stream)),
            "okq_quantize_values_bulk" if bulk else "okq_quantize_values")
+
+
+def debug_bulk_timeout(cache: Cache, layer: int, v: torch.Tensor, modality: torch.Tensor, R: torch.Tensor,
+                       limit_clocks: int = 20_000_000, stream=None):
+    """okq_debug_bulk_timeout: the bulk value quantiser with its first tile withheld and every wait limited to
+    `limit_clocks` SM clocks; the device status word becomes ERR_TIMEOUT (testing aid)."""
+    strides = (C.c_int64 * 3)(v.stride(0), v.stride(1), v.stride(2))
+    n_R = R.shape[0] if R.dim() == 4 else 1
+    _check(lib().okq_debug_bulk_timeout(C.byref(cache.c), layer, _ptr(v), strides, v.shape[2], _ptr(modality), _ptr(R), n_R,
+                                        limit_clocks, _stream(stream)), "okq_debug_bulk_timeout")
 
 
 def append(cache: Cache, layer: int, layer_count: int, k_new, v_new, modality_new, signs, R, n_R=1, stream=None):

@@ -545,7 +545,7 @@ __global__ void k_import(CacheView cv, int layer, const unsigned char* k_codes, 
 
 okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __half* v, const int64_t strides[3],
                                      const unsigned char* modality, int n_tokens, int n_win, const float* R, int n_R,
-                                     int n_sm, cudaStream_t s);
+                                     int n_sm, cudaStream_t s, long long wait_limit = 0, int skip_tile = -1);
 
 constexpr int TAIL_SLICES = 16;   // blocks per (sequence, head) that share the copy of the modality bytes
 
@@ -623,6 +623,20 @@ okq_status okq_quantize_values_bulk(const okq_cache* cache, int32_t layer, const
   k_bulk_tail<<<dim3(cv.n_kv_heads, cv.batch, TAIL_SLICES), 128, 0, s>>>(cv, layer, v, strides[0], strides[1], strides[2],
                                                                         n_tokens, 1, n_tokens > 0 ? modality : nullptr);
   return launch_status();
+}
+
+okq_status okq_debug_bulk_timeout(const okq_cache* cache, int32_t layer, const void* v_fp16, const int64_t strides[3],
+                                  int32_t n_tokens, const uint8_t* modality, const float* R, int32_t n_R,
+                                  int64_t limit_clocks, void* stream) {
+  okq_status st = check_bulk(cache, layer, v_fp16, strides, n_tokens);
+  if (st != OKQ_OK) return st;
+  if (!modality || !R || (n_R != 1 && n_R != cache->n_kv_heads) || limit_clocks <= 0) return OKQ_ERR_INVALID_ARG;
+  if (!aligned16(R)) return OKQ_ERR_ALIGNMENT;
+  CacheView cv = make_view(cache);
+  st = launch_quantize_values_tc(cv, layer, static_cast<const __half*>(v_fp16), strides, modality, n_tokens,
+                                 cv.v_packed(n_tokens) / W, R, n_R, sm_count(), static_cast<cudaStream_t>(stream),
+                                 (long long)limit_clocks, 0);
+  return st != OKQ_OK ? st : launch_status();
 }
 
 okq_status okq_append(const okq_cache* cache, int32_t layer, int32_t layer_count, const void* k_new,

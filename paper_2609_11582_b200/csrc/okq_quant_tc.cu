@@ -89,6 +89,7 @@ struct TcSmem {
   uint32_t tmem_slot;
   FixItem fix[FIX_MAX];
   int fix_count;
+  long long limit;                                     // SM clocks a wait may take
   volatile int abort;                                  // set by a role whose bounded wait ran out
   volatile int tmem_busy;                              // set if products may still be in flight at the end (tensor memory is then not released)
 };
@@ -137,7 +138,7 @@ __device__ __forceinline__ bool mbar_wait(TcSmem& sm, unsigned long long* bar, u
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                  : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
     done = ok != 0;
-    if (!done && (sm.abort || clock64() - t0 > WAIT_LIMIT_CLOCKS)) break;
+    if (!done && (sm.abort || clock64() - t0 > sm.limit)) break;
   }
   if (!done) sm.abort = 1;
   return __all_sync(0xffffffffu, done);   // called by whole warps: one answer per warp
@@ -148,7 +149,7 @@ __device__ __forceinline__ bool mbar_drain(unsigned long long* bar, uint32_t par
   const uint32_t mbar = smem_u32(bar);
   bool done = false;
   const long long t0 = clock64();
-  while (!done && clock64() - t0 < WAIT_LIMIT_CLOCKS / 8) {
+  while (!done && clock64() - t0 < WAIT_LIMIT_CLOCKS / 8) {   // a quarter of a second, whatever the caller's limit
     uint32_t ok;
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                  : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
@@ -227,7 +228,7 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
                                                              const unsigned char* __restrict__ modality, int n_tokens,
                                                              int n_win, const float* __restrict__ R, int n_R,
                                                              const __half* __restrict__ vrows, long long vs_b, long long vs_h,
-                                                             long long vs_t) {
+                                                             long long vs_t, long long wait_limit, int skip_tile) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   TcSmem& sm = *reinterpret_cast<TcSmem*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -250,6 +251,7 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
     sm.abort = 0;
     sm.tmem_busy = 0;
     sm.fix_count = 0;
+    sm.limit = wait_limit;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (warp == 0) {
@@ -297,6 +299,11 @@ __global__ void __launch_bounds__(NT_ALL, 1) k_quantize_values_tc(const __grid_c
     int armed = 0;   // tiles whose copies have been issued
     for (int i = 0; i < my_tiles; i++) {
       const int buf = i & 1, fill = i >> 1;
+      if (tile_begin + i == skip_tile) {   // testing aid: this tile never arrives, so that every role's wait runs out
+        step_coords();
+        mod_cur = fetch_mod(i + 1);
+        continue;
+      }
       if (fill >= 1 && !mbar_wait(sm, &sm.empty[buf], (uint32_t)(fill - 1) & 1u)) break;
       reinterpret_cast<uint32_t*>(sm.mod[buf])[lane] = mod_cur;
       __syncwarp();
@@ -628,7 +635,7 @@ EncodeTiledFn encode_tiled() {
 
 okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __half* v, const int64_t strides[3],
                                      const unsigned char* modality, int n_tokens, int n_win, const float* R, int n_R,
-                                     int n_sm, cudaStream_t s) {
+                                     int n_sm, cudaStream_t s, long long wait_limit, int skip_tile) {
   static thread_local unsigned long long attr_mask = 0;
   int attr_dev = 0;
   if (attr_needed(attr_mask, attr_dev)) {
@@ -656,7 +663,7 @@ okq_status launch_quantize_values_tc(const CacheView& cv, int layer, const __hal
   if (cr != CUDA_SUCCESS) { set_last_cuda_error((int)cudaErrorInvalidValue); return OKQ_ERR_CUDA; }
   const int grid = (int)(n_tiles < n_sm ? n_tiles : n_sm);
   k_quantize_values_tc<<<grid, NT_ALL, sizeof(TcSmem) + 1024, s>>>(vmap, cv, layer, modality, n_tokens, n_win, R, n_R, v, (long long)strides[0],
-                                                                   (long long)strides[1], (long long)strides[2]);
+                                                                   (long long)strides[1], (long long)strides[2], wait_limit > 0 ? wait_limit : WAIT_LIMIT_CLOCKS, skip_tile);
   return OKQ_OK;
 }
 

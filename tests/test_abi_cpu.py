@@ -31,6 +31,7 @@ def test_every_declared_symbol_is_exported(L):
 
 def test_status_strings(L):
     assert L.okq_status_string(0) == b"ok"
+    assert L.okq_status_string(B.ERR_TIMEOUT) == b"bounded device wait timed out"   # the device status of a wait that ran out
     seen = {L.okq_status_string(i) for i in range(8)}
     assert len(seen) == 8
     assert L.okq_last_cuda_error() == 0

@@ -87,3 +87,32 @@ def test_guard_words_and_determinism():
     torch.cuda.synchronize()
     assert e["k_codes"].shape == (Bn, H, cap, 32)
     del rec_view
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """The tensor-core value quantiser with its first tile withheld and every wait limited to about ten milliseconds:
+    each role's wait for that tile runs out, the kernel returns by itself and the device status word says
+    ERR_TIMEOUT.  Nothing faults: the context stays usable, and the same call without the handicap then gives the
+    codes of the exact quantiser."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=2)
+    n = 1024 + 40
+    dev = torch.device("cuda")
+    k, v = WL.gen_kv(w, 0, n_tokens=n)
+    mod = WL.modality_layout(w, n).unsqueeze(0).repeat(w.batch, 1).contiguous().to(dev)
+    R = WL.gen_rotations(w, 0)[None].contiguous().to(dev)
+    vd = v.to(dev)
+    cache = B.Cache(1, w.batch, w.n_kv_heads, w.n_q_heads, 1088, device=dev)
+    B.debug_bulk_timeout(cache, 0, vd, mod, R, limit_clocks=20_000_000)
+    torch.cuda.synchronize()                      # returns: the kernel ended by itself
+    assert cache.device_status() == B.ERR_TIMEOUT
+    assert b"timed out" in B.lib().okq_status_string(B.ERR_TIMEOUT)
+    cache.status.zero_()
+    B.quantize_values(cache, 0, vd, mod, R, bulk=True)
+    torch.cuda.synchronize()
+    assert cache.device_status() == 0
+    exact = B.Cache(1, w.batch, w.n_kv_heads, w.n_q_heads, 1088, device=dev)
+    B.quantize_values(exact, 0, vd, mod, R)
+    torch.cuda.synchronize()
+    ea, eb = B.cache_export(cache, 0), B.cache_export(exact, 0)
+    npk = (n // W) * W
+    assert torch.equal(ea["v_codes"][:, :, :npk], eb["v_codes"][:, :, :npk]) and torch.equal(ea["v_norm"][:, :, :npk], eb["v_norm"][:, :, :npk])
