@@ -2,37 +2,22 @@
 oracle on the synthetic workload: storage rates exactly, error metrics by their ordering.
 
 The TurboQuant baseline (norm, randomised Hadamard, fixed Lloyd-Max codebook of the N(0, 1/d) reference, no
-window statistics, no modality rotation) is written here from the paper's preliminaries, in fp64; it is a
-comparison method, not part of the product.  CPU only."""
+window statistics, no modality rotation) is the oracle's codec (oracle/okq_ladder_oracle.py, written from the paper's
+preliminaries and pinned on its own); it is a comparison method, not part of the product.  CPU only."""
 import numpy as np
 import pytest
-from scipy.stats import norm as gauss
 
-from oracle import okq_calib_oracle as CO
+from oracle import okq_ladder_oracle as LO
 from oracle import okq_oracle as O
 from paper_2609_11582_b200 import workloads as WL
 
 D, W = 128, 32
 
 
-def lloyd_max(bits, sigma):
-    """Lloyd-Max levels of N(0, sigma^2) by fixed-point iteration on the closed-form cell means."""
-    n = 1 << bits
-    lv = np.linspace(-2, 2, n) * sigma
-    for _ in range(500):
-        t = np.concatenate([[-np.inf], (lv[:-1] + lv[1:]) / 2, [np.inf]])
-        a, b = t[:-1] / sigma, t[1:] / sigma
-        lv = sigma * (gauss.pdf(a) - gauss.pdf(b)) / (gauss.cdf(b) - gauss.cdf(a))
-    return lv
-
-
-def turboquant(x, H, bits):
-    """x: fp64 [n, 128] -> reconstruction: norm * H^T cb[nearest level of H x / norm]."""
-    lv = lloyd_max(bits, 1.0 / np.sqrt(D))
-    nrm = np.linalg.norm(x, axis=1, keepdims=True)
-    z = (x / np.where(nrm == 0, 1, nrm)) @ H.T
-    codes = np.abs(z[..., None] - lv).argmin(axis=-1)
-    return (lv[codes] @ H) * nrm
+def turboquant(x16, signs, bits):
+    """x16: fp16 [n, 128] -> reconstruction norm * H^T cb[nearest level of H x / norm], fp64."""
+    codes, norm = LO.turboquant_encode(np.ascontiguousarray(x16).view(np.uint16), signs, bits)
+    return LO.turboquant_decode(codes, norm, signs, bits)
 
 
 def softmax(s):
@@ -72,12 +57,6 @@ def metrics(data, k_hat, v_hat):
     return recon, kl, out
 
 
-def test_lloyd_max_two_bit_levels_are_the_codebook():
-    lv = lloyd_max(2, 1.0 / np.sqrt(D))
-    levels, thresh = O.codebook()
-    assert np.allclose(lv, levels, rtol=2e-6) and np.isclose((lv[2] + lv[3]) / 2, thresh, rtol=2e-6)
-
-
 def test_storage_rates_of_the_table():
     # TurboQuant: b bits per coordinate + one fp16 norm per vector
     tq = lambda kb, vb: ((kb * D + 16) + (vb * D + 16)) / (2 * D)
@@ -88,12 +67,10 @@ def test_storage_rates_of_the_table():
 
 def test_error_ordering_of_the_table(data):
     k16, v16, q, signs, R, mod = data
-    H = CO.hadamard_matrix(signs)
-    k, v = k16.astype(np.float64), v16.astype(np.float64)
     rows = {
-        "TurboQuant K2/V2": metrics(data, turboquant(k, H, 2), turboquant(v, H, 2)),
+        "TurboQuant K2/V2": metrics(data, turboquant(k16, signs, 2), turboquant(v16, signs, 2)),
         "ours, MXFP4 meta": metrics(data, *ours(data, 1)),
-        "TurboQuant K3/V2": metrics(data, turboquant(k, H, 3), turboquant(v, H, 2)),
+        "TurboQuant K3/V2": metrics(data, turboquant(k16, signs, 3), turboquant(v16, signs, 2)),
         "ours, fp16 meta": metrics(data, *ours(data, 0)),
     }
     for name, (r, kl, o) in rows.items():
