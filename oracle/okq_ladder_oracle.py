@@ -38,6 +38,7 @@ def lloyd_max(bits: int, iters: int = 2000):
             lv = new
             break
         lv = new
+    lv = (lv - lv[::-1]) / 2          # the quantiser of a symmetric density is symmetric: the middle threshold is exactly 0
     return lv, (lv[:-1] + lv[1:]) / 2
 
 

@@ -29,6 +29,13 @@ class okq_cache(C.Structure):
                 ("seq_len", C.c_void_p), ("status", C.c_void_p)]
 
 
+class okq_ladder_cache(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32), ("capacity", C.c_int32),
+                ("bits", C.c_int32), ("reserved", C.c_int32),
+                ("k_codes", C.c_void_p), ("k_norm", C.c_void_p), ("k_meta", C.c_void_p), ("v_codes", C.c_void_p),
+                ("v_norm", C.c_void_p), ("modality", C.c_void_p)]
+
+
 class OkqError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -99,6 +106,17 @@ def lib():
                                          C.c_void_p, C.c_void_p]
         L.okq_cache_import.restype = C.c_int
         L.okq_cache_import.argtypes = [C.POINTER(okq_cache), C.c_int32] + [C.c_void_p] * 6
+        L.okq_ladder_codebook.restype = C.c_int32
+        L.okq_ladder_codebook.argtypes = [C.c_int32, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+        L.okq_ladder_quantize_keys.restype = C.c_int
+        L.okq_ladder_quantize_keys.argtypes = [C.POINTER(okq_ladder_cache), C.c_void_p, C.POINTER(C.c_int64), C.c_int32,
+                                               C.c_void_p, C.c_void_p]
+        L.okq_ladder_quantize_values.restype = C.c_int
+        L.okq_ladder_quantize_values.argtypes = [C.POINTER(okq_ladder_cache), C.c_void_p, C.POINTER(C.c_int64), C.c_int32,
+                                                 C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        L.okq_ladder_decode_attention.restype = C.c_int
+        L.okq_ladder_decode_attention.argtypes = [C.POINTER(okq_ladder_cache), C.c_int32, C.c_void_p, C.c_float, C.c_void_p,
+                                                  C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -108,7 +126,9 @@ def exported_symbols():
             "okq_quantize_keys", "okq_quantize_values", "okq_append", "okq_decode_attention", "okq_cache_export",
             "okq_cache_import", "okq_profile_events", "okq_decode_select", "okq_decode_attention_simt",
             "okq_decode_attention_noalloc", "okq_quantize_values_bulk", "okq_debug_bulk_timeout", "okq_cache_export_mx",
-            "okq_calib_workspace_bytes", "okq_calib_attention_weights", "okq_calib_moments", "okq_calib_rotation"]
+            "okq_calib_workspace_bytes", "okq_calib_attention_weights", "okq_calib_moments", "okq_calib_rotation",
+            "okq_ladder_codebook", "okq_ladder_quantize_keys", "okq_ladder_quantize_values",
+            "okq_ladder_decode_attention"]
 
 
 def _ptr(t) -> int:
@@ -300,3 +320,53 @@ def calib_rotation(Cm, signs, workspace, stream=None):
     _check(lib().okq_calib_rotation(_ptr(Cm), _ptr(signs), _ptr(workspace), workspace.numel(), _ptr(R), _ptr(lam),
                                     _ptr(sweeps), _stream(stream)), "okq_calib_rotation")
     return R, lam, sweeps
+
+
+# ---------------------------------------------------------------- bit-width ladder (okq_ladder.h)
+class LadderCache:
+    """Device buffers of an okq_ladder_cache at `bits` bits per code (canonical layout, one layer)."""
+
+    def __init__(self, batch, n_kv_heads, n_q_heads, capacity, bits, device="cuda"):
+        self.bits, self.capacity = bits, capacity
+        dev = torch.device(device)
+        rows = (batch, n_kv_heads, capacity)
+        self.k_codes = torch.zeros(rows + (16 * bits,), dtype=torch.uint8, device=dev)
+        self.v_codes = torch.zeros(rows + (16 * bits,), dtype=torch.uint8, device=dev)
+        self.k_norm = torch.zeros(rows, dtype=torch.float16, device=dev)
+        self.v_norm = torch.zeros(rows, dtype=torch.float16, device=dev)
+        self.k_meta = torch.zeros((batch, n_kv_heads, capacity // WINDOW, HEAD_DIM, 2), dtype=torch.float16, device=dev)
+        self.modality = torch.zeros((batch, capacity), dtype=torch.uint8, device=dev)
+        self.c = okq_ladder_cache(batch, n_kv_heads, n_q_heads, capacity, bits, 0, _ptr(self.k_codes), _ptr(self.k_norm),
+                                  _ptr(self.k_meta), _ptr(self.v_codes), _ptr(self.v_norm), _ptr(self.modality))
+
+
+def ladder_codebook(bits: int):
+    """(levels, thresholds) the kernels hold for `bits`, as Python lists of floats."""
+    lv, th = (C.c_float * 16)(), (C.c_float * 15)()
+    n = lib().okq_ladder_codebook(bits, lv, th)
+    if n == 0:
+        raise OkqError(ERR_UNSUPPORTED, "okq_ladder_codebook")
+    return list(lv)[:n], list(th)[:n - 1]
+
+
+def ladder_quantize_keys(cache: LadderCache, k: torch.Tensor, signs: torch.Tensor, stream=None):
+    assert k.dtype == torch.float16 and k.stride(3) == 1
+    strides = (C.c_int64 * 3)(k.stride(0), k.stride(1), k.stride(2))
+    _check(lib().okq_ladder_quantize_keys(C.byref(cache.c), _ptr(k), strides, k.shape[2], _ptr(signs), _stream(stream)),
+           "okq_ladder_quantize_keys")
+
+
+def ladder_quantize_values(cache: LadderCache, v: torch.Tensor, modality: torch.Tensor, R: torch.Tensor, stream=None):
+    assert v.dtype == torch.float16 and v.stride(3) == 1 and modality.dtype == torch.uint8 and modality.is_contiguous()
+    strides = (C.c_int64 * 3)(v.stride(0), v.stride(1), v.stride(2))
+    n_R = R.shape[0] if R.dim() == 4 else 1
+    _check(lib().okq_ladder_quantize_values(C.byref(cache.c), _ptr(v), strides, v.shape[2], _ptr(modality), _ptr(R), n_R,
+                                            _stream(stream)), "okq_ladder_quantize_values")
+
+
+def ladder_decode_attention(cache: LadderCache, n_tokens: int, q, signs, R, out, sm_scale=None, stream=None):
+    """q: fp16 [batch, n_q_heads, 128]; out: float32 [batch, n_q_heads, 128]."""
+    n_R = R.shape[0] if R.dim() == 4 else 1
+    scale = HEAD_DIM ** -0.5 if sm_scale is None else sm_scale
+    _check(lib().okq_ladder_decode_attention(C.byref(cache.c), n_tokens, _ptr(q), scale, _ptr(signs), _ptr(R), n_R,
+                                             _ptr(out), _stream(stream)), "okq_ladder_decode_attention")

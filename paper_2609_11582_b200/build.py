@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libokq.so")
-SOURCES = ["okq_host.cu", "okq_quant.cu", "okq_decode.cu", "okq_decode_mma.cu", "okq_decode_tc.cu", "okq_quant_tc.cu", "okq_calib.cu"]
+SOURCES = ["okq_host.cu", "okq_quant.cu", "okq_decode.cu", "okq_decode_mma.cu", "okq_decode_tc.cu", "okq_quant_tc.cu", "okq_calib.cu", "okq_ladder.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]
 

@@ -96,3 +96,41 @@ def test_calibration_argument_checks(L):
     assert L.okq_calib_attention_weights(fake, fake, 7, 64, C.c_float(1.0), 1, fake, 16, fake, null) == B.ERR_WORKSPACE
     assert L.okq_calib_attention_weights(C.c_void_p(4100), fake, 7, 64, C.c_float(1.0), 1, fake, 1 << 30, fake, null) == B.ERR_ALIGNMENT
     assert L.okq_calib_rotation(fake, fake, fake, 1024, fake, fake, null, null) == B.ERR_WORKSPACE
+
+
+def test_ladder_codebook_constants_equal_the_oracle_quantiser(L):
+    """The value levels and thresholds compiled into the ladder kernels are the fp32 roundings of the Lloyd-Max
+    quantiser of N(0, 1/128) that the oracle derives by iteration (Eq. 3)."""
+    import numpy as np
+    from oracle import okq_ladder_oracle as LO
+    for bits in (2, 3, 4):
+        lv, th = B.ladder_codebook(bits)
+        olv, oth = LO.codebook32(bits)
+        assert np.array_equal(np.array(lv, dtype=np.float32), olv), bits
+        assert np.array_equal(np.array(th, dtype=np.float32), oth), bits
+    lv, th = (C.c_float * 16)(), (C.c_float * 15)()
+    assert L.okq_ladder_codebook(5, lv, th) == 0 and L.okq_ladder_codebook(1, lv, th) == 0
+
+
+def test_ladder_validation_before_any_launch(L):
+    fake = 1 << 20
+    strides = (C.c_int64 * 3)(64 * 128, 64 * 128, 128)
+
+    def cache(bits=3, capacity=64, n_q=7, **kw):
+        ptrs = dict(k_codes=fake, k_norm=fake, k_meta=fake, v_codes=fake, v_norm=fake, modality=fake)
+        ptrs.update(kw)
+        return B.okq_ladder_cache(1, 1, n_q, capacity, bits, 0, ptrs["k_codes"], ptrs["k_norm"], ptrs["k_meta"],
+                                  ptrs["v_codes"], ptrs["v_norm"], ptrs["modality"])
+    keys = lambda c, n=64, k=fake: L.okq_ladder_quantize_keys(C.byref(c), k, strides, n, fake, None)
+    assert keys(cache(bits=5)) == B.ERR_UNSUPPORTED
+    assert keys(cache(bits=1)) == B.ERR_UNSUPPORTED
+    assert keys(cache(n_q=9)) == B.ERR_UNSUPPORTED
+    assert keys(cache(capacity=70)) == B.ERR_INVALID_ARG
+    assert keys(cache(), n=48) == B.ERR_INVALID_ARG            # not a whole number of windows
+    assert keys(cache(), n=96) == B.ERR_INVALID_ARG            # beyond the capacity
+    assert keys(cache(k_meta=0)) == B.ERR_INVALID_ARG
+    assert keys(cache(k_codes=fake + 4)) == B.ERR_ALIGNMENT
+    assert keys(cache(), k=fake + 2) == B.ERR_ALIGNMENT
+    assert keys(cache(), n=0) == B.OK                          # nothing to do, nothing launched
+    assert L.okq_ladder_quantize_values(C.byref(cache()), fake, strides, 64, fake, fake, 2, None) == B.ERR_INVALID_ARG
+    assert L.okq_ladder_decode_attention(C.byref(cache()), 64, fake, 0.1, fake, fake, 1, 0, None) == B.ERR_INVALID_ARG

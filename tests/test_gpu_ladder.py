@@ -1,0 +1,160 @@
+"""GPU parity of the bit-width ladder entry points (okq_ladder.h) against the ladder oracle at 2, 3 and 4 bits:
+the quantisers bit for bit (norms, (m, s), every code of the bit stream), decode attention against the plain
+definition softmax(q K_hat^T / sqrt(d)) V_hat evaluated in fp64 over the oracle's dequantised cache."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import okq_ladder_oracle as LO
+from oracle import okq_oracle as O
+from paper_2609_11582_b200 import binding as B
+from paper_2609_11582_b200 import workloads as WL
+from tests import harness as Hn
+
+pytestmark = pytest.mark.gpu
+D, W = 128, 32
+
+
+def unpack_stream(rows: np.ndarray, bits: int) -> np.ndarray:
+    """uint8 [..., 16 * bits] little-endian bit stream -> codes uint8 [..., 128] (channel c at bits [bits c, bits c + bits))."""
+    b = np.unpackbits(rows, axis=-1, bitorder="little").reshape(rows.shape[:-1] + (D, bits))
+    return (b.astype(np.uint16) << np.arange(bits, dtype=np.uint16)).sum(axis=-1).astype(np.uint8)
+
+
+class LadderCase:
+    def __init__(self, w: WL.Workload, bits: int, n_tokens: int, modality=None, k=None, v=None):
+        self.w, self.bits, self.n = w, bits, n_tokens
+        self.signs = WL.gen_signs(w, 0)
+        self.R = WL.gen_rotations(w, 0)                        # [3,128,128]
+        self.q = WL.gen_queries(w, 0)                          # [B,Hq,128] fp16
+        gk, gv = WL.gen_kv(w, 0, n_tokens=n_tokens)
+        self.k = gk if k is None else k
+        self.v = gv if v is None else v
+        self.mod = WL.modality_layout(w, n_tokens) if modality is None else modality
+        self.mod_b = self.mod.unsqueeze(0).repeat(w.batch, 1).contiguous()
+        self.cache = B.LadderCache(w.batch, w.n_kv_heads, w.n_q_heads, n_tokens + W, bits)
+        self.d_signs, self.d_R = self.signs.cuda(), self.R.unsqueeze(0).contiguous().cuda()
+        B.ladder_quantize_keys(self.cache, self.k.cuda(), self.d_signs)
+        B.ladder_quantize_values(self.cache, self.v.cuda(), self.mod_b.cuda(), self.d_R)
+        torch.cuda.synchronize()
+
+    def oracle_units(self):
+        """Per (sequence, KV head): the oracle's quantised keys and values."""
+        w = self.w
+        mod = self.mod.numpy()
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                kq = LO.quantize_keys(Hn.u16(self.k[b, h]), self.signs.numpy(), self.bits)
+                vq = LO.quantize_values(Hn.u16(self.v[b, h]), mod, self.R.numpy(), self.bits)
+                yield b, h, kq, vq
+
+    def check_cache(self):
+        c, n, bits = self.cache, self.n, self.bits
+        kc = unpack_stream(c.k_codes.cpu().numpy(), bits)
+        vc = unpack_stream(c.v_codes.cpu().numpy(), bits)
+        kn, vn, km = Hn.u16(c.k_norm), Hn.u16(c.v_norm), Hn.u16(c.k_meta)
+        for b, h, kq, vq in self.oracle_units():
+            assert np.array_equal(kn[b, h, :n], kq["norm"]), "key norms"
+            assert np.array_equal(km[b, h, :n // W], kq["meta"]), "key (m, s)"
+            assert np.array_equal(kc[b, h, :n], kq["codes"]), f"key codes: {(kc[b, h, :n] != kq['codes']).sum()} differ"
+            assert np.array_equal(vn[b, h, :n], vq["norm"]), "value norms"
+            assert np.array_equal(vc[b, h, :n], vq["codes"]), f"value codes: {(vc[b, h, :n] != vq['codes']).sum()} differ"
+        mod = np.where(self.mod.numpy() > 2, 0, self.mod.numpy())
+        assert np.array_equal(c.modality.cpu().numpy()[:, :n], np.broadcast_to(mod, (self.w.batch, n)))
+
+    def oracle_attention(self):
+        w = self.w
+        G = w.group
+        out = np.zeros((w.batch, w.n_q_heads, D))
+        qf = O.half_to_float(Hn.u16(self.q)).astype(np.float64).reshape(w.batch, w.n_q_heads, D)
+        mod = self.mod.numpy()
+        for b, h, kq, vq in self.oracle_units():
+            kh = LO.dequant_keys(kq, self.signs.numpy())
+            vh = LO.dequant_values(vq, mod, self.R.numpy(), self.bits)
+            s = qf[b, h * G:(h + 1) * G] @ kh.T / np.sqrt(D)
+            p = np.exp(s - s.max(axis=1, keepdims=True))
+            out[b, h * G:(h + 1) * G] = (p / p.sum(axis=1, keepdims=True)) @ vh
+        return out
+
+    def gpu_attention(self, n_tokens=None):
+        w = self.w
+        out = torch.full((w.batch, w.n_q_heads, D), float("nan"), dtype=torch.float32, device="cuda")
+        B.ladder_decode_attention(self.cache, self.n if n_tokens is None else n_tokens, self.q.cuda(), self.d_signs,
+                                  self.d_R, out)
+        torch.cuda.synchronize()
+        return out.cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_quantisers_bit_exact_and_decode_close(bits):
+    """Two sequences, four KV heads, 20 windows with all three modalities."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=2, prefix_text=40, video_chunk=150, audio_chunk=50)
+    c = LadderCase(w, bits, 640)
+    c.check_cache()
+    print(f"K{bits}V{bits} decode:", Hn.assert_attention_close(c.gpu_attention(), c.oracle_attention()))
+
+
+def test_two_bit_ladder_equals_the_hot_path_cache():
+    """At 2 bits the ladder cache holds the codes, norms and (m, s) of the 2-bit hot path (exported canonical arrays)."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], n_tokens=256)
+    c = LadderCase(w, 2, 256)
+    hot = Hn.Case(w, n_tokens=256)
+    e = {k: v.cpu() for k, v in hot.gpu_export(0).items()}
+    cap = hot.cache.capacity
+    # the hot path's canonical code bytes hold channel c at bits 2 (c % 4) of byte c / 4: the same bit stream
+    assert np.array_equal(e["k_codes"].numpy().reshape(1, 4, cap, 32)[:, :, :256], c.cache.k_codes.cpu().numpy()[:, :, :256])
+    assert np.array_equal(e["v_codes"].numpy().reshape(1, 4, cap, 32)[:, :, :256], c.cache.v_codes.cpu().numpy()[:, :, :256])
+    assert np.array_equal(Hn.u16(e["k_norm"]).reshape(1, 4, cap)[:, :, :256], Hn.u16(c.cache.k_norm)[:, :, :256])
+    assert np.array_equal(Hn.u16(e["k_meta"]).reshape(1, 4, cap // W, D, 2)[:, :, :8], Hn.u16(c.cache.k_meta)[:, :, :8])
+    got = c.gpu_attention()
+    ref, _ = hot.oracle_attention(0)
+    Hn.assert_attention_close(got, ref)
+
+
+@pytest.mark.parametrize("bits", [3, 4])
+def test_degenerate_inputs(bits):
+    """Zero vectors (norm 0), a constant channel (step 0), a window whose keys are all equal, modality ids above 2."""
+    w = WL.scaled(WL.WORKLOADS["tiny"], n_tokens=128)
+    k, v = WL.gen_kv(w, 0, n_tokens=128)
+    k, v = k.clone(), v.clone()
+    k[0, 0, 5] = 0; v[0, 0, 5] = 0; v[0, 0, 77] = 0
+    k[0, 0, 32:64] = k[0, 0, 32]                      # every channel constant over window 1
+    k[0, 0, 64:96, 3] = 0                             # one channel of the input zero over window 2
+    mod = WL.modality_layout(w, 128).clone()
+    mod[10:20] = 9
+    c = LadderCase(w, bits, 128, modality=mod, k=k, v=v)
+    c.check_cache()
+    Hn.assert_attention_close(c.gpu_attention(), c.oracle_attention())
+
+
+def test_prefix_of_the_cache_and_empty_prefix():
+    """Decode over the first windows only; n_tokens = 0 launches and writes zeros (empty softmax)."""
+    w = WL.scaled(WL.WORKLOADS["tiny"], n_tokens=256)
+    c = LadderCase(w, 3, 256)
+    full = c.gpu_attention()
+    short = LadderCase(w, 3, 96, k=c.k[:, :, :96].contiguous(), v=c.v[:, :, :96].contiguous(), modality=c.mod[:96].contiguous())
+    assert np.array_equal(c.gpu_attention(96), short.gpu_attention())
+    assert not np.array_equal(full, short.gpu_attention())
+    assert np.array_equal(c.gpu_attention(0), np.zeros_like(full))
+
+
+def test_error_falls_with_the_width_on_the_gpu_cache():
+    """Ladder ordering measured on the GPU's own caches: attention error against the unquantised fp64 attention
+    falls from 2 to 3 to 4 bits."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], n_tokens=1024)
+    errs = []
+    for bits in (2, 3, 4):
+        c = LadderCase(w, bits, 1024)
+        G = w.group
+        qf = O.half_to_float(Hn.u16(c.q)).astype(np.float64).reshape(1, w.n_q_heads, D)
+        kf = O.half_to_float(Hn.u16(c.k)).astype(np.float64).reshape(1, w.n_kv_heads, 1024, D)
+        vf = O.half_to_float(Hn.u16(c.v)).astype(np.float64).reshape(1, w.n_kv_heads, 1024, D)
+        ref = np.zeros((1, w.n_q_heads, D))
+        for h in range(w.n_kv_heads):
+            s = qf[0, h * G:(h + 1) * G] @ kf[0, h].T / np.sqrt(D)
+            p = np.exp(s - s.max(axis=1, keepdims=True))
+            ref[0, h * G:(h + 1) * G] = (p / p.sum(axis=1, keepdims=True)) @ vf[0, h]
+        got = c.gpu_attention()
+        errs.append(np.linalg.norm(got - ref) / np.linalg.norm(ref))
+    print("attention rel-L2 error vs fp16 cache at 2/3/4 bits:", errs)
+    assert errs[0] > errs[1] > errs[2]
