@@ -65,6 +65,18 @@ okq_status okq_ladder_decode_attention(const okq_ladder_cache* cache, int32_t n_
                                        float sm_scale, const float* signs, const float* R, int32_t n_R,
                                        float* out, void* stream);
 
+/* TurboQuant baseline codec (the paper's Preliminaries, Eq. 2 and Eq. 3), for the synthetic error comparison against
+ * OmniKVQuant at equal code width: per vector an fp16 norm, the randomised Hadamard rotation and the nearest level
+ * of the same fixed codebook; no window statistics and no modality rotation, the same for keys and values.
+ * x_fp16: device fp16 [n_vectors][128] contiguous; codes: device uint8 [n_vectors][16 * bits] (bit stream as above);
+ * norms: device fp16 [n_vectors].  n_vectors = 0 is a no-op. */
+okq_status okq_turboquant_encode(const void* x_fp16, int64_t n_vectors, int32_t bits, const float* signs, uint8_t* codes,
+                                 void* norms, void* stream);
+
+/* x_hat = |x| H^T level[code] as device float [n_vectors][128]. */
+okq_status okq_turboquant_decode(const uint8_t* codes, const void* norms, int64_t n_vectors, int32_t bits,
+                                 const float* signs, float* x_hat, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -117,6 +117,10 @@ def lib():
         L.okq_ladder_decode_attention.restype = C.c_int
         L.okq_ladder_decode_attention.argtypes = [C.POINTER(okq_ladder_cache), C.c_int32, C.c_void_p, C.c_float, C.c_void_p,
                                                   C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.okq_turboquant_encode.restype = C.c_int
+        L.okq_turboquant_encode.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.okq_turboquant_decode.restype = C.c_int
+        L.okq_turboquant_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -128,7 +132,7 @@ def exported_symbols():
             "okq_decode_attention_noalloc", "okq_quantize_values_bulk", "okq_debug_bulk_timeout", "okq_cache_export_mx",
             "okq_calib_workspace_bytes", "okq_calib_attention_weights", "okq_calib_moments", "okq_calib_rotation",
             "okq_ladder_codebook", "okq_ladder_quantize_keys", "okq_ladder_quantize_values",
-            "okq_ladder_decode_attention"]
+            "okq_ladder_decode_attention", "okq_turboquant_encode", "okq_turboquant_decode"]
 
 
 def _ptr(t) -> int:
@@ -370,3 +374,22 @@ def ladder_decode_attention(cache: LadderCache, n_tokens: int, q, signs, R, out,
     scale = HEAD_DIM ** -0.5 if sm_scale is None else sm_scale
     _check(lib().okq_ladder_decode_attention(C.byref(cache.c), n_tokens, _ptr(q), scale, _ptr(signs), _ptr(R), n_R,
                                              _ptr(out), _stream(stream)), "okq_ladder_decode_attention")
+
+
+def turboquant_encode(x: torch.Tensor, signs: torch.Tensor, bits: int, stream=None):
+    """x: fp16 [n, 128] contiguous -> (codes uint8 [n, 16 * bits], norms fp16 [n])."""
+    assert x.dtype == torch.float16 and x.is_contiguous() and x.shape[-1] == HEAD_DIM
+    n = x.numel() // HEAD_DIM
+    codes = torch.empty((n, 16 * bits), dtype=torch.uint8, device=x.device)
+    norms = torch.empty((n,), dtype=torch.float16, device=x.device)
+    _check(lib().okq_turboquant_encode(_ptr(x), n, bits, _ptr(signs), _ptr(codes), _ptr(norms), _stream(stream)),
+           "okq_turboquant_encode")
+    return codes, norms
+
+
+def turboquant_decode(codes: torch.Tensor, norms: torch.Tensor, signs: torch.Tensor, bits: int, stream=None):
+    n = norms.numel()
+    x_hat = torch.empty((n, HEAD_DIM), dtype=torch.float32, device=codes.device)
+    _check(lib().okq_turboquant_decode(_ptr(codes), _ptr(norms), n, bits, _ptr(signs), _ptr(x_hat), _stream(stream)),
+           "okq_turboquant_decode")
+    return x_hat

@@ -339,6 +339,57 @@ __global__ void __launch_bounds__(LD_THREADS) k_ladder_decode(LadderView cv, int
   }
 }
 
+// TurboQuant codec (Preliminaries, Eq. 2-3): norm, randomised Hadamard rotation, nearest level of the fixed codebook;
+// no window statistics, no modality rotation.  32 vectors per block of 128 threads.
+__global__ void __launch_bounds__(128) k_turboquant_encode(const __half* __restrict__ x, long long n, int bits,
+                                                           const float* __restrict__ signs, unsigned char* __restrict__ codes,
+                                                           __half* __restrict__ norms) {
+  __shared__ unsigned char code[W][D];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const long long base = (long long)blockIdx.x * W;
+  const float4 sg = *reinterpret_cast<const float4*>(signs + 4 * lane);
+  const float* th = c_thresholds[bits - 2];
+  const int nth = (1 << bits) - 1;
+  for (int kk = 0; kk < 8; kk++) {
+    const int i = warp * 8 + kk;
+    if (base + i >= n) break;
+    const float4 v = load_row4(x + (base + i) * D, lane);
+    const float nrm = warp_norm(v);
+    const __half nh = __float2half_rn(nrm);
+    const float nf = __half2float(nh);
+    const float cinv = nf != 0.0f ? __fdiv_rn(RSQRT_D, nf) : 0.0f;
+    const float4 y = warp_fwht(make_float4(__fmul_rn(sg.x, v.x), __fmul_rn(sg.y, v.y), __fmul_rn(sg.z, v.z), __fmul_rn(sg.w, v.w)), lane);
+    const float z[4] = {nf != 0.0f ? __fmul_rn(y.x, cinv) : 0.0f, nf != 0.0f ? __fmul_rn(y.y, cinv) : 0.0f,
+                        nf != 0.0f ? __fmul_rn(y.z, cinv) : 0.0f, nf != 0.0f ? __fmul_rn(y.w, cinv) : 0.0f};
+#pragma unroll
+    for (int k4 = 0; k4 < 4; k4++) {
+      int cd = 0;
+      for (int j = 0; j < nth; j++) cd += z[k4] > th[j];
+      code[i][4 * lane + k4] = (unsigned char)cd;
+    }
+    if (lane == 0) norms[base + i] = nh;
+  }
+  __syncthreads();
+  const int i = tid >> 2, part = tid & 3;
+  if (base + i < n) pack_quarter(&code[i][32 * part], bits, codes + (base + i) * 16 * bits + 4 * bits * part);
+}
+
+// x_hat = |x| H^T level[code], H^T y = diag(signs) Had y / sqrt(128); one warp per vector
+__global__ void __launch_bounds__(128) k_turboquant_decode(const unsigned char* __restrict__ codes, const __half* __restrict__ norms,
+                                                           long long n, int bits, const float* __restrict__ signs,
+                                                           float* __restrict__ x_hat) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long i = (long long)blockIdx.x * 4 + warp;
+  if (i >= n) return;
+  const unsigned char* row = codes + i * 16 * bits;
+  const float* lv = c_levels[bits - 2];
+  const float4 y = warp_fwht(make_float4(lv[load_code(row, bits, 4 * lane + 0)], lv[load_code(row, bits, 4 * lane + 1)],
+                                         lv[load_code(row, bits, 4 * lane + 2)], lv[load_code(row, bits, 4 * lane + 3)]), lane);
+  const float4 sg = *reinterpret_cast<const float4*>(signs + 4 * lane);
+  const float f = RSQRT_D * __half2float(norms[i]);
+  *reinterpret_cast<float4*>(x_hat + i * D + 4 * lane) = make_float4(sg.x * y.x * f, sg.y * y.y * f, sg.z * y.z * f, sg.w * y.w * f);
+}
+
 okq_status check_ladder(const okq_ladder_cache* c, int n_tokens) {
   if (!c) return OKQ_ERR_INVALID_ARG;
   if (c->bits < 2 || c->bits > 4) return OKQ_ERR_UNSUPPORTED;
@@ -417,6 +468,30 @@ okq_status okq_ladder_decode_attention(const okq_ladder_cache* cache, int32_t n_
   }
   k_ladder_decode<<<dim3(cache->n_kv_heads, cache->batch), LD_THREADS, sizeof(DecodeSmemL), static_cast<cudaStream_t>(stream)>>>(
       ladder_view(cache), n_tokens, static_cast<const __half*>(q), sm_scale, signs, R, n_R, out);
+  return launch_status();
+}
+
+okq_status okq_turboquant_encode(const void* x_fp16, int64_t n_vectors, int32_t bits, const float* signs, uint8_t* codes,
+                                 void* norms, void* stream) {
+  if (bits < 2 || bits > 4) return OKQ_ERR_UNSUPPORTED;
+  if (n_vectors < 0 || !x_fp16 || !signs || !codes || !norms) return OKQ_ERR_INVALID_ARG;
+  if (!aligned16(x_fp16) || !aligned16(signs) || !aligned16(codes)) return OKQ_ERR_ALIGNMENT;
+  if (n_vectors == 0) return OKQ_OK;
+  if ((n_vectors + W - 1) / W > 0x7fffffffLL) return OKQ_ERR_CAPACITY;
+  k_turboquant_encode<<<(unsigned)((n_vectors + W - 1) / W), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const __half*>(x_fp16), n_vectors, bits, signs, codes, static_cast<__half*>(norms));
+  return launch_status();
+}
+
+okq_status okq_turboquant_decode(const uint8_t* codes, const void* norms, int64_t n_vectors, int32_t bits,
+                                 const float* signs, float* x_hat, void* stream) {
+  if (bits < 2 || bits > 4) return OKQ_ERR_UNSUPPORTED;
+  if (n_vectors < 0 || !codes || !norms || !signs || !x_hat) return OKQ_ERR_INVALID_ARG;
+  if (!aligned16(codes) || !aligned16(signs) || !aligned16(x_hat)) return OKQ_ERR_ALIGNMENT;
+  if (n_vectors == 0) return OKQ_OK;
+  if ((n_vectors + 3) / 4 > 0x7fffffffLL) return OKQ_ERR_CAPACITY;
+  k_turboquant_decode<<<(unsigned)((n_vectors + 3) / 4), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+      codes, static_cast<const __half*>(norms), n_vectors, bits, signs, x_hat);
   return launch_status();
 }
 

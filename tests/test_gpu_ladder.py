@@ -158,3 +158,63 @@ def test_error_falls_with_the_width_on_the_gpu_cache():
         errs.append(np.linalg.norm(got - ref) / np.linalg.norm(ref))
     print("attention rel-L2 error vs fp16 cache at 2/3/4 bits:", errs)
     assert errs[0] > errs[1] > errs[2]
+
+
+# ---------------------------------------------------------------- TurboQuant baseline codec
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_turboquant_codec_against_the_oracle(bits):
+    """Codes and norms bit for bit; the reconstruction within fp32 rounding of the oracle's fp64 one.  n is not a
+    multiple of the 32 vectors a block takes; one vector is zero."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], n_tokens=1024)
+    k, _ = WL.gen_kv(w, 0, n_tokens=1024)
+    x = k[0, 1, :1000 + bits].clone().contiguous()
+    x[17] = 0
+    signs = WL.gen_signs(w, 0)
+    codes, norms = B.turboquant_encode(x.cuda(), signs.cuda(), bits)
+    x_hat = B.turboquant_decode(codes, norms, signs.cuda(), bits)
+    torch.cuda.synchronize()
+    ocodes, onorm = LO.turboquant_encode(Hn.u16(x), signs.numpy(), bits)
+    assert np.array_equal(Hn.u16(norms), onorm)
+    assert np.array_equal(unpack_stream(codes.cpu().numpy(), bits), ocodes)
+    ref = LO.turboquant_decode(ocodes, onorm, signs.numpy(), bits)
+    got = x_hat.cpu().numpy().astype(np.float64)
+    assert np.abs(got - ref).max() <= 2e-6 * np.abs(ref).max()
+    assert (got[17] == 0).all()
+
+
+def test_error_table_from_the_gpu_caches():
+    """The error-comparison table re-run on caches the GPU wrote: reconstruction MSE of the keys, attention KL and
+    output MSE (fp64, from the exported codes) of TurboQuant K2/V2, K3/V2 and OmniKVQuant K2V2 with fp16 (m, s);
+    every metric of OmniKVQuant lies below TurboQuant at the same code width, as in the paper's table."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=1, n_tokens=2048)
+    c = LadderCase(w, 2, 2048)
+    signs, R, mod = c.signs.numpy(), c.R.numpy(), c.mod.numpy()
+    kf = O.half_to_float(Hn.u16(c.k[0, 0])).astype(np.float64).reshape(2048, D)
+    vf = O.half_to_float(Hn.u16(c.v[0, 0])).astype(np.float64).reshape(2048, D)
+    qf = O.half_to_float(Hn.u16(c.q[0, :w.group])).astype(np.float64).reshape(w.group, D)
+
+    def softmax(s):
+        p = np.exp(s - s.max(axis=-1, keepdims=True))
+        return p / p.sum(axis=-1, keepdims=True)
+
+    def metrics(k_hat, v_hat):
+        p, p_hat = softmax(qf @ kf.T / np.sqrt(D)), softmax(qf @ k_hat.T / np.sqrt(D))
+        return (float(((kf - k_hat) ** 2).sum(axis=1).mean()),
+                float((p * (np.log(p + 1e-300) - np.log(p_hat + 1e-300))).sum(axis=1).mean()),
+                float((((p @ vf) - (p_hat @ v_hat)) ** 2).sum(axis=1).mean()))
+
+    def tq(x, bits):
+        codes, norms = B.turboquant_encode(x.contiguous().cuda(), c.d_signs, bits)
+        return B.turboquant_decode(codes, norms, c.d_signs, bits).cpu().numpy().astype(np.float64)
+
+    kq = {"codes": unpack_stream(c.cache.k_codes.cpu().numpy(), 2)[0, 0, :2048], "norm": Hn.u16(c.cache.k_norm)[0, 0, :2048],
+          "meta": Hn.u16(c.cache.k_meta)[0, 0, :64]}
+    vq = {"codes": unpack_stream(c.cache.v_codes.cpu().numpy(), 2)[0, 0, :2048], "norm": Hn.u16(c.cache.v_norm)[0, 0, :2048]}
+    rows = {"TurboQuant K2/V2": metrics(tq(c.k[0, 0], 2), tq(c.v[0, 0], 2)),
+            "TurboQuant K3/V2": metrics(tq(c.k[0, 0], 3), tq(c.v[0, 0], 2)),
+            "OmniKVQuant K2V2": metrics(LO.dequant_keys(kq, signs), LO.dequant_values(vq, mod, R, 2))}
+    for name, (r, kl, o) in rows.items():
+        print(f"{name:18s} recon MSE {r:9.4f}  attn KL {kl:9.5f}  output MSE {o:9.6f}")
+    for i in range(3):
+        assert rows["OmniKVQuant K2V2"][i] < rows["TurboQuant K2/V2"][i]
+    assert rows["OmniKVQuant K2V2"][0] < rows["TurboQuant K3/V2"][0] < rows["TurboQuant K2/V2"][0]
