@@ -206,6 +206,59 @@ def run_prefill(args, w, B, dev, rank, emit=True):
         print(json.dumps(line), flush=True)
 
 
+def run_ladder(args, B, dev, rank, emit=True):
+    """Secondary measurement: the bit-width ladder entry points (K2V2 / K3V3 / K4V4 over the canonical bit-stream
+    cache; plain CUDA-core kernels, one thread block per (sequence, KV head) in decode) and the TurboQuant codec,
+    on 64 sequences x 4 KV heads x 8192 tokens of the 7B layer shape.  GB/s of packed bytes read per decode."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=64, name="layer7b[batch=64]")
+    Bn, H, Hq, N = w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
+    k, v = WL.gen_kv(w, 0, device=dev)
+    q = WL.gen_queries(w, 0, device=dev)
+    signs = WL.gen_signs(w, 0).to(dev)
+    R = WL.gen_rotations(w, 0).unsqueeze(0).contiguous().to(dev)
+    mod = WL.modality_layout(w).unsqueeze(0).repeat(Bn, 1).contiguous().to(dev)
+    out = torch.empty((Bn, Hq, 128), dtype=torch.float32, device=dev)
+    peak, peak_kind = measured_peaks()
+    th = Bn * H * N
+
+    def timed(fn):
+        for _ in range(args.warmup):
+            fn()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in ev:
+            a.record(); fn(); b.record()
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in ev) / args.steps
+
+    res = {}
+    for bits in (2, 3, 4):
+        cache = B.LadderCache(Bn, H, Hq, N, bits, device=dev)
+        ms_k = timed(lambda: B.ladder_quantize_keys(cache, k, signs))
+        ms_v = timed(lambda: B.ladder_quantize_values(cache, v, mod, R))
+        ms_d = timed(lambda: B.ladder_decode_attention(cache, N, q, signs, R, out))
+        bytes_th = 2 * 16 * bits + 4 + 16            # codes, two fp16 norms, (m, s) of 128 channels per 32 tokens
+        res[f"K{bits}V{bits}"] = {"bytes_per_token_head": bytes_th, "bits_per_element": bytes_th * 8 / 256,
+                                  "quantize_keys_ms": ms_k, "quantize_values_ms": ms_v, "decode_ms": ms_d,
+                                  "decode_gbs": th * bytes_th / (ms_d * 1e-3) / 1e9,
+                                  "decode_frac": th * bytes_th / (ms_d * 1e-3) / 1e9 / peak}
+        del cache
+    x = k.reshape(-1, 128)
+    ms_e = timed(lambda: B.turboquant_encode(x, signs, 2))
+    codes, norms = B.turboquant_encode(x, signs, 2)
+    ms_x = timed(lambda: B.turboquant_decode(codes, norms, signs, 2))
+    res["turboquant_k2"] = {"encode_ms": ms_e, "decode_ms": ms_x, "encode_gbs": th * (256 + 34) / (ms_e * 1e-3) / 1e9}
+    line = {"metric": "bit-width ladder decode attention: packed bytes per second", "phase": "ladder", "unit": "GB/s",
+            "value": res["K4V4"]["decode_gbs"], "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": res["K4V4"]["decode_ms"], "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "batch": Bn, "n_kv_heads": H, "context": N}, "peak": peak, "peak_kind": peak_kind,
+            "ladder": res}
+    if not emit:
+        return line
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
 def quick_decode(B, dev, w, mx=False, caption=False, steps=8, warmup=3):
     """Short secondary measurement of the decode step (append + decode over all layers, inputs resident) on another
     workload / metadata format / schedule: step time, GB/s of packed bytes, split-K kernel time and fraction."""
@@ -317,10 +370,11 @@ def main():
                     help="streaming schedule of the cache: window = pack every 32 tokens (the headline configuration), "
                          "caption = the paper's captioning schedule (keys every 128 tokens, values behind a 128-token "
                          "fp16 window; secondary measurement, no cpu_baseline)")
-    ap.add_argument("--phase", default="decode", choices=["decode", "prefill", "calib"],
+    ap.add_argument("--phase", default="decode", choices=["decode", "prefill", "calib", "ladder"],
                     help="decode: the headline decode step; prefill: bulk quantisation of a fresh fp16 K/V cache "
                          "(secondary measurement, default workload prefill7b); calib: offline calibration of the "
-                         "value rotations (secondary measurement)")
+                         "value rotations (secondary measurement); ladder: the K2V2 / K3V3 / K4V4 entry points and the "
+                         "TurboQuant codec (secondary measurement)")
     args = ap.parse_args()
     if args.workload is None:
         args.workload = "prefill7b" if args.phase == "prefill" else "step7b"
@@ -344,6 +398,8 @@ def main():
         return run_prefill(args, w, B, dev, rank)
     if args.phase == "calib":
         return run_calib(args, B, dev, rank)
+    if args.phase == "ladder":
+        return run_ladder(args, B, dev, rank)
 
     # ---- build the packed cache on the device (setup, untimed)
     L, Bn, H, Hq, N = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
@@ -554,7 +610,8 @@ def main():
                          ("caption", lambda: quick_decode(B, dev, w, caption=True)),
                          ("long7b", lambda: quick_decode(B, dev, WL.WORKLOADS["long7b"])),
                          ("step30b", lambda: quick_decode(B, dev, WL.WORKLOADS["step30b"], steps=4, warmup=2)),
-                         ("prefill", lambda: run_prefill(argparse.Namespace(steps=3, warmup=1), WL.WORKLOADS["prefill7b"], B, dev, 0, emit=False))):
+                         ("prefill", lambda: run_prefill(argparse.Namespace(steps=3, warmup=1), WL.WORKLOADS["prefill7b"], B, dev, 0, emit=False)),
+                         ("ladder", lambda: run_ladder(argparse.Namespace(steps=3, warmup=1), B, dev, 0, emit=False)["ladder"])):
             try:
                 r = fn()
                 if name == "prefill":

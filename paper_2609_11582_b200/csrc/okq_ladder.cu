@@ -134,11 +134,18 @@ __global__ void __launch_bounds__(128) k_ladder_keys(LadderView cv, const __half
   }
 }
 
+struct ValueSmem {
+  __align__(16) float x[W][D + 4];   // the window's value rows (fp32), 16-byte aligned rows
+  unsigned char code[W][D];
+  unsigned char mod[W];
+  float inv[W];
+  int uniform;
+};
+
 __global__ void __launch_bounds__(128) k_ladder_values(LadderView cv, const __half* __restrict__ v, long long sb, long long sh,
                                                        long long st, const unsigned char* __restrict__ modality, int n_tokens,
                                                        const float* __restrict__ R, int n_R) {
-  __shared__ QuantSmem sm;
-  __shared__ float inv[W];
+  __shared__ ValueSmem sm;
   const int win = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const size_t u = cv.unit(b, h);
@@ -147,6 +154,9 @@ __global__ void __launch_bounds__(128) k_ladder_values(LadderView cv, const __ha
     m = m > 2 ? 0 : m;
     sm.mod[tid] = (unsigned char)m;
     if (h == 0) cv.modality[(size_t)b * cv.capacity + win * W + tid] = (unsigned char)m;
+    const unsigned m0 = __shfl_sync(0xffffffffu, m, 0);
+    const int uni = __all_sync(0xffffffffu, m == m0);
+    if (tid == 0) sm.uniform = uni;
   }
   for (int kk = 0; kk < 8; kk++) {
     const int i = warp * 8 + kk;
@@ -154,26 +164,60 @@ __global__ void __launch_bounds__(128) k_ladder_values(LadderView cv, const __ha
     const float n = warp_norm(x);
     const __half nh = __float2half_rn(n);
     const float nf = __half2float(nh);
-    sm.z[i][4 * lane + 0] = x.x; sm.z[i][4 * lane + 1] = x.y;
-    sm.z[i][4 * lane + 2] = x.z; sm.z[i][4 * lane + 3] = x.w;
+    *reinterpret_cast<float4*>(&sm.x[i][4 * lane]) = x;
     if (lane == 0) {
       cv.v_norm[u * cv.capacity + (size_t)win * W + i] = nh;
-      inv[i] = nf != 0.0f ? __fdiv_rn(1.0f, nf) : 0.0f;
+      sm.inv[i] = nf != 0.0f ? __fdiv_rn(1.0f, nf) : 0.0f;
     }
   }
   __syncthreads();
   {
+    // thread = output coordinate c: z_c = (sum_k R_m[c][k] v_k) / norm as one fused-multiply-add chain in ascending k
     const int c = tid, nth = (1 << cv.bits) - 1;
     const float* Rset = R + (size_t)(n_R == 1 ? 0 : h) * 3 * D * D;
     const float* th = c_thresholds[cv.bits - 2];
-    for (int i = 0; i < W; i++) {
-      const float* Rrow = Rset + ((size_t)sm.mod[i] * D + c) * D;
-      float a = 0.0f;
-      for (int kq = 0; kq < D; kq++) a = __fmaf_rn(__ldg(Rrow + kq), sm.z[i][kq], a);
-      const float z = __fmul_rn(a, inv[i]);
-      int code = 0;
-      for (int j = 0; j < nth; j++) code += z > th[j];
-      sm.code[i][c] = (unsigned char)code;
+    if (sm.uniform) {   // one matrix for the window: every row element is read once for the 32 tokens
+      const float4* Rrow = reinterpret_cast<const float4*>(Rset + ((size_t)sm.mod[0] * D + c) * D);
+      float acc[W];
+#pragma unroll
+      for (int i = 0; i < W; i++) acc[i] = 0.0f;
+      for (int k4 = 0; k4 < D / 4; k4++) {
+        const float4 r4 = __ldg(Rrow + k4);
+#pragma unroll
+        for (int i = 0; i < W; i++) {
+          const float4 x4 = *reinterpret_cast<const float4*>(&sm.x[i][4 * k4]);
+          float a = acc[i];
+          a = __fmaf_rn(r4.x, x4.x, a);
+          a = __fmaf_rn(r4.y, x4.y, a);
+          a = __fmaf_rn(r4.z, x4.z, a);
+          a = __fmaf_rn(r4.w, x4.w, a);
+          acc[i] = a;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < W; i++) {
+        const float z = __fmul_rn(acc[i], sm.inv[i]);
+        int code = 0;
+        for (int j = 0; j < nth; j++) code += z > th[j];
+        sm.code[i][c] = (unsigned char)code;
+      }
+    } else {
+      for (int i = 0; i < W; i++) {
+        const float4* Rrow = reinterpret_cast<const float4*>(Rset + ((size_t)sm.mod[i] * D + c) * D);
+        float a = 0.0f;
+        for (int k4 = 0; k4 < D / 4; k4++) {
+          const float4 r4 = __ldg(Rrow + k4);
+          const float4 x4 = *reinterpret_cast<const float4*>(&sm.x[i][4 * k4]);
+          a = __fmaf_rn(r4.x, x4.x, a);
+          a = __fmaf_rn(r4.y, x4.y, a);
+          a = __fmaf_rn(r4.z, x4.z, a);
+          a = __fmaf_rn(r4.w, x4.w, a);
+        }
+        const float z = __fmul_rn(a, sm.inv[i]);
+        int code = 0;
+        for (int j = 0; j < nth; j++) code += z > th[j];
+        sm.code[i][c] = (unsigned char)code;
+      }
     }
   }
   __syncthreads();
@@ -203,6 +247,7 @@ struct DecodeSmemL {
   float acc[3][GP_L][D];      // end: rotated-basis sums per modality
   float linv[GP_L];
   unsigned char mod[W];
+  __align__(16) unsigned char kc[W * 64], vc[W * 64];   // the window's code rows (W * 16 * bits bytes each), staged
 };
 
 // grid (heads, batch), 256 threads: warp j = head j for the query rotation and the softmax; thread (c, hh) = channel
@@ -246,6 +291,13 @@ __global__ void __launch_bounds__(LD_THREADS) k_ladder_decode(LadderView cv, int
       sm.m[tid] = __half2float(meta[0]); sm.s[tid] = __half2float(meta[1]);
     }
     if (tid < W) sm.mod[tid] = cv.modality[(size_t)b * cv.capacity + (size_t)win * W + tid];
+    {   // the window's rows are contiguous: W * rb bytes = 2 * bits * 32 pieces of 16 bytes per side
+      const int n16 = W * rb / 16;
+      const uint4* ksrc = reinterpret_cast<const uint4*>(cv.k_codes + tok0 * rb);
+      const uint4* vsrc = reinterpret_cast<const uint4*>(cv.v_codes + tok0 * rb);
+      if (tid < n16) reinterpret_cast<uint4*>(sm.kc)[tid] = ksrc[tid];
+      else if (tid >= 128 && tid - 128 < n16) reinterpret_cast<uint4*>(sm.vc)[tid - 128] = vsrc[tid - 128];
+    }
     __syncthreads();
     {   // weights and bias of head `warp`
       float bsum = 0.f;
@@ -264,7 +316,7 @@ __global__ void __launch_bounds__(LD_THREADS) k_ladder_decode(LadderView cv, int
     // scores: warp w takes tokens 4 w .. 4 w + 3, a lane four channels
     for (int tt = 0; tt < 4; tt++) {
       const int t = 4 * warp + tt;
-      const unsigned char* row = cv.k_codes + (tok0 + t) * rb;
+      const unsigned char* row = sm.kc + t * rb;
       float cd[4];
 #pragma unroll
       for (int k4 = 0; k4 < 4; k4++) cd[k4] = (float)load_code(row, bits, 4 * lane + k4);
@@ -306,12 +358,17 @@ __global__ void __launch_bounds__(LD_THREADS) k_ladder_decode(LadderView cv, int
 #pragma unroll
         for (int j = 0; j < 4; j++) acc[m][j] *= al[j];
       for (int t = 0; t < W; t++) {
-        const float lv = sm.lev[load_code(cv.v_codes + (tok0 + t) * rb, bits, c)];
-        const int md = sm.mod[t];
+        const float lv = sm.lev[load_code(sm.vc + t * rb, bits, c)];
+        const int md = sm.mod[t];   // the same for every thread: a uniform branch around register-indexed sums
+        if (md == 0) {
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-          const float w = sm.sc[4 * hh + j][t] * lv;
-          if (md == 0) acc[0][j] += w; else if (md == 1) acc[1][j] += w; else acc[2][j] += w;
+          for (int j = 0; j < 4; j++) acc[0][j] = fmaf(sm.sc[4 * hh + j][t], lv, acc[0][j]);
+        } else if (md == 1) {
+#pragma unroll
+          for (int j = 0; j < 4; j++) acc[1][j] = fmaf(sm.sc[4 * hh + j][t], lv, acc[1][j]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; j++) acc[2][j] = fmaf(sm.sc[4 * hh + j][t], lv, acc[2][j]);
         }
       }
     }
