@@ -209,8 +209,8 @@ def run_prefill(args, w, B, dev, rank, emit=True):
 def run_ladder(args, B, dev, rank, emit=True):
     """Secondary measurement: the bit-width ladder entry points (K2V2 / K3V3 / K4V4 over the canonical bit-stream
     cache; plain CUDA-core kernels, one thread block per (sequence, KV head) in decode) and the TurboQuant codec,
-    on 64 sequences x 4 KV heads x 8192 tokens of the 7B layer shape.  GB/s of packed bytes read per decode."""
-    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=64, name="layer7b[batch=64]")
+    on 256 sequences x 4 KV heads x 8192 tokens of the 7B layer shape (1024 thread blocks in decode).  GB/s of packed bytes read per decode."""
+    w = WL.scaled(WL.WORKLOADS["layer7b"], batch=256, name="layer7b[batch=256]")
     Bn, H, Hq, N = w.batch, w.n_kv_heads, w.n_q_heads, w.n_tokens
     k, v = WL.gen_kv(w, 0, device=dev)
     q = WL.gen_queries(w, 0, device=dev)
