@@ -25,6 +25,7 @@
 // block-wide step; at the end the block merges its pairs' pieces into one partial per
 // (sequence, head) it touched.  The combine kernel merges the partials, adds the raw fp16 tail
 // tokens, applies R_m^T once per head and normalises.
+#include <type_traits>
 #include "okq_common.cuh"
 #include "okq_device.cuh"
 #include "okq_decode_shared.cuh"
@@ -341,10 +342,6 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
       const int mymod = wmod[lane];
       const int first = __shfl_sync(0xffffffffu, mymod, 0);
       const bool uniform = __all_sync(0xffffffffu, mymod == first);
-      unsigned present = uniform ? (1u << first)
-                                 : ((__any_sync(0xffffffffu, mymod == 0) ? 1u : 0u) |
-                                    (__any_sync(0xffffffffu, mymod == 1) ? 2u : 0u) |
-                                    (__any_sync(0xffffffffu, mymod == 2) ? 4u : 0u));
       const uint4 vc0 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 16 * vpiece_slot(lane));
       const uint4 vc1 = *reinterpret_cast<const uint4*>(st + OFF_VCODE + 16 * vpiece_slot(32 + lane));
       const uint32_t vw[8] = {vc0.x, vc0.y, vc0.z, vc0.w, vc1.x, vc1.y, vc1.z, vc1.w};
@@ -353,58 +350,99 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
       // (3a - b) / (2 (b - a)): weight of the bit-1 plane relative to the code plane
       constexpr float DELTA_REL = (3.0f * CB_INNER - CB_OUTER) / (2.0f * (CB_OUTER - CB_INNER));
       const __half2 drel = __float2half2_rn(DELTA_REL);
-      for (int pass = 0; pass < 3 && present; pass++) {
-        int m = (cur_mod >= 0 && (present >> cur_mod) & 1) ? cur_mod : (__ffs(present) - 1);
-        present &= ~(1u << m);
-        if (m != cur_mod) {
-          if (cur_mod >= 0) deposit(ho);
-          cur_mod = m;
-        }
-        uint32_t b0[4], b1[4];
-        unsigned halfmask = 3u;  // which 16-token halves hold a token of modality m
-        if (uniform) {
+      // the two bit-plane products of the numerators b0 (zero where a token is not of the current modality) over
+      // the 16-token halves named by halfmask, and the weight sum
+      auto half_products = [&](const uint32_t (&b0)[4], const uint32_t (&b1)[4], auto kv_c) {
+        constexpr int kv = decltype(kv_c)::value;
+        constexpr uint32_t mA = 0x00030003u << (4 * kv), mB = 0x000c000cu << (4 * kv);
+        constexpr uint32_t nA = 0x00020002u << (4 * kv), nB = 0x00080008u << (4 * kv);
+        const uint32_t p0 = b0[2 * kv], p1 = b0[2 * kv + 1], q0 = b1[2 * kv], q1 = b1[2 * kv + 1];
+        // the two bit-plane products of one m-tile hit the same accumulator: keep them four
+        // MMAs apart so the second never waits for the first
 #pragma unroll
-          for (int nu = 0; nu < 4; nu++) b0[nu] = pb[nu];
-        } else {
-          bool any_lo = false, any_hi = false;
+        for (int mq = 0; mq < 8; mq += 4) {
+          uint32_t w8[4];
 #pragma unroll
-          for (int nu = 0; nu < 4; nu++) {
-            const bool k0 = wmod[8 * nu + 2 * t] == m, k1 = wmod[8 * nu + 2 * t + 1] == m;
-            b0[nu] = pb[nu] & ((k0 ? 0x0000ffffu : 0u) | (k1 ? 0xffff0000u : 0u));
-            if (nu < 2) any_lo |= (k0 | k1); else any_hi |= (k0 | k1);
+          for (int i = 0; i < 4; i++) {
+            const uint32_t w = vw[mq + i];
+            w8[i] = w >> 8;
+            mma16816(acc[mq + i], w & mA, w8[i] & mA, w & mB, w8[i] & mB, p0, p1);
           }
-          halfmask = (__any_sync(0xffffffffu, any_lo) ? 1u : 0u) | (__any_sync(0xffffffffu, any_hi) ? 2u : 0u);
+#pragma unroll
+          for (int i = 0; i < 4; i++) {
+            const uint32_t w = vw[mq + i];
+            mma16816(acc[mq + i], w & nA, w8[i] & nA, w & nB, w8[i] & nB, q0, q1);
+          }
         }
+      };
+      auto products = [&](const uint32_t (&b0)[4], unsigned halfmask, auto whole) {
+        uint32_t b1[4];
 #pragma unroll
         for (int nu = 0; nu < 4; nu++) {
           b1[nu] = h2u(__hmul2(u2h(b0[nu]), drel));
           float2 pf = __half22float2(u2h(b0[nu]));   // weight sum from the rounded numerators
           run_S = fmaf(pf.x + pf.y, (float)(1 << (2 * nu)) * (1.0f / 64.0f), run_S);
         }
+        if constexpr (decltype(whole)::value) {   // both halves, straight-line, compile-time masks
+          half_products(b0, b1, std::integral_constant<int, 0>{});
+          half_products(b0, b1, std::integral_constant<int, 1>{});
+        } else {
 #pragma unroll 1   // rolled on purpose: unrolling both halves makes ptxas spill the accumulators
-        for (int kv = 0; kv < 2; kv++) {
-          if (!((halfmask >> kv) & 1)) continue;
-          const uint32_t mA = 0x00030003u << (4 * kv), mB = 0x000c000cu << (4 * kv);
-          const uint32_t nA = 0x00020002u << (4 * kv), nB = 0x00080008u << (4 * kv);
-          const uint32_t p0 = kv ? b0[2] : b0[0], p1 = kv ? b0[3] : b0[1];
-          const uint32_t q0 = kv ? b1[2] : b1[0], q1 = kv ? b1[3] : b1[1];
-          // the two bit-plane products of one m-tile hit the same accumulator: keep them four
-          // MMAs apart so the second never waits for the first
+          for (int kv = 0; kv < 2; kv++) {
+            if (!((halfmask >> kv) & 1)) continue;
+            const uint32_t mA = 0x00030003u << (4 * kv), mB = 0x000c000cu << (4 * kv);
+            const uint32_t nA = 0x00020002u << (4 * kv), nB = 0x00080008u << (4 * kv);
+            const uint32_t p0 = kv ? b0[2] : b0[0], p1 = kv ? b0[3] : b0[1];
+            const uint32_t q0 = kv ? b1[2] : b1[0], q1 = kv ? b1[3] : b1[1];
 #pragma unroll
-          for (int mq = 0; mq < 8; mq += 4) {
-            uint32_t w8[4];
+            for (int mq = 0; mq < 8; mq += 4) {
+              uint32_t w8[4];
 #pragma unroll
-            for (int i = 0; i < 4; i++) {
-              const uint32_t w = vw[mq + i];
-              w8[i] = w >> 8;
-              mma16816(acc[mq + i], w & mA, w8[i] & mA, w & mB, w8[i] & mB, p0, p1);
-            }
+              for (int i = 0; i < 4; i++) {
+                const uint32_t w = vw[mq + i];
+                w8[i] = w >> 8;
+                mma16816(acc[mq + i], w & mA, w8[i] & mA, w & mB, w8[i] & mB, p0, p1);
+              }
 #pragma unroll
-            for (int i = 0; i < 4; i++) {
-              const uint32_t w = vw[mq + i];
-              mma16816(acc[mq + i], w & nA, w8[i] & nA, w & nB, w8[i] & nB, q0, q1);
+              for (int i = 0; i < 4; i++) {
+                const uint32_t w = vw[mq + i];
+                mma16816(acc[mq + i], w & nA, w8[i] & nA, w & nB, w8[i] & nB, q0, q1);
+              }
             }
           }
+        }
+      };
+      if (uniform && first == cur_mod) {
+        // the common case: every token of the window belongs to the modality the registers hold
+        products(pb, 3u, std::true_type{});
+      } else {
+        unsigned present = uniform ? (1u << first)
+                                   : ((__any_sync(0xffffffffu, mymod == 0) ? 1u : 0u) |
+                                      (__any_sync(0xffffffffu, mymod == 1) ? 2u : 0u) |
+                                      (__any_sync(0xffffffffu, mymod == 2) ? 4u : 0u));
+        for (int pass = 0; pass < 3 && present; pass++) {
+          int m = (cur_mod >= 0 && (present >> cur_mod) & 1) ? cur_mod : (__ffs(present) - 1);
+          present &= ~(1u << m);
+          if (m != cur_mod) {
+            if (cur_mod >= 0) deposit(ho);
+            cur_mod = m;
+          }
+          uint32_t b0[4];
+          unsigned halfmask = 3u;  // which 16-token halves hold a token of modality m
+          if (uniform) {
+#pragma unroll
+            for (int nu = 0; nu < 4; nu++) b0[nu] = pb[nu];
+          } else {
+            bool any_lo = false, any_hi = false;
+#pragma unroll
+            for (int nu = 0; nu < 4; nu++) {
+              const bool k0 = wmod[8 * nu + 2 * t] == m, k1 = wmod[8 * nu + 2 * t + 1] == m;
+              b0[nu] = pb[nu] & ((k0 ? 0x0000ffffu : 0u) | (k1 ? 0xffff0000u : 0u));
+              if (nu < 2) any_lo |= (k0 | k1); else any_hi |= (k0 | k1);
+            }
+            halfmask = (__any_sync(0xffffffffu, any_lo) ? 1u : 0u) | (__any_sync(0xffffffffu, any_hi) ? 2u : 0u);
+          }
+          products(b0, halfmask, std::false_type{});
         }
       }
       // before the barrier: the score warp may overwrite this hand-off record right after it
