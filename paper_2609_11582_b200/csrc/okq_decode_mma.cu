@@ -141,52 +141,15 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
   const int g = lane >> 2, t = lane & 3;
   float run_m = -INFINITY, run_l = 0.f;
 
-  auto issue = [&](int k) {
-    if (k < sg.n_my) {
-      const int win = sg.w0 + k;
-      unsigned char* dst = sm.stage[pair][k % NSTAGE];
-      if (FMT == FMT_FP16) {
-        const unsigned char* src = sg.rec0 + (size_t)win * RECORD_BYTES;
-#pragma unroll
-        for (int i = 0; i < 6; i++) {
-          int c16 = lane + 32 * i;
-          if (c16 < RECORD_BYTES / 16) cp_async16(dst + 16 * c16, src + 16 * c16);
-        }
-      } else {
-        // body (16-byte aligned) behind the 512 bytes the decoded (m, s) will occupy; the 136
-        // metadata bytes are only 8-byte aligned
-        const unsigned char* body = sg.rec0 + mx_body_off(win);
-        const unsigned char* meta = sg.rec0 + mx_meta_off(win);
-#pragma unroll
-        for (int i = 0; i < 5; i++) {
-          int c16 = lane + 32 * i;
-          if (c16 < BODY_BYTES / 16) cp_async16(dst + META_BYTES_FP16 + 16 * c16, body + 16 * c16);
-        }
-        if (lane < MX_META_BYTES / 8) cp_async8(dst + STAGE_MX + 8 * lane, meta + 8 * lane);
-      }
-      if (lane < 2) cp_async16(dst + STAGE_MOD + 16 * lane, sg.mod0 + (size_t)win * W + 16 * lane);
-    }
-    cp_async_commit();
-  };
-#pragma unroll
-  for (int k = 0; k < PREFETCH; k++) issue(k);
   uint2 qreg[16];
   float fsc;
   query_fragments(sg.q, sg.signs, G, sm_scale, lane, qreg, fsc);   // while the first windows are on their way
+  pair_barrier(pair);   // the value warp has the first window in place
 
   for (int k = 0; k <= sg.n_my; k++) {
     if (k < sg.n_my) {
-      issue(k + PREFETCH);
-      cp_async_wait<PREFETCH>();
-      __syncwarp();
+      // copied (and, with MXFP4 metadata, expanded into the fp16 planes) by the value warp, complete before the last barrier
       unsigned char* st = sm.stage[pair][k % NSTAGE];
-      if (FMT == FMT_MXFP4) {   // decode the stored (m, s) into the fp16 planes of the staged image
-        uint2 m4, s4;
-        mx_decode_lane(st + STAGE_MX, lane, m4, s4);
-        *reinterpret_cast<uint2*>(st + OFF_KM + 8 * lane) = m4;
-        *reinterpret_cast<uint2*>(st + OFF_KS + 8 * lane) = s4;
-        __syncwarp();
-      }
       const uint4* mp = reinterpret_cast<const uint4*>(st + OFF_KM + 64 * t);
       const uint4* sp = reinterpret_cast<const uint4*>(st + OFF_KS + 64 * t);
       // bias sum_c q'_c m_c (two independent chains)
@@ -265,7 +228,6 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
     }
     pair_barrier(pair);
   }
-  cp_async_wait<0>();
   run_l += __shfl_xor_sync(0xffffffffu, run_l, 1);
   run_l += __shfl_xor_sync(0xffffffffu, run_l, 2);
   if (t == 0) {
@@ -289,6 +251,52 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
   // nothing deposited yet (the deposited registers themselves are only read where a maximum says so)
   if (lane < 3 * GP) (&sm.spill_m[pair][0][0])[lane] = -INFINITY;
   __syncwarp();
+  // The value warp also streams the records: it has registers to spare and the copies of window k + 2 are issued
+  // while it works on window k - 1; a window is complete (cp.async.wait_group) before the barrier after which the
+  // score warp reads it.
+  auto issue = [&](int k) {
+    if (k < sg.n_my) {
+      const int win = sg.w0 + k;
+      unsigned char* dst = sm.stage[pair][k % NSTAGE];
+      if (FMT == FMT_FP16) {
+        const unsigned char* src = sg.rec0 + (size_t)win * RECORD_BYTES;
+#pragma unroll
+        for (int i = 0; i < 6; i++) {
+          int c16 = lane + 32 * i;
+          if (c16 < RECORD_BYTES / 16) cp_async16(dst + 16 * c16, src + 16 * c16);
+        }
+      } else {
+        // body (16-byte aligned) behind the 512 bytes the decoded (m, s) will occupy; the 136
+        // metadata bytes are only 8-byte aligned
+        const unsigned char* body = sg.rec0 + mx_body_off(win);
+        const unsigned char* meta = sg.rec0 + mx_meta_off(win);
+#pragma unroll
+        for (int i = 0; i < 5; i++) {
+          int c16 = lane + 32 * i;
+          if (c16 < BODY_BYTES / 16) cp_async16(dst + META_BYTES_FP16 + 16 * c16, body + 16 * c16);
+        }
+        if (lane < MX_META_BYTES / 8) cp_async8(dst + STAGE_MX + 8 * lane, meta + 8 * lane);
+      }
+      if (lane < 2) cp_async16(dst + STAGE_MOD + 16 * lane, sg.mod0 + (size_t)win * W + 16 * lane);
+    }
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int k = 0; k < PREFETCH; k++) issue(k);
+  // with MXFP4 metadata: the stored (m, s) of a window that has landed, expanded into the fp16 planes of its staged image
+  auto expand_meta = [&](int k) {
+    if (FMT == FMT_MXFP4 && k < sg.n_my) {
+      __syncwarp();   // the other lanes' copies have landed too
+      unsigned char* st = sm.stage[pair][k % NSTAGE];
+      uint2 m4, s4;
+      mx_decode_lane(st + STAGE_MX, lane, m4, s4);
+      *reinterpret_cast<uint2*>(st + OFF_KM + 8 * lane) = m4;
+      *reinterpret_cast<uint2*>(st + OFF_KS + 8 * lane) = s4;
+    }
+  };
+  cp_async_wait<PREFETCH - 1>();
+  expand_meta(0);
+  pair_barrier(pair);   // window 0 is in place
 
   // Adds the live accumulators (which refer to the running maxima ho.m) to the current modality's sums in
   // shared memory and clears them.  Apart from modality changes this happens every FLUSH windows: the
@@ -327,6 +335,7 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
   };
 
   for (int k = 0; k <= sg.n_my; k++) {
+    issue(k + PREFETCH);
     if (k >= 1) {
       const unsigned char* st = sm.stage[pair][(k - 1) % NSTAGE];
       const Handoff& ho = sm.hand[pair][(k - 1) & 1];
@@ -448,8 +457,11 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
       // before the barrier: the score warp may overwrite this hand-off record right after it
       if (k == sg.n_my || ++since >= FLUSH) deposit(ho);
     }
+    cp_async_wait<1>();   // all but the copies just issued: window k + 1 is complete
+    expand_meta(k + 1);
     pair_barrier(pair);
   }
+  cp_async_wait<0>();
   // leave the three modalities' accumulators (each lane its own column) and their maxima in the pair's piece
   if (sg.keep) return;   // the block's merge reads this pair's sums where they are
 #pragma unroll 1
