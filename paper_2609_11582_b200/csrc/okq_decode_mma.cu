@@ -193,17 +193,20 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
       const uint32_t knu[4] = {kn4.x, kn4.y, kn4.z, kn4.w}, vnu[4] = {vn4.x, vn4.y, vn4.z, vn4.w};
       // the code sums carry 2^-24 (subnormal code operands), the bias sum does not
       const float bias0 = ((dbA[0] + dbB[0]) + (dbA[2] + dbB[2])) * 0x1p-24f, bias1 = bias0;
+      // sc = score / fsc: the head's scale fsc > 0 (query scaling, 1/sqrt(d), log2 e) enters the exponent below in
+      // one multiply-add and the maximum once
       float sc[4][2];
       float mx = -INFINITY;
 #pragma unroll
       for (int nu = 0; nu < 4; nu++) {
         float2 kn = __half22float2(u2h(knu[nu]));
-        sc[nu][0] = ((d[nu][0] + d[nu][2]) + bias0) * (kn.x * fsc);
-        sc[nu][1] = ((d[nu][1] + d[nu][3]) + bias1) * (kn.y * fsc);
+        sc[nu][0] = ((d[nu][0] + d[nu][2]) + bias0) * kn.x;
+        sc[nu][1] = ((d[nu][1] + d[nu][3]) + bias1) * kn.y;
         mx = fmaxf(mx, fmaxf(sc[nu][0], sc[nu][1]));
       }
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      mx *= fsc;
       // the reference maximum only moves when it is exceeded by more than 2^RESCALE_LOG2, so the
       // value accumulators are rescaled a few times per range instead of at every new maximum
       const float m_new = mx > run_m + RESCALE_LOG2 ? mx : run_m;
@@ -218,7 +221,7 @@ __device__ __forceinline__ void score_warp(MmaSmem<FMT>& sm, const Segment& sg, 
         float2 vn = __half22float2(u2h(vnu[nu]));
         const float off = (float)(6 - 2 * nu) - run_m;
         const float cinv = (float)(1 << (2 * nu)) * (1.0f / 64.0f);
-        float p0 = ex2(sc[nu][0] + off), p1 = ex2(sc[nu][1] + off);
+        float p0 = ex2(fmaf(sc[nu][0], fsc, off)), p1 = ex2(fmaf(sc[nu][1], fsc, off));
         run_l = fmaf(p0 + p1, cinv, run_l);
         pb[nu] = pack_sat(p0 * vn.x, p1 * vn.y);
       }
