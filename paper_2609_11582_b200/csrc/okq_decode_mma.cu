@@ -13,11 +13,13 @@
 //   * the value codebook {-b,-a,a,b} is affine in the two code bits:
 //     cb[c] = (b-a)*c + (3a-b)*bit1(c) - b, so two bit-plane products plus the running sum
 //     of the weights reproduce it exactly.
-// A CTA runs 8 warp pairs.  The "score" warp of a pair streams window records through a
-// cp.async ring, computes the scores and the online softmax (FlashAttention order) and hands
-// the fp16 numerators to its "value" warp through shared memory; the value warp accumulates
-// the codebook sums of the previous window meanwhile.  One named barrier per pair and
-// iteration keeps the two in step (no spin-waits anywhere).  Values accumulate in the rotated
+// A CTA runs 8 warp pairs.  The "score" warp of a pair computes the scores and the online
+// softmax (FlashAttention order) and hands the fp16 numerators to its "value" warp through
+// shared memory; the value warp accumulates the codebook sums of the previous window meanwhile
+// and streams the window records through a cp.async ring, two windows ahead of the score warp
+// (with MXFP4 metadata it also expands them into the fp16 planes).  One named barrier per pair
+// and iteration keeps the two in step (no spin-waits anywhere).  Windows whose tokens all belong
+// to the modality the registers hold take a straight-line path.  Values accumulate in the rotated
 // basis of the current modality, in registers for at most 32 windows at a time; each modality's
 // running sums live in shared memory.
 // The grid is persistent: CTA i owns an equal slice of the flattened (layer, sequence, head,
