@@ -273,8 +273,10 @@ __device__ __forceinline__ void value_warp(MmaSmem<FMT>& sm, const Segment& sg, 
       } else {
         // body (16-byte aligned) behind the 512 bytes the decoded (m, s) will occupy; the 136
         // metadata bytes are only 8-byte aligned
-        const unsigned char* body = sg.rec0 + mx_body_off(win);
-        const unsigned char* meta = sg.rec0 + mx_meta_off(win);
+        // two windows share one block [meta 0 | meta 1 | body 0 | body 1]: offsets in 32 bits
+        const uint32_t odd = (uint32_t)win & 1u, blk = ((uint32_t)win >> 1) * (uint32_t)MX_PAIR_BYTES;
+        const unsigned char* body = sg.rec0 + (blk + 2u * MX_META_BYTES + odd * (uint32_t)BODY_BYTES);
+        const unsigned char* meta = sg.rec0 + (blk + odd * (uint32_t)MX_META_BYTES);
 #pragma unroll
         for (int i = 0; i < 5; i++) {
           int c16 = lane + 32 * i;
