@@ -38,7 +38,7 @@ BYTES_PER_TOKEN_HEAD = 84          # 32 B key codes + 2 B key norm + 16 B (m, s)
 # 4-layer slice of the workload (176 MB of records, larger than L2) and divided by its token-heads;
 # traffic grows in proportion to the token-heads.  To be re-measured whenever the split-K kernel changes.
 NCU_DRAM_BYTES_PER_TOKEN_HEAD = 86.36
-NCU_DRAM_BYTES_PER_TOKEN_HEAD_MX = 75.37   # same capture with --meta mxfp4
+NCU_DRAM_BYTES_PER_TOKEN_HEAD_MX = 74.82   # same capture with --meta mxfp4
 
 
 def measured_peaks():
